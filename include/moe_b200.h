@@ -1,0 +1,131 @@
+/*
+ * moe_b200.h -- C ABI of the fused routed-MoE decode step for NVIDIA B200 (sm_100a).
+ *
+ * One call to moe_forward() runs one decode step of the complete routed
+ * Mixture-of-Experts operator of the paper (Section 3: top-k/quantize,
+ * up-projection, down-projection, reduce) in ONE persistent kernel launch:
+ *
+ *   router logits (Section 3.3) -> softmax or sigmoid(+selection bias) top-k
+ *   (Section 4.1) -> per-token 1x128 FP8 E4M3 quantisation of the input
+ *   (Section 4.1) -> gate/up projection against FP8 weights with 128x128 fp32
+ *   block scales, tokens on the MMA N dimension (Eq. 9) -> SiLU(gate)*up and
+ *   FP8 requantisation (Section 3.3, up-projection epilogue) -> down
+ *   projection -> top-k weighted reduction in fixed slot order (Section 3.2).
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers, row-major, contiguous, owned by
+ *     the caller; the library never frees or reallocates them.  Every pointer
+ *     must be 16-byte aligned.
+ *   - H and I must be multiples of 128, 1 <= top_k <= min(E, 32), E <= 512.
+ *   - W13 rows [0,I) of each expert are the gate projection, rows [I,2I) the
+ *     up projection.
+ *   - Calls are asynchronous on `stream`; nothing synchronises the host.
+ *   - Every function returns MOE_OK or a negative error code and never throws
+ *     or aborts; moe_last_error() returns a description of the most recent
+ *     failure on the calling thread.  Problems found on the device (a wait that
+ *     ran out) are recorded in the workspace and read with moe_sync_status().
+ *   - There is no CPU fallback: without a CUDA device of compute capability
+ *     10.x every entry point that needs one returns MOE_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef MOE_B200_H_
+#define MOE_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_plan* moe_plan_t;
+typedef void* moe_stream_t; /* a cudaStream_t */
+
+enum {
+    MOE_OK = 0,
+    MOE_ERR_ARG = -1,              /* null pointer, T out of range, ... */
+    MOE_ERR_SHAPE = -2,            /* H/I not multiples of 128, top_k or E out of range */
+    MOE_ERR_ALIGN = -3,            /* a pointer is not 16-byte aligned */
+    MOE_ERR_WORKSPACE = -4,        /* workspace missing or too small */
+    MOE_ERR_CUDA = -5,             /* a CUDA runtime/driver call failed */
+    MOE_ERR_OCCUPANCY = -6,        /* the persistent grid cannot be co-resident */
+    MOE_ERR_TIMEOUT = -7,          /* a device-side wait ran out (see moe_sync_status) */
+    MOE_ERR_UNSUPPORTED_ARCH = -8  /* no sm_100 device */
+};
+
+enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID_BIAS = 1 };
+
+/* Largest number of tokens one kernel launch handles; larger T is split into launches of this size. */
+#define MOE_MAX_TOKENS_PER_LAUNCH 64
+
+/*
+ * moe_plan: fix the layer shape and routing policy (Section 3.4: shape and
+ * schedule are fixed ahead of time, token count is a run-time argument).
+ *   H hidden size, E experts, I intermediate size, top_k experts per token,
+ *   scoring MOE_SCORE_*, renorm != 0 renormalises the selected weights.
+ * Queries the current device, checks that the persistent grid (one CTA per SM)
+ * is co-resident (Section 3.2, "verifies the realized occupancy") and stores
+ * host-side state only.  *out receives the plan; free it with moe_plan_destroy.
+ */
+int moe_plan(int H, int E, int I, int top_k, int scoring, int renorm, moe_plan_t* out);
+
+/* As moe_plan, plus the routed scaling factor multiplied into the routing weights (Section 4.1: 2.5 for the
+ * sigmoid policies; 1.0 otherwise). */
+int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float routed_scale, moe_plan_t* out);
+
+void moe_plan_destroy(moe_plan_t plan);
+
+/* Bytes of device scratch a call with up to T_max tokens needs (flags, logits, quantised activations,
+ * intermediate FP8 tile, split-K partials, per-slot outputs).  0 on invalid arguments. */
+size_t moe_workspace_bytes(moe_plan_t plan, int T_max);
+
+/* Zero the control words and flags of a workspace.  Must run once (stream-ordered) before the first
+ * moe_forward that uses the workspace, and again after an MOE_ERR_TIMEOUT.  `workspace` is device memory,
+ * 256-byte aligned, of at least moe_workspace_bytes() bytes. */
+int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes, moe_stream_t stream);
+
+/*
+ * moe_forward: one decode step for T tokens (Section 3; Eq. 9 for the projections).
+ *   hidden_bf16 [T,H] bf16          Wr_bf16 [E,H] bf16         sel_bias [E] fp32 or NULL (sigmoid policy only)
+ *   W13_fp8 [E,2I,H] E4M3 bytes     W13_scale [E,2I/128,H/128] fp32
+ *   W2_fp8  [E,H,I]  E4M3 bytes     W2_scale  [E,H/128,I/128] fp32
+ *   out_bf16 [T,H] bf16 (written)   workspace: see moe_workspace_init; sized for >= min(T,64) tokens
+ * All launches that share one workspace must be ordered on the device (same stream, or events): two calls
+ * that overlap on the GPU race on the scratch.  T > 64 is processed as consecutive launches of <= 64 tokens.
+ * Returns MOE_OK once the work is enqueued.
+ */
+int moe_forward(moe_plan_t plan, int T,
+                const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                const void* W13_fp8, const float* W13_scale,
+                const void* W2_fp8, const float* W2_scale,
+                void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream);
+
+/*
+ * moe_forward_debug: moe_forward, then copies (device to device, on `stream`) the routing and input
+ * quantisation results of the step into caller buffers; any of them may be NULL.  Requires T <= 64.
+ *   topk_ids [T,top_k] int32 (slot order: key descending, index ascending)   topk_w [T,top_k] fp32
+ *   xq [T,H] E4M3 bytes   xs [T,H/128] fp32   logits [T,E] fp32
+ */
+int moe_forward_debug(moe_plan_t plan, int T,
+                      const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                      const void* W13_fp8, const float* W13_scale,
+                      const void* W2_fp8, const float* W2_scale,
+                      void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream,
+                      int32_t* topk_ids, float* topk_w, uint8_t* xq, float* xs, float* logits);
+
+/* Synchronise `stream`, read the workspace's device status word and return MOE_OK, MOE_ERR_TIMEOUT or
+ * MOE_ERR_CUDA.  After MOE_ERR_TIMEOUT the workspace must be re-initialised. */
+int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream);
+
+/* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
+int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);
+
+/* Set the device-side wait limit in milliseconds (default 1000).  A wait that runs out makes the kernel
+ * record MOE_ERR_TIMEOUT and return; it never traps. */
+int moe_plan_set_timeout_ms(moe_plan_t plan, int ms);
+
+const char* moe_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H_ */

@@ -157,3 +157,19 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Decode bf16 bit patterns (uint16) to float64 (exact)."""
     b = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
     return b.view(np.float32).astype(np.float64)
+
+
+def route_and_quantize(hidden_bf16: np.ndarray, Wr_bf16: np.ndarray, bias: Optional[np.ndarray], top_k: int,
+                       scoring: int = SCORE_SOFTMAX, renorm: int = 1, routed_scale: float = 1.0, group: int = 128):
+    """Steps 1-5 only (logits, scores, top-k, weights, input quantisation).
+
+    Implemented by running the full oracle against one all-zero stand-in expert, so no step is duplicated here.
+    """
+    E, H = Wr_bf16.shape
+    z13 = np.zeros((1, 2 * group, H), np.uint8)
+    z2 = np.zeros((1, H, group), np.uint8)
+    s13 = np.ones((1, 2, H // group), np.float32)
+    s2 = np.ones((1, H // group, 1), np.float32)
+    r = moe_forward(hidden_bf16, Wr_bf16, bias, z13, s13, z2, s2, top_k=top_k, scoring=scoring, renorm=renorm,
+                    routed_scale=routed_scale, group=group, expert_map=np.zeros(E, np.int32))
+    return {k: r[k] for k in ("ids", "w", "margin", "logits", "xq", "xs")}

@@ -1,0 +1,177 @@
+"""Thin ctypes binding of the C ABI in include/moe_b200.h.
+
+Argument marshalling only: every step of the operator runs inside the CUDA library.
+Functions carry the names of the C entry points; `MoEPlan` is a small convenience
+wrapper that owns a plan and a torch-allocated workspace.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+SCORE_SOFTMAX = 0
+SCORE_SIGMOID_BIAS = 1
+
+EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
+           "moe_forward_debug", "moe_sync_status", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
+
+_lib = None
+
+
+class MoEError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"moe_b200 error {code}: {msg}")
+        self.code = code
+
+
+def lib_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libmoe_b200.so")
+
+
+def load_library():
+    """dlopen the in-tree CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise MoEError(-8, f"{path} is missing: run `python -m paper_2609_04244_b200.build` (needs nvcc); "
+                           "there is no CPU fallback")
+    lib = ctypes.CDLL(path)
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.moe_plan.restype = i
+    lib.moe_plan.argtypes = [i, i, i, i, i, i, ctypes.POINTER(vp)]
+    lib.moe_plan_ex.restype = i
+    lib.moe_plan_ex.argtypes = [i, i, i, i, i, i, f, ctypes.POINTER(vp)]
+    lib.moe_plan_destroy.restype = None
+    lib.moe_plan_destroy.argtypes = [vp]
+    lib.moe_workspace_bytes.restype = sz
+    lib.moe_workspace_bytes.argtypes = [vp, i]
+    lib.moe_workspace_init.restype = i
+    lib.moe_workspace_init.argtypes = [vp, vp, sz, vp]
+    lib.moe_forward.restype = i
+    lib.moe_forward.argtypes = [vp, i] + [vp] * 9 + [sz, vp]
+    lib.moe_forward_debug.restype = i
+    lib.moe_forward_debug.argtypes = [vp, i] + [vp] * 9 + [sz, vp] + [vp] * 5
+    lib.moe_sync_status.restype = i
+    lib.moe_sync_status.argtypes = [vp, vp, vp]
+    lib.moe_plan_info.restype = i
+    lib.moe_plan_info.argtypes = [vp, i] + [ctypes.POINTER(i)] * 4
+    lib.moe_plan_set_timeout_ms.restype = i
+    lib.moe_plan_set_timeout_ms.argtypes = [vp, i]
+    lib.moe_last_error.restype = ctypes.c_char_p
+    lib.moe_last_error.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise MoEError(rc, load_library().moe_last_error().decode())
+
+
+def _p(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise MoEError(-1, "tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def moe_plan(H: int, E: int, I: int, top_k: int, scoring: int, renorm: int, routed_scale: float = 1.0):
+    h = ctypes.c_void_p()
+    lib = load_library()
+    _check(lib.moe_plan_ex(H, E, I, top_k, scoring, renorm, ctypes.c_float(routed_scale), ctypes.byref(h)))
+    return h
+
+
+def moe_plan_destroy(plan) -> None:
+    load_library().moe_plan_destroy(plan)
+
+
+def moe_workspace_bytes(plan, T_max: int) -> int:
+    return int(load_library().moe_workspace_bytes(plan, T_max))
+
+
+def moe_workspace_init(plan, workspace: torch.Tensor, stream=None) -> None:
+    _check(load_library().moe_workspace_init(plan, _p(workspace), workspace.numel() * workspace.element_size(),
+                                             _stream(stream)))
+
+
+def moe_forward(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, workspace, stream=None) -> None:
+    _check(load_library().moe_forward(plan, T, _p(hidden), _p(Wr), _p(sel_bias), _p(W13q), _p(W13s), _p(W2q), _p(W2s),
+                                      _p(out), _p(workspace), workspace.numel() * workspace.element_size(),
+                                      _stream(stream)))
+
+
+def moe_forward_debug(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, workspace, stream=None,
+                      topk_ids=None, topk_w=None, xq=None, xs=None, logits=None) -> None:
+    _check(load_library().moe_forward_debug(plan, T, _p(hidden), _p(Wr), _p(sel_bias), _p(W13q), _p(W13s), _p(W2q),
+                                            _p(W2s), _p(out), _p(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream),
+                                            _p(topk_ids), _p(topk_w), _p(xq), _p(xs), _p(logits)))
+
+
+def moe_sync_status(plan, workspace, stream=None) -> None:
+    _check(load_library().moe_sync_status(plan, _p(workspace), _stream(stream)))
+
+
+def moe_plan_info(plan, T: int) -> dict:
+    g, s, n, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    _check(load_library().moe_plan_info(plan, T, ctypes.byref(g), ctypes.byref(s), ctypes.byref(n), ctypes.byref(b)))
+    return {"grid": g.value, "stages": s.value, "n_hw": n.value, "smem_bytes": b.value}
+
+
+class MoEPlan:
+    """Owns a plan handle and a workspace sized for `T_max` tokens on the current CUDA device."""
+
+    def __init__(self, H, E, I, top_k, scoring=SCORE_SOFTMAX, renorm=1, routed_scale=1.0, T_max=64):
+        self.H, self.E, self.I, self.top_k = H, E, I, top_k
+        self.handle = moe_plan(H, E, I, top_k, scoring, renorm, routed_scale)
+        self.workspace = torch.empty(moe_workspace_bytes(self.handle, T_max), dtype=torch.uint8, device="cuda")
+        moe_workspace_init(self.handle, self.workspace)
+
+    def forward(self, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out=None, stream=None):
+        T = hidden.shape[0]
+        if out is None:
+            out = torch.empty((T, self.H), dtype=torch.bfloat16, device=hidden.device)
+        moe_forward(self.handle, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, self.workspace, stream)
+        return out
+
+    def forward_debug(self, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, stream=None):
+        T, dev = hidden.shape[0], hidden.device
+        out = torch.empty((T, self.H), dtype=torch.bfloat16, device=dev)
+        dbg = {"ids": torch.empty((T, self.top_k), dtype=torch.int32, device=dev),
+               "w": torch.empty((T, self.top_k), dtype=torch.float32, device=dev),
+               "xq": torch.empty((T, self.H), dtype=torch.uint8, device=dev),
+               "xs": torch.empty((T, self.H // 128), dtype=torch.float32, device=dev),
+               "logits": torch.empty((T, self.E), dtype=torch.float32, device=dev)}
+        moe_forward_debug(self.handle, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, self.workspace, stream,
+                          dbg["ids"], dbg["w"], dbg["xq"], dbg["xs"], dbg["logits"])
+        dbg["out"] = out
+        return dbg
+
+    def sync_status(self, stream=None):
+        moe_sync_status(self.handle, self.workspace, stream)
+
+    def info(self, T):
+        return moe_plan_info(self.handle, T)
+
+    def close(self):
+        if self.handle is not None:
+            moe_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

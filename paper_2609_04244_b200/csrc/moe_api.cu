@@ -1,0 +1,352 @@
+// Host side of the C ABI declared in include/moe_b200.h: plan, workspace layout, TMA descriptors, launch.
+#include "moe_kernel.cuh"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "../../include/moe_b200.h"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    });
+    return fn;
+}
+
+// 2-D byte tensor [rows, cols] (cols contiguous), box = box_rows x 128 bytes, 128-byte swizzle.
+bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+    size_t ctrl, hq_flag, pu_flag, pd_flag, hb_cnt, flags_end;   // zero-initialised region = [0, flags_end)
+    size_t logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, total;
+};
+
+struct MapKey {
+    const void* ptr;
+    uint64_t rows, cols;
+    uint32_t box_rows;
+    bool operator==(const MapKey& o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+};
+
+}  // namespace
+
+struct moe_plan {
+    int H, E, I, K, scoring, renorm;
+    float routed_scale;
+    int device, sms, smem_optin;
+    unsigned long long timeout_ns;
+    std::mutex mu;
+    std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
+
+    int n_hw(int T) const { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
+    int cap(int T) const { return T < moe::kMaxTokens ? T : moe::kMaxTokens; }
+
+    WsLayout layout(int T_max) const {
+        const int Tc = cap(T_max), N = n_hw(Tc), G = sms;
+        WsLayout L;
+        size_t o = 0;
+        L.ctrl = o;     o += moe::kCtrlWords * 4;
+        L.hq_flag = o;  o += align_up((size_t)E * (I / 128) * 4, 256);
+        L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
+        L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
+        L.hb_cnt = o;   o += align_up((size_t)(H / 128) * 4, 256);
+        L.flags_end = o;
+        L.logits = o;   o += align_up((size_t)Tc * E * 4, 256);
+        L.ids = o;      o += align_up((size_t)Tc * K * 4, 256);
+        L.wts = o;      o += align_up((size_t)Tc * K * 4, 256);
+        L.xs = o;       o += align_up((size_t)Tc * (H / 128) * 4, 256);
+        L.xq = o;       o += align_up((size_t)moe::kMaxTokens * H, 1024);
+        L.hq = o;       o += align_up((size_t)E * N * I, 1024);
+        L.hs = o;       o += align_up((size_t)E * N * (I / 128) * 4, 256);
+        L.part_up = o;  o += align_up((size_t)G * 2 * N * 128 * 4, 256);
+        L.part_dn = o;  o += align_up((size_t)G * N * 128 * 4, 256);
+        L.y = o;        o += align_up((size_t)Tc * K * H * 4, 256);
+        L.total = o;
+        return L;
+    }
+
+    int stages_for(int N, int T) const {
+        for (int s = moe::kMaxStages; s >= 2; --s) {
+            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, s);
+            if (L.total + 1024 <= smem_optin) return s;
+        }
+        return 0;
+    }
+
+    bool get_map(CUtensorMap* out, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+        MapKey k{ptr, rows, cols, box_rows};
+        std::lock_guard<std::mutex> lock(mu);
+        for (auto& kv : maps)
+            if (kv.first == k) { *out = kv.second; return true; }
+        CUtensorMap m;
+        if (!encode_2d(&m, ptr, rows, cols, box_rows)) return false;
+        if (maps.size() >= 256) maps.erase(maps.begin());
+        maps.emplace_back(k, m);
+        *out = m;
+        return true;
+    }
+};
+
+using Plan = struct moe_plan;
+
+namespace {
+
+template <int N>
+int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx, const CUtensorMap& mh,
+           const moe::Params& P, int smem_bytes, cudaStream_t stream) {
+    static int configured_device = -1;
+    if (configured_device != p->device) {
+        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
+            return fail(MOE_ERR_CUDA, "cudaFuncSetAttribute(max dynamic smem) failed: %s", cudaGetErrorString(cudaGetLastError()));
+        configured_device = p->device;
+    }
+    moe::moe_decode_kernel<N><<<p->sms, moe::kThreads, smem_bytes, stream>>>(m13, m2, mx, mh, P);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
+    return MOE_OK;
+}
+
+template <int N>
+int occupancy(int smem_bytes, int* blocks) {
+    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return -1;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, moe::moe_decode_kernel<N>, moe::kThreads, smem_bytes) == cudaSuccess ? 0 : -1;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
+                  const float* W13s, const void* W2, const float* W2s, void* out, void* ws, size_t ws_bytes,
+                  cudaStream_t stream) {
+    const int N = p->n_hw(T);
+    const WsLayout L = p->layout(T);
+    if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
+    const int stages = p->stages_for(N, T);
+    if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
+    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, stages);
+    uint8_t* w = static_cast<uint8_t*>(ws);
+
+    CUtensorMap m13, m2, mx, mh;
+    if (!p->get_map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) ||
+        !p->get_map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
+        !p->get_map(&mx, w + L.xq, moe::kMaxTokens, p->H, N) ||
+        !p->get_map(&mh, w + L.hq, (uint64_t)p->E * N, p->I, N))
+        return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+
+    moe::Params P;
+    P.T = T; P.H = p->H; P.E = p->E; P.I = p->I; P.K = p->K; P.scoring = p->scoring; P.renorm = p->renorm;
+    P.routed_scale = p->routed_scale;
+    P.stages = stages;
+    P.timeout_ns = p->timeout_ns;
+    P.hidden = static_cast<const __nv_bfloat16*>(hidden);
+    P.Wr = static_cast<const __nv_bfloat16*>(Wr);
+    P.bias = (p->scoring == MOE_SCORE_SIGMOID_BIAS) ? bias : nullptr;
+    P.W13s = W13s; P.W2s = W2s;
+    P.out = static_cast<__nv_bfloat16*>(out);
+    P.ctrl = reinterpret_cast<unsigned*>(w + L.ctrl);
+    P.logits = reinterpret_cast<float*>(w + L.logits);
+    P.ids = reinterpret_cast<int*>(w + L.ids);
+    P.wts = reinterpret_cast<float*>(w + L.wts);
+    P.xq = w + L.xq;
+    P.xs = reinterpret_cast<float*>(w + L.xs);
+    P.hq = w + L.hq;
+    P.hs = reinterpret_cast<float*>(w + L.hs);
+    P.hq_flag = reinterpret_cast<unsigned*>(w + L.hq_flag);
+    P.part_up = reinterpret_cast<float*>(w + L.part_up);
+    P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
+    P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
+    P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
+    P.y = reinterpret_cast<float*>(w + L.y);
+    P.hb_cnt = reinterpret_cast<unsigned*>(w + L.hb_cnt);
+
+    const int smem_bytes = SL.total + 1024;
+    switch (N) {
+        case 16: return launch<16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        case 32: return launch<32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        default: return launch<64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    }
+}
+
+int check_forward_args(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
+                       const float* W13s, const void* W2, const float* W2s, void* out, void* ws) {
+    if (!p) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (T < 1) return fail(MOE_ERR_ARG, "T must be >= 1 (got %d)", T);
+    if (!hidden || !Wr || !W13 || !W13s || !W2 || !W2s || !out) return fail(MOE_ERR_ARG, "a tensor pointer is NULL");
+    if (!ws) return fail(MOE_ERR_WORKSPACE, "workspace is NULL");
+    if (p->scoring == MOE_SCORE_SIGMOID_BIAS && bias && !aligned16(bias)) return fail(MOE_ERR_ALIGN, "sel_bias not 16-byte aligned");
+    if (!aligned16(hidden) || !aligned16(Wr) || !aligned16(W13) || !aligned16(W13s) || !aligned16(W2) || !aligned16(W2s) ||
+        !aligned16(out))
+        return fail(MOE_ERR_ALIGN, "tensor pointers must be 16-byte aligned");
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(MOE_ERR_ALIGN, "workspace must be 256-byte aligned");
+    return MOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_last_error(void) { return g_err; }
+
+int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float routed_scale, moe_plan_t* out) {
+    if (!out) return fail(MOE_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    if (H <= 0 || I <= 0 || H % 128 || I % 128) return fail(MOE_ERR_SHAPE, "H and I must be positive multiples of 128");
+    if (E < 1 || E > moe::kMaxExperts) return fail(MOE_ERR_SHAPE, "E must be in [1,%d]", moe::kMaxExperts);
+    if (top_k < 1 || top_k > E || top_k > moe::kMaxTopK) return fail(MOE_ERR_SHAPE, "top_k must be in [1,min(E,%d)]", moe::kMaxTopK);
+    if (scoring != MOE_SCORE_SOFTMAX && scoring != MOE_SCORE_SIGMOID_BIAS) return fail(MOE_ERR_ARG, "unknown scoring %d", scoring);
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+        cudaGetLastError();
+        return fail(MOE_ERR_UNSUPPORTED_ARCH, "no CUDA device: this library has no CPU fallback");
+    }
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
+        return fail(MOE_ERR_CUDA, "cannot query the current device");
+    if (prop.major != 10) return fail(MOE_ERR_UNSUPPORTED_ARCH, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+    Plan* p = new Plan();
+    p->H = H; p->E = E; p->I = I; p->K = top_k; p->scoring = scoring; p->renorm = renorm ? 1 : 0;
+    p->routed_scale = routed_scale;
+    p->device = dev;
+    p->sms = prop.multiProcessorCount;
+    p->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    p->timeout_ns = 1000ull * 1000ull * 1000ull;
+    // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
+    int blocks = 0;
+    const int st = p->stages_for(64, moe::kMaxTokens);
+    if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
+    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, st).total + 1024;
+    if (occupancy<64>(smem, &blocks) != 0 || blocks < 1 || occupancy<16>(smem, &blocks) != 0 || blocks < 1 ||
+        occupancy<32>(smem, &blocks) != 0 || blocks < 1) {
+        delete p;
+        return fail(MOE_ERR_OCCUPANCY, "persistent kernel is not resident with %d bytes of shared memory", smem);
+    }
+    if (!get_encode_fn()) { delete p; return fail(MOE_ERR_CUDA, "driver does not export cuTensorMapEncodeTiled"); }
+    *out = p;
+    return MOE_OK;
+}
+
+int moe_plan(int H, int E, int I, int top_k, int scoring, int renorm, moe_plan_t* out) {
+    return moe_plan_ex(H, E, I, top_k, scoring, renorm, 1.0f, out);
+}
+
+void moe_plan_destroy(moe_plan_t plan) { delete plan; }
+
+size_t moe_workspace_bytes(moe_plan_t plan, int T_max) {
+    if (!plan || T_max < 1) return 0;
+    return plan->layout(T_max).total;
+}
+
+int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes, moe_stream_t stream) {
+    if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (!workspace) return fail(MOE_ERR_WORKSPACE, "workspace is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return fail(MOE_ERR_ALIGN, "workspace must be 256-byte aligned");
+    const WsLayout L = plan->layout(1);
+    if (workspace_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace too small");
+    if (cudaMemsetAsync(workspace, 0, L.flags_end, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
+    return MOE_OK;
+}
+
+int moe_forward(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
+                void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream) {
+    int rc = check_forward_args(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, workspace);
+    if (rc != MOE_OK) return rc;
+    for (int t0 = 0; t0 < T; t0 += moe::kMaxTokens) {
+        const int tc = (T - t0 < moe::kMaxTokens) ? T - t0 : moe::kMaxTokens;
+        rc = forward_chunk(plan, tc, static_cast<const uint16_t*>(hidden_bf16) + (size_t)t0 * plan->H, Wr_bf16, sel_bias,
+                           W13_fp8, W13_scale, W2_fp8, W2_scale, static_cast<uint16_t*>(out_bf16) + (size_t)t0 * plan->H,
+                           workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+        if (rc != MOE_OK) return rc;
+    }
+    return MOE_OK;
+}
+
+int moe_forward_debug(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                      const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
+                      void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream,
+                      int32_t* topk_ids, float* topk_w, uint8_t* xq, float* xs, float* logits) {
+    if (plan && T > moe::kMaxTokens) return fail(MOE_ERR_ARG, "moe_forward_debug needs T <= %d", moe::kMaxTokens);
+    int rc = moe_forward(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, workspace,
+                         workspace_bytes, stream);
+    if (rc != MOE_OK) return rc;
+    const WsLayout L = plan->layout(T);
+    const uint8_t* w = static_cast<const uint8_t*>(workspace);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    if (topk_ids && e == cudaSuccess) e = cudaMemcpyAsync(topk_ids, w + L.ids, (size_t)T * plan->K * 4, cudaMemcpyDeviceToDevice, s);
+    if (topk_w && e == cudaSuccess) e = cudaMemcpyAsync(topk_w, w + L.wts, (size_t)T * plan->K * 4, cudaMemcpyDeviceToDevice, s);
+    if (xq && e == cudaSuccess) e = cudaMemcpyAsync(xq, w + L.xq, (size_t)T * plan->H, cudaMemcpyDeviceToDevice, s);
+    if (xs && e == cudaSuccess) e = cudaMemcpyAsync(xs, w + L.xs, (size_t)T * (plan->H / 128) * 4, cudaMemcpyDeviceToDevice, s);
+    if (logits && e == cudaSuccess) e = cudaMemcpyAsync(logits, w + L.logits, (size_t)T * plan->E * 4, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return fail(MOE_ERR_CUDA, "debug copy failed: %s", cudaGetErrorString(e));
+    return MOE_OK;
+}
+
+int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream) {
+    if (!plan || !workspace) return fail(MOE_ERR_ARG, "plan or workspace is NULL");
+    unsigned ctrl[8] = {0};
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaMemcpy(ctrl, workspace, sizeof(ctrl), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(MOE_ERR_CUDA, "CUDA error while reading status: %s", cudaGetErrorString(e));
+    if (ctrl[moe::kStatus] != 0 || ctrl[moe::kAbort] != 0) {
+        const unsigned st = ctrl[moe::kStatus];
+        return fail(MOE_ERR_TIMEOUT, "device wait ran out (site %u, CTA %u); re-initialise the workspace", (st >> 8) & 0xFF, st >> 16);
+    }
+    return MOE_OK;
+}
+
+int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes) {
+    if (!plan || T < 1) return fail(MOE_ERR_ARG, "bad arguments");
+    const int Tc = plan->cap(T), N = plan->n_hw(Tc), st = plan->stages_for(N, Tc);
+    if (grid) *grid = plan->sms;
+    if (stages) *stages = st;
+    if (n_hw) *n_hw = N;
+    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, st).total + 1024;
+    return MOE_OK;
+}
+
+int moe_plan_set_timeout_ms(moe_plan_t plan, int ms) {
+    if (!plan || ms < 1) return fail(MOE_ERR_ARG, "bad arguments");
+    plan->timeout_ns = (unsigned long long)ms * 1000000ull;
+    return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,97 @@
+"""Shared helper of the GPU parity tests: run the CUDA library and the CPU oracle on the same seeded inputs.
+
+Acceptance (written out here, used by every parity test):
+  * top-k ids bit-exact (slot order included) for every token whose selection margin exceeds
+    tau = 1e-4*max(1,|key_K|); a token inside that band may differ only by candidates inside the band and
+    is then compared against the oracle evaluated with the GPU's routing;
+  * input-quantisation bytes and scales bit-exact;
+  * output: relative L2 error <= 5e-3 and |diff| <= 2e-2*rms(oracle) + 1e-3 per element.
+"""
+import numpy as np
+import torch
+
+import oracle
+from paper_2609_04244_b200 import MoEPlan
+from paper_2609_04244_b200 import workloads as wl
+
+REL_L2_TOL = 5e-3
+
+
+def _u16(t):
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def check_against_oracle(shape, T, d, dbg, routed_scale=1.0, max_oracle_tokens=None):
+    """d: inputs (device tensors) from workloads.make_layer; dbg: dict from MoEPlan.forward_debug."""
+    hid, Wr = _u16(d["hidden"]), _u16(d["Wr"])
+    bias = None if d["bias"] is None else d["bias"].cpu().numpy()
+    K = shape.top_k
+    rt = oracle.route_and_quantize(hid, Wr, bias, K, shape.scoring, shape.renorm, routed_scale)
+    g_ids = dbg["ids"].cpu().numpy()
+    g_w = dbg["w"].cpu().numpy()
+    # --- input quantisation: bit exact
+    assert np.array_equal(dbg["xq"].cpu().numpy(), rt["xq"]), "input FP8 bytes differ"
+    assert np.array_equal(dbg["xs"].cpu().numpy(), rt["xs"]), "input scales differ"
+    np.testing.assert_allclose(dbg["logits"].cpu().numpy(), rt["logits"], rtol=0, atol=2e-5 * max(1.0, np.abs(rt["logits"]).max()))
+    # --- routing
+    ambiguous = []
+    for t in range(T):
+        if np.array_equal(g_ids[t], rt["ids"][t]):
+            continue
+        lo = rt["logits"][t].astype(np.float64)
+        key = lo if shape.scoring == 0 else 1 / (1 + np.exp(-lo)) + (0 if bias is None else bias)
+        kK = key[rt["ids"][t][-1]]
+        tau = 1e-4 * max(1.0, abs(kK))
+        assert rt["margin"][t] <= tau or _only_order_within_band(g_ids[t], rt["ids"][t], key, tau), \
+            f"token {t}: ids {g_ids[t]} != oracle {rt['ids'][t]} with margin {rt['margin'][t]}"
+        diff = set(g_ids[t]) ^ set(rt["ids"][t])
+        assert all(abs(key[e] - kK) <= 2 * tau for e in diff), f"token {t}: swapped experts outside the near-tie band"
+        assert len(set(g_ids[t])) == K
+        ambiguous.append(t)
+    exact = [t for t in range(T) if t not in ambiguous]
+    np.testing.assert_allclose(g_w[exact], rt["w"][exact], rtol=2e-5, atol=1e-7)
+    # --- expert path: oracle needs only the experts actually used
+    tok = list(range(T)) if max_oracle_tokens is None else list(range(min(T, max_oracle_tokens)))
+    ids_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_ids, rt["ids"])[tok]
+    w_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_w, rt["w"])[tok]
+    used = np.unique(ids_use)
+    emap = np.full(shape.E, -1, np.int32)
+    emap[used] = np.arange(len(used))
+    sel = torch.as_tensor(used, device=d["W13q"].device, dtype=torch.long)
+    r = oracle.moe_forward(hid[tok], Wr, bias, d["W13q"][sel].cpu().numpy(), d["W13s"][sel].cpu().numpy(),
+                           d["W2q"][sel].cpu().numpy(), d["W2s"][sel].cpu().numpy(), top_k=K, scoring=shape.scoring,
+                           renorm=shape.renorm, routed_scale=routed_scale, expert_map=emap,
+                           ids_in=ids_use, w_in=w_use)
+    ref = r["out_f64"]
+    got = dbg["out"].float().cpu().numpy().astype(np.float64)[tok]
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    rms = np.sqrt(np.mean(ref ** 2))
+    worst = np.abs(got - ref).max()
+    assert rel <= REL_L2_TOL, f"rel L2 {rel:.3e}"
+    assert worst <= 2e-2 * rms + 1e-3, f"max |diff| {worst:.3e} vs rms {rms:.3e}"
+    return {"rel_l2": float(rel), "max_abs": float(worst), "rms": float(rms), "ambiguous": len(ambiguous),
+            "unique_experts": int(len(np.unique(g_ids)))}
+
+
+def _only_order_within_band(a, b, key, tau):
+    """Same set, and every position where the order differs involves keys closer than tau."""
+    if set(a) != set(b):
+        return False
+    return all(x == y or abs(key[x] - key[y]) <= tau for x, y in zip(a, b))
+
+
+def run_case(shape, T, regime="natural", layer=0, dist="gauss", routed_scale=1.0, max_oracle_tokens=None, repeat=1):
+    d = wl.make_layer(shape, T, regime=regime, layer=layer, device="cuda", dist=dist)
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, routed_scale, T_max=T)
+    try:
+        dbg = plan.forward_debug(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
+        plan.sync_status()
+        res = check_against_oracle(shape, T, d, dbg, routed_scale, max_oracle_tokens)
+        for _ in range(repeat - 1):   # run-to-run bit-identical (deterministic reduction)
+            out2 = plan.forward(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
+            plan.sync_status()
+            assert torch.equal(out2, dbg["out"]), "output not bit-identical between runs"
+        res["info"] = plan.info(T)
+        return res
+    finally:
+        plan.close()

@@ -1,0 +1,51 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_04244_b200 import workloads as wl
+from tests.parity import run_case
+
+pytestmark = pytest.mark.gpu
+
+TINY = wl.MoEShape("tiny", 1, H=256, E=8, I=128, top_k=2, scoring=wl.SCORE_SOFTMAX)
+SMALL_SIG = wl.MoEShape("small_sig", 5, H=512, E=32, I=256, top_k=4, scoring=wl.SCORE_SIGMOID_BIAS)
+RAGGED = wl.MoEShape("ragged", 2, H=384, E=20, I=640, top_k=3, scoring=wl.SCORE_SOFTMAX)
+
+
+@pytest.mark.parametrize("T", [1, 2, 5, 16, 17, 33, 64])
+def test_tiny_all_token_tiles(T):
+    r = run_case(TINY, T, repeat=2)
+    assert r["rel_l2"] < 2e-3, r
+
+
+@pytest.mark.parametrize("shape,T", [(SMALL_SIG, 1), (SMALL_SIG, 8), (SMALL_SIG, 40), (RAGGED, 3), (RAGGED, 24)])
+def test_small_shapes_sigmoid_and_ragged(shape, T):
+    r = run_case(shape, T, repeat=2)
+    assert r["rel_l2"] < 2e-3, r
+
+
+def test_config1_tiny_moe():
+    r = run_case(wl.SHAPES["c1_tiny"], 1, repeat=3)
+    assert r["rel_l2"] < 2e-3 and r["unique_experts"] == 2, r
+
+
+@pytest.mark.parametrize("T", [1, 8])
+def test_config2_qwen3_like(T):
+    r = run_case(wl.SHAPES["c2_qwen3_30b_a3b"], T, repeat=2)
+    assert r["rel_l2"] < 2e-3, r
+
+
+@pytest.mark.parametrize("regime,T", [("same", 4), ("disjoint", 4), ("disjoint", 32), ("natural", 64)])
+def test_config3_routing_regimes(regime, T):
+    r = run_case(wl.SHAPES["c2_qwen3_30b_a3b"], T, regime=regime, max_oracle_tokens=8)
+    if regime == "same":
+        assert r["unique_experts"] == 8
+    if regime == "disjoint":
+        assert r["unique_experts"] == min(128, 8 * T)
+    assert r["rel_l2"] < 2e-3, r
+
+
+def test_more_than_64_tokens_is_chunked():
+    r = run_case(SMALL_SIG, 100, max_oracle_tokens=None)
+    assert r["rel_l2"] < 2e-3, r
