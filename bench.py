@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the fused routed-MoE decode step on B200.
+
+One "step" = one layer-step of the whole operator (router, top-k, input quantisation, gate/up projection,
+SwiGLU + requantisation, down projection, weighted reduction) = one launch of the persistent kernel.
+Default workload: the Qwen3-30B-A3B-like layer (H=2048, E=128, top-8, I=768) at T=1.  Consecutive steps rotate
+over L distinct layer copies (different weights and routers) so that every step streams its experts from HBM,
+not from L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--tokens T] [--regime R] [--impl reference]
+
+Prints ONE JSON line.  `value` is microseconds per layer-step with all inputs resident in HBM; `e2e` is the same
+through the public API with the step's input copied from pinned host memory and the result copied back.
+`--impl reference` times the CPU oracle (the reference arm) on the same workload.
+With N > 1 (torchrun) every rank runs an independent replica: the operator does not shard (no collectives).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "us_per_moe_layer_step"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the fused kernel from the ncu
+# captures summarised under profiles/; keyed by (config, tokens).  None where no capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--config", default="c2_qwen3_30b_a3b")
+    ap.add_argument("--tokens", type=int, default=1)
+    ap.add_argument("--regime", default="natural", choices=["natural", "same", "disjoint"])
+    ap.add_argument("--layers", type=int, default=0, help="distinct layer copies to rotate over (0 = auto)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.stop = threading.Event()
+        self.thread = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def start(self):
+        if self.ok:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+
+    def finish(self, t0=None, t1=None):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        self.stop.set()
+        self.thread.join(timeout=1.0)
+        nv = self.nv
+        inside = [s for s in self.samples if t0 is None or (t0 <= s[0] <= t1)]
+        use = inside if inside else self.samples[-5:]
+        mhz = sorted(s[1] for s in use)
+        bits = 0
+        for s in use:
+            bits |= s[2]
+        names = []
+        table = [("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap")]
+        for name, attr in table:
+            if bits & getattr(nv, attr, 0):
+                names.append(name)
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": self.max_mhz, "reasons": names,
+                "samples": len(use), "window": "timed region" if inside else "around timed region"}
+
+
+def oracle_inputs(d, ids):
+    """Host copies of exactly what the oracle needs: hidden, router, bias and the selected experts' weights."""
+    import numpy as np
+    import torch
+    used = np.unique(ids)
+    emap = np.full(d["Wr"].shape[0], -1, np.int32)
+    emap[used] = np.arange(len(used))
+    sel = torch.as_tensor(used, device=d["W13q"].device, dtype=torch.long)
+    u16 = lambda t: t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+    return dict(hidden=u16(d["hidden"]), Wr=u16(d["Wr"]), bias=None if d["bias"] is None else d["bias"].cpu().numpy(),
+                W13q=d["W13q"][sel].cpu().numpy(), W13s=d["W13s"][sel].cpu().numpy(), W2q=d["W2q"][sel].cpu().numpy(),
+                W2s=d["W2s"][sel].cpu().numpy(), emap=emap)
+
+
+def time_oracle(shape, host, reps_budget_s=12.0, max_reps=50):
+    """Wall-clock of the CPU oracle, as it stands, on one layer-step; returns (us per step, reps, threads)."""
+    import oracle
+    reps, total = 0, 0.0
+    while reps < max_reps and (reps < 2 or total < reps_budget_s):
+        t0 = time.perf_counter()
+        oracle.moe_forward(host["hidden"], host["Wr"], host["bias"], host["W13q"], host["W13s"], host["W2q"],
+                           host["W2s"], top_k=shape.top_k, scoring=shape.scoring, renorm=shape.renorm,
+                           expert_map=host["emap"])
+        total += time.perf_counter() - t0
+        reps += 1
+    return total / reps * 1e6, reps, oracle.threads()
+
+
+def run_reference(args, shape):
+    """The reference arm: the CPU oracle on the bench workload (host cores), same metric and config keys."""
+    import numpy as np
+    import torch
+    from paper_2609_04244_b200 import workloads as wl
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    T = args.tokens
+    # inputs generated on the host: route first, then generate only the experts the oracle will touch
+    seed = wl.workload_seed(shape, T, args.regime, 0)
+    hidden = wl.make_hidden(shape, T, seed, "cpu")
+    Wr, bias = wl.make_router(shape, seed, "cpu")
+    Wr = wl.force_routing(Wr, hidden, shape.top_k, args.regime)
+    u16 = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    rt = oracle.route_and_quantize(u16(hidden), u16(Wr), None if bias is None else bias.numpy(), shape.top_k,
+                                   shape.scoring, shape.renorm)
+    used = np.unique(rt["ids"])
+    w = wl.make_expert_weights(shape, seed, "cpu", experts=[int(e) for e in used])
+    d = {"hidden": hidden, "Wr": Wr, "bias": bias, **w}
+    host = oracle_inputs(d, rt["ids"])
+    steps, warm = max(1, min(args.steps, 20)), max(0, min(args.warmup, 2))
+    for _ in range(warm):
+        time_oracle(shape, host, reps_budget_s=0.0, max_reps=2)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.moe_forward(host["hidden"], host["Wr"], host["bias"], host["W13q"], host["W13s"], host["W2q"],
+                           host["W2s"], top_k=shape.top_k, scoring=shape.scoring, renorm=shape.renorm,
+                           expert_map=host["emap"])
+    us = (time.perf_counter() - t0) / steps * 1e6
+    sample = f"{steps} full layer-steps at T={T} (steps capped at 20 for the CPU arm)"
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{shape.name} T={T} regime={args.regime}", "H": shape.H, "E": shape.E, "I": shape.I,
+                       "top_k": shape.top_k, "tokens": T},
+            "cpu_baseline": {"value": us, "unit": "us", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    from paper_2609_04244_b200 import workloads as wl
+    shape = wl.SHAPES[args.config]
+    if args.impl == "reference":
+        run_reference(args, shape)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2609_04244_b200 import MoEPlan
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fused kernel has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    T, K, W = args.tokens, args.steps, max(args.warmup, 3)
+    # enough distinct layer copies that the bytes streamed between two uses of a copy exceed 2x L2 (126 MB)
+    per_step = wl.algorithmic_bytes(shape, T, min(shape.E, int(round(wl.expected_unique_experts(shape.E, shape.top_k, T)))))
+    free_b, _ = torch.cuda.mem_get_info()
+    layer_bytes = shape.E * shape.bytes_per_expert
+    L = args.layers or max(2, min(16, -(-2 * 126 * 2**20 // per_step) + 1))
+    L = max(1, min(L, int(0.6 * free_b // layer_bytes)))
+    layers = [wl.make_layer(shape, T, regime=args.regime, layer=rank * 64 + l, device=dev) for l in range(L)]
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T)
+    info = plan.info(T)
+    outs = [torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+
+    def step(i):
+        d = layers[i % L]
+        plan.forward(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], out=outs[i % L])
+
+    # unique experts per layer copy (from the kernel's own routing) -> algorithmic bytes per step
+    uniq = []
+    for l in range(L):
+        d = layers[l]
+        dbg = plan.forward_debug(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
+        plan.sync_status()
+        uniq.append(int(torch.unique(dbg["ids"]).numel()))
+    ids0 = dbg["ids"].cpu().numpy() if L == 1 else None
+    bytes_per_step = float(np.mean([wl.algorithmic_bytes(shape, T, u) for u in uniq]))
+    launches_per_step = -(-T // 64)
+
+    # The timed steps are replayed from CUDA graphs (Section 4.1 of the paper times graph replays): a graph holds
+    # up to 1000 consecutive steps, so the host's per-call cost (Python, ctypes, launch) is not what is measured.
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+
+    def capture(first, n):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(n):
+                step(first + i)
+        return g
+
+    CH = 1000
+    graphs, done = [], 0
+    full = capture(W, CH) if K >= CH else None          # replayed K // CH times; the layer rotation inside it is
+    while done + CH <= K:                               # what keeps L2 cold, not the seam between two replays
+        graphs.append(full)
+        done += CH
+    if K - done:
+        graphs.append(capture(W + done, K - done))
+    for g in {id(g): g for g in graphs}.values():       # one untimed replay of each graph (first-launch upload)
+        g.replay()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_wall0 = time.perf_counter()
+    ev0.record(stream)
+    for g in graphs:
+        g.replay()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    if t_wall1 - t_wall0 < 0.25:        # timed region too short for a clock sample: keep the same load running briefly
+        t_end = time.perf_counter() + 0.3
+        while time.perf_counter() < t_end:
+            graphs[0].replay()
+            torch.cuda.synchronize()
+        clocks = sampler.finish()
+        clocks["window"] = "timed region + 0.3 s of the same load"
+    else:
+        clocks = sampler.finish(t_wall0, t_wall1)
+    plan.sync_status()
+
+    # end to end: the step's input comes from pinned host memory, the result goes back to the host
+    e2e = None
+    if not args.no_e2e:
+        h_in = [layers[l]["hidden"].cpu().pin_memory() for l in range(L)]
+        h_out = torch.empty((T, shape.H), dtype=torch.bfloat16).pin_memory()
+        d_in = torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev)
+
+        def e2e_step(i):
+            d = layers[i % L]
+            d_in.copy_(h_in[i % L], non_blocking=True)
+            plan.forward(d_in, d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], out=outs[i % L])
+            h_out.copy_(outs[i % L], non_blocking=True)
+            stream.synchronize()          # the caller consumes the result before the next step
+
+        Ke = min(K, 2000)
+        for i in range(W):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(Ke):
+            e2e_step(W + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e = {"ms": e2e_ms, "steps": Ke}
+        plan.sync_status()
+
+    if world > 1:
+        t = torch.tensor([ms, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t[0])
+        if e2e:
+            e2e["ms"] = float(t[1])
+
+    if rank == 0:
+        us_step = ms * 1e3 / K                     # per rank; replicas run side by side
+        value = us_step / world                    # whole-job: microseconds per layer-step over all replicas
+        kernel_us = us_step / launches_per_step
+        peak, peak_kind = peak_hbm()
+        achieved = bytes_per_step / launches_per_step / (kernel_us * 1e-6) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp8_e4m3 x fp8_e4m3 -> f32", "data": "synthetic",
+            "config": {"workload": f"{shape.name} T={T} regime={args.regime}", "H": shape.H, "E": shape.E, "I": shape.I,
+                       "top_k": shape.top_k, "tokens": T, "unique_experts_mean": float(np.mean(uniq)),
+                       "layer_copies": L, "l2": f"rotates over {L} distinct layer copies "
+                       f"({L * bytes_per_step / 2**20:.0f} MiB streamed between reuses, L2 is 126 MiB)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "grid": info["grid"], "stages": info["stages"], "n_hw": info["n_hw"],
+                       "launch": "CUDA graph replay, one kernel node per step"},
+            "achieved_gbs": achieved, "algorithmic_bytes_per_step": bytes_per_step,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}", "kernel": "moe_decode_kernel", "kernel_us": kernel_us,
+                         "traffic": NCU_TRAFFIC_BYTES.get((shape.name, T))},
+            "gpu_launches": K * launches_per_step,
+            "clocks": clocks,
+        }
+        if e2e:
+            eus = e2e["ms"] * 1e3 / e2e["steps"] / world
+            line["e2e"] = {"value": eus, "unit": "us", "h2d_bytes_per_step": 2 * T * shape.H,
+                           "d2h_bytes_per_step": 2 * T * shape.H, "steps": e2e["steps"]}
+        if world == 1 and not args.no_cpu_baseline:
+            d = layers[L - 1]
+            ids = dbg["ids"].cpu().numpy()
+            host = oracle_inputs(d, ids)
+            us_cpu, reps, thr = time_oracle(shape, host)
+            line["cpu_baseline"] = {"value": us_cpu, "unit": "us", "cores": thr, "kind": "oracle",
+                                    "sample": f"{reps} full layer-steps of the same workload (T={T}), mean"}
+        print(json.dumps(line), flush=True)
+    plan.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

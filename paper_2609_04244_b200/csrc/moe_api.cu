@@ -144,8 +144,8 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
 }
 
 template <int N>
-int occupancy(int smem_bytes, int* blocks) {
-    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return -1;
+int occupancy(int smem_optin, int smem_bytes, int* blocks) {
+    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return -1;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, moe::moe_decode_kernel<N>, moe::kThreads, smem_bytes) == cudaSuccess ? 0 : -1;
 }
 
@@ -252,8 +252,9 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
     const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, st).total + 1024;
-    if (occupancy<64>(smem, &blocks) != 0 || blocks < 1 || occupancy<16>(smem, &blocks) != 0 || blocks < 1 ||
-        occupancy<32>(smem, &blocks) != 0 || blocks < 1) {
+    const int optin = p->smem_optin;
+    if (occupancy<64>(optin, smem, &blocks) != 0 || blocks < 1 || occupancy<16>(optin, smem, &blocks) != 0 || blocks < 1 ||
+        occupancy<32>(optin, smem, &blocks) != 0 || blocks < 1) {
         delete p;
         return fail(MOE_ERR_OCCUPANCY, "persistent kernel is not resident with %d bytes of shared memory", smem);
     }
