@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--tokens", type=int, default=1)
     ap.add_argument("--regime", default="natural", choices=["natural", "same", "disjoint"])
     ap.add_argument("--layers", type=int, default=0, help="distinct layer copies to rotate over (0 = auto)")
+    ap.add_argument("--experts", type=int, default=0,
+                    help="override the number of experts E (same per-expert shapes): a small case for profiler captures")
+    ap.add_argument("--no-graph", action="store_true", help="launch the timed steps directly instead of from CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -195,6 +198,9 @@ def main():
     args = parse_args()
     from paper_2609_04244_b200 import workloads as wl
     shape = wl.SHAPES[args.config]
+    if args.experts:
+        import dataclasses
+        shape = dataclasses.replace(shape, E=args.experts, name=f"{shape.name}[E={args.experts}]")
     if args.impl == "reference":
         run_reference(args, shape)
         return
@@ -256,6 +262,16 @@ def main():
                 step(first + i)
         return g
 
+    class _Direct:                                      # --no-graph: same interface, plain launches
+        def __init__(self, first, n):
+            self.first, self.n = first, n
+
+        def replay(self):
+            for i in range(self.n):
+                step(self.first + i)
+
+    if args.no_graph:
+        capture = _Direct
     CH = 1000
     graphs, done = [], 0
     full = capture(W, CH) if K >= CH else None          # replayed K // CH times; the layer rotation inside it is
@@ -347,7 +363,7 @@ def main():
                        f"({L * bytes_per_step / 2**20:.0f} MiB streamed between reuses, L2 is 126 MiB)",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "grid": info["grid"], "stages": info["stages"], "n_hw": info["n_hw"],
-                       "launch": "CUDA graph replay, one kernel node per step"},
+                       "launch": "direct launches" if args.no_graph else "CUDA graph replay, one kernel node per step"},
             "achieved_gbs": achieved, "algorithmic_bytes_per_step": bytes_per_step,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "kernel": "moe_decode_kernel", "kernel_us": kernel_us,

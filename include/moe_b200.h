@@ -119,6 +119,14 @@ int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream);
 /* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);
 
+/* Diagnostics: synchronise `stream` and copy the phase time stamps of the last launch on this workspace to
+ * HOST memory host_out[grid*16] (nanoseconds of the GPU's global timer).  Per CTA: 0 start, 1 input quantised,
+ * 2 router logits done, 3 arrived at the routing flag, 4 routing published grid-wide, 5 scales cached,
+ * 6 top-k done, 7 routing metadata done, 8 first weight tile requested, 9 first ring of requests issued,
+ * 10 first weight tile landed, 11 first accumulator read, 12 up phase done, 13 down phase done, 14 reduction
+ * done, 15 exit.  Section 3.3 of the paper argues which of these gaps must hide under the weight stream. */
+int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint64_t* host_out);
+
 /* Set the device-side wait limit in milliseconds (default 1000).  A wait that runs out makes the kernel
  * record MOE_ERR_TIMEOUT and return; it never traps. */
 int moe_plan_set_timeout_ms(moe_plan_t plan, int ms);

@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_debug", "moe_sync_status", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -58,6 +58,8 @@ def load_library():
     lib.moe_forward_debug.argtypes = [vp, i] + [vp] * 9 + [sz, vp] + [vp] * 5
     lib.moe_sync_status.restype = i
     lib.moe_sync_status.argtypes = [vp, vp, vp]
+    lib.moe_debug_stamps.restype = i
+    lib.moe_debug_stamps.argtypes = [vp, vp, vp, vp]
     lib.moe_plan_info.restype = i
     lib.moe_plan_info.argtypes = [vp, i] + [ctypes.POINTER(i)] * 4
     lib.moe_plan_set_timeout_ms.restype = i
@@ -124,6 +126,14 @@ def moe_sync_status(plan, workspace, stream=None) -> None:
     _check(load_library().moe_sync_status(plan, _p(workspace), _stream(stream)))
 
 
+def moe_debug_stamps(plan, workspace, grid: int, stream=None):
+    """Phase time stamps [grid, 16] (ns) of the last launch on this workspace; see include/moe_b200.h."""
+    import numpy as np
+    buf = np.zeros((grid, 16), dtype=np.uint64)
+    _check(load_library().moe_debug_stamps(plan, _p(workspace), _stream(stream), ctypes.c_void_p(buf.ctypes.data)))
+    return buf
+
+
 def moe_plan_info(plan, T: int) -> dict:
     g, s, n, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     _check(load_library().moe_plan_info(plan, T, ctypes.byref(g), ctypes.byref(s), ctypes.byref(n), ctypes.byref(b)))
@@ -161,6 +171,9 @@ class MoEPlan:
 
     def sync_status(self, stream=None):
         moe_sync_status(self.handle, self.workspace, stream)
+
+    def stamps(self, stream=None):
+        return moe_debug_stamps(self.handle, self.workspace, self.info(1)["grid"], stream)
 
     def info(self, T):
         return moe_plan_info(self.handle, T)

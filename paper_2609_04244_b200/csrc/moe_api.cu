@@ -54,8 +54,8 @@ bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t ctrl, hq_flag, pu_flag, pd_flag, hb_cnt, flags_end;   // zero-initialised region = [0, flags_end)
-    size_t logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, total;
+    size_t ctrl, e_cnt, e_ready, dn_done, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
+    size_t stamps, logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, total;
 };
 
 struct MapKey {
@@ -83,11 +83,13 @@ struct moe_plan {
         WsLayout L;
         size_t o = 0;
         L.ctrl = o;     o += moe::kCtrlWords * 4;
-        L.hq_flag = o;  o += align_up((size_t)E * (I / 128) * 4, 256);
+        L.e_cnt = o;    o += align_up((size_t)E * 4, 256);
+        L.e_ready = o;  o += align_up((size_t)E * 4, 256);
+        L.dn_done = o;  o += align_up((size_t)E * (H / 128) * 4, 256);
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
-        L.hb_cnt = o;   o += align_up((size_t)(H / 128) * 4, 256);
         L.flags_end = o;
+        L.stamps = o;   o += align_up((size_t)G * 16 * 8, 256);
         L.logits = o;   o += align_up((size_t)Tc * E * 4, 256);
         L.ids = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.wts = o;      o += align_up((size_t)Tc * K * 4, 256);
@@ -128,25 +130,27 @@ using Plan = struct moe_plan;
 
 namespace {
 
-template <int N>
+template <int N, int TC>
 int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx, const CUtensorMap& mh,
            const moe::Params& P, int smem_bytes, cudaStream_t stream) {
     static int configured_device = -1;
     if (configured_device != p->device) {
-        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
+        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
             return fail(MOE_ERR_CUDA, "cudaFuncSetAttribute(max dynamic smem) failed: %s", cudaGetErrorString(cudaGetLastError()));
         configured_device = p->device;
     }
-    moe::moe_decode_kernel<N><<<p->sms, moe::kThreads, smem_bytes, stream>>>(m13, m2, mx, mh, P);
+    moe::moe_decode_kernel<N, TC><<<p->sms, moe::kThreads, smem_bytes, stream>>>(m13, m2, mx, mh, P);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
     return MOE_OK;
 }
 
-template <int N>
-int occupancy(int smem_optin, int smem_bytes, int* blocks) {
-    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return -1;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, moe::moe_decode_kernel<N>, moe::kThreads, smem_bytes) == cudaSuccess ? 0 : -1;
+template <int N, int TC>
+bool resident(int smem_optin, int smem_bytes) {
+    int blocks = 0;
+    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return false;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, moe::moe_decode_kernel<N, TC>, moe::kThreads, smem_bytes) != cudaSuccess) return false;
+    return blocks >= 1;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -187,20 +191,26 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.xs = reinterpret_cast<float*>(w + L.xs);
     P.hq = w + L.hq;
     P.hs = reinterpret_cast<float*>(w + L.hs);
-    P.hq_flag = reinterpret_cast<unsigned*>(w + L.hq_flag);
+    P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
+    P.e_ready = reinterpret_cast<unsigned*>(w + L.e_ready);
+    P.dn_done = reinterpret_cast<unsigned*>(w + L.dn_done);
     P.part_up = reinterpret_cast<float*>(w + L.part_up);
     P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
     P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
     P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
     P.y = reinterpret_cast<float*>(w + L.y);
-    P.hb_cnt = reinterpret_cast<unsigned*>(w + L.hb_cnt);
+    P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
+    P.w13s_bytes = (size_t)p->E * (2 * p->I / 128) * (p->H / 128) * 4;
+    P.w2s_bytes = (size_t)p->E * (p->H / 128) * (p->I / 128) * 4;
 
     const int smem_bytes = SL.total + 1024;
-    switch (N) {
-        case 16: return launch<16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-        case 32: return launch<32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-        default: return launch<64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    }
+    if (T == 1) return launch<16, 1>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (T == 2) return launch<16, 2>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (T <= 16) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (T <= 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
 }
 
 int check_forward_args(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
@@ -230,6 +240,11 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (E < 1 || E > moe::kMaxExperts) return fail(MOE_ERR_SHAPE, "E must be in [1,%d]", moe::kMaxExperts);
     if (top_k < 1 || top_k > E || top_k > moe::kMaxTopK) return fail(MOE_ERR_SHAPE, "top_k must be in [1,min(E,%d)]", moe::kMaxTopK);
     if (scoring != MOE_SCORE_SOFTMAX && scoring != MOE_SCORE_SIGMOID_BIAS) return fail(MOE_ERR_ARG, "unknown scoring %d", scoring);
+    {   // the kernel indexes k-steps with 32-bit integers
+        const long long ks = (long long)E * (H / 128) * (I / 128);
+        if (ks * 256 >= (1ll << 31) || (long long)E * 2 * I * H / 128 >= (1ll << 31))
+            return fail(MOE_ERR_SHAPE, "layer too large for 32-bit k-step indices");
+    }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
         cudaGetLastError();
@@ -248,13 +263,13 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     p->smem_optin = (int)prop.sharedMemPerBlockOptin;
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
-    int blocks = 0;
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
     const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, st).total + 1024;
     const int optin = p->smem_optin;
-    if (occupancy<64>(optin, smem, &blocks) != 0 || blocks < 1 || occupancy<16>(optin, smem, &blocks) != 0 || blocks < 1 ||
-        occupancy<32>(optin, smem, &blocks) != 0 || blocks < 1) {
+    if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) ||
+        !resident<16, 8>(optin, smem) || !resident<16, 4>(optin, smem) || !resident<16, 2>(optin, smem) ||
+        !resident<16, 1>(optin, smem)) {
         delete p;
         return fail(MOE_ERR_OCCUPANCY, "persistent kernel is not resident with %d bytes of shared memory", smem);
     }
@@ -331,6 +346,16 @@ int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream) {
         const unsigned st = ctrl[moe::kStatus];
         return fail(MOE_ERR_TIMEOUT, "device wait ran out (site %u, CTA %u); re-initialise the workspace", (st >> 8) & 0xFF, st >> 16);
     }
+    return MOE_OK;
+}
+
+int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint64_t* host_out) {
+    if (!plan || !workspace || !host_out) return fail(MOE_ERR_ARG, "plan, workspace or host_out is NULL");
+    const WsLayout L = plan->layout(1);
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(host_out, static_cast<const uint8_t*>(workspace) + L.stamps, (size_t)plan->sms * 16 * 8, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(MOE_ERR_CUDA, "CUDA error while reading stamps: %s", cudaGetErrorString(e));
     return MOE_OK;
 }
 

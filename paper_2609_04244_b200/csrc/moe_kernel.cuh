@@ -41,6 +41,8 @@ constexpr int kATileBytes = kBlock * kBlock;  // 16 KiB of FP8
 constexpr int kMaxTopK = 32;
 constexpr int kMaxExperts = 512;
 constexpr int kMaxTokens = 64;
+constexpr int kTmemBufs = 4;                     // accumulator buffers in TMEM (one K block each)
+constexpr int kScaleSlots = kMaxStages + 8;   // ring of per-k-step scale records, deeper than any producer lead
 
 // control words at the head of the workspace
 enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kRouteReady = 4, kExitCnt = 5, kCtrlWords = 64 };
@@ -65,14 +67,17 @@ struct Params {
     uint8_t* xq;        // [64,H]
     float* xs;          // [T,H/128]
     uint8_t* hq;        // [E,N,I]
-    float* hs;          // [E,N,I/128]
-    unsigned* hq_flag;  // [E,I/128]
+    float* hs;          // [E,I/128,N]
+    unsigned* e_cnt;    // [E]   published I-blocks of an expert's intermediate tile
+    unsigned* e_ready;  // [E]   == tag once the whole intermediate tile of the expert is published
+    unsigned* dn_done;  // [E,H/128] == tag once the expert's down-projection rows of that block are stored
     float* part_up;     // [grid][2N][128]
     float* part_dn;     // [grid][N][128]
     unsigned* pu_flag;  // [grid]
     unsigned* pd_flag;  // [grid]
     float* y;           // [T,K,H]
-    unsigned* hb_cnt;   // [H/128]
+    size_t w13s_bytes, w2s_bytes;   // sizes of the block-scale arrays (bound for 16-byte scale fetches)
+    unsigned long long* stamps;     // [grid][8] globaltimer stamps of the phases of the last launch (diagnostics)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -111,6 +116,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// plain bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16), completes on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -136,16 +148,31 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// 32 lanes x 16 consecutive 32-bit columns -> 16 registers per thread
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
+// 32 TMEM lanes x C consecutive 32-bit columns -> C registers per thread (thread = lane, register = column)
+template <int C>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
+    static_assert(C == 1 || C == 2 || C == 4 || C == 8 || C == 16, "unsupported column count");
+    uint32_t r[C];
+    if constexpr (C == 1) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr));
+    } else if constexpr (C == 2) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(taddr));
+    } else if constexpr (C == 4) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr));
+    } else if constexpr (C == 8) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                     : "r"(taddr));
+    } else {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+            : "r"(taddr));
+    }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < C; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -174,6 +201,8 @@ __device__ __forceinline__ bool epi_all(bool ok) {
         : "=r"(r) : "r"((uint32_t)ok) : "memory");
     return r != 0;
 }
+
+#define MOE_STAMP(i) do { P.stamps[(size_t)blockIdx.x * 16 + (i)] = gtime(); } while (0)
 
 // K-major, 128-byte swizzled operand tile (rows of 128 bytes, 8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
@@ -219,20 +248,22 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, xs_off, red_off, misc_off, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, xs_off, red_off, misc_off, sc_off, sc_bytes, total;
 };
 __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int stages) {
     SmemLayout L;
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
     int o = stages * L.stage_bytes;
-    L.bar_off = o;  o += (2 * kMaxStages + 8) * 8;
+    L.bar_off = o;  o += (2 * kMaxStages + 16) * 8;
     L.misc_off = o; o += 64;
+    L.sc_bytes = 32 + N * 4;                   // [16 B gate/down weight-scale chunk][16 B up chunk][N activation scales]
+    L.sc_off = o;   o += kScaleSlots * L.sc_bytes;
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
-    L.act_off = o;  o += E * 4;
+    L.act_off = o;  o += (E + 1) * 4;
     L.xs_off = o;   o += T * (H / kBlock) * 4;
     L.red_off = o;  o += kWarps * 64 * 4;      // cross-warp reduction scratch (>= 4*64 floats for amax, 8*8 for logits)
     L.total = o;
@@ -240,7 +271,103 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
 }
 
 // per-phase split of a linear k-step list into contiguous per-CTA ranges
-__device__ __forceinline__ long long range_lo(long long S, int c, int G) { return (S * c) / G; }
+__device__ __forceinline__ int range_lo(int S, int c, int G) { return (int)(((long long)S * c) / G); }
+
+// position inside the linear k-step list of one projection: k-step -> (K block, row block, active expert)
+struct Walk {
+    int kb, mb, u, e, KB, MB;
+    __device__ __forceinline__ void init(int s, int KB_, int MB_, const int* act) {
+        KB = KB_; MB = MB_;
+        const int unit = s / KB;
+        kb = s - unit * KB;
+        u = unit / MB;
+        mb = unit - u * MB;
+        e = act[u];
+    }
+    __device__ __forceinline__ void next(const int* act) {
+        if (++kb == KB) {
+            kb = 0;
+            if (++mb == MB) { mb = 0; ++u; }
+            e = act[u];
+        }
+    }
+};
+
+// monotone map float -> uint32 (larger float <=> larger integer); +0 and -0 are merged first
+__device__ __forceinline__ uint32_t orderable(float f) {
+    const uint32_t u = __float_as_uint(f + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+struct Params;
+// Scores and top-k of one token by one warp (Section 4.1 routing policies): softmax over all experts or
+// sigmoid plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots are in
+// (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
+template <int EPL, class ParamsT>
+__device__ __forceinline__ void topk_token(const ParamsT& P, int t, int lane, int* s_ids, float* s_w,
+                                           unsigned long long* s_mask, bool write_global) {
+    const int E = P.E, K = P.K;
+    const float* lg = P.logits + (size_t)t * E;
+    uint32_t ok[EPL];
+    float l[EPL];
+    float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) {
+        const int e = lane + 32 * j;
+        l[j] = (e < E) ? __ldcg(lg + e) : -INFINITY;
+        mx = fmaxf(mx, l[j]);
+    }
+    if (P.scoring == 0) {
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+            const int e = lane + 32 * j;
+            ok[j] = (e < E) ? orderable(l[j]) : 0u;
+            sum += (e < E) ? expf(l[j] - mx) : 0.f;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    } else {
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+            const int e = lane + 32 * j;
+            if (e < E) {
+                const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l[j]));
+                ok[j] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
+            } else ok[j] = 0u;
+        }
+    }
+    int myid = 0;
+    for (int k = 0; k < K; ++k) {
+        uint32_t best = 0u;
+        int bj = 0;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) if (ok[j] > best) { best = ok[j]; bj = j; }   // strict '>' keeps the lowest index
+        const uint32_t wmax = __reduce_max_sync(0xffffffffu, best);
+        const uint32_t cand = (best == wmax && best != 0u) ? (uint32_t)(lane + 32 * bj) : 0xFFFFFFFFu;
+        uint32_t win = __reduce_min_sync(0xffffffffu, cand);
+        if (win == 0xFFFFFFFFu) win = (uint32_t)k;                                     // only with NaN logits
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) if ((uint32_t)(lane + 32 * j) == win) ok[j] = 0u;
+        if (lane == k) myid = (int)win;
+    }
+    float v = 0.f;
+    if (lane < K) {
+        const float lv = __ldcg(lg + myid);
+        v = (P.scoring == 0) ? __fdiv_rn(expf(lv - mx), sum) : __fdiv_rn(1.0f, 1.0f + expf(-lv));
+    }
+    float vsum = v;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) vsum += __shfl_xor_sync(0xffffffffu, vsum, o);
+    if (lane < K) {
+        const float w = (P.renorm ? __fdiv_rn(v, vsum) : v) * P.routed_scale;
+        s_ids[t * K + lane] = myid;
+        s_w[t * K + lane] = w;
+        atomicOr(&s_mask[myid], 1ull << t);
+        if (write_global) { P.ids[t * K + lane] = myid; P.wts[t * K + lane] = w; }
+    }
+}
 
 // quantise 4 floats with scale s into 4 E4M3 bytes (memory order x0..x3)
 __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x3, float s) {
@@ -254,7 +381,8 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int N>
+// N  = MMA N (token tile, 16/32/64); TC = token columns the accumulator warps actually read (power of two >= T).
+template <int N, int TC>
 __global__ void __launch_bounds__(kThreads, 1)
 moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                   const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmHq,
@@ -271,9 +399,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
-    const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + 2);
-    const uint32_t bar_drain = smem_u32(bars + 2 * kMaxStages + 4);
-    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] last-arriver flag
+    const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kTmemBufs);
+    const uint32_t bar_drain = smem_u32(bars + 2 * kMaxStages + 2 * kTmemBufs);
+    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [3] give-up flag of the accumulator warps
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
@@ -284,12 +412,14 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     Waiter wt;
     wt.init(P.ctrl, P.timeout_ns);
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
+    if (tid == 0) MOE_STAMP(0);
 
-    constexpr uint32_t kTmemCols = (4 * N < 32) ? 32 : 4 * N;   // 2 buffers x (gate N + up N)
+    constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
         for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        misc[3] = 0u;
         mbar_init(bar_drain, 1);
         fence_barrier_init();
     }
@@ -311,6 +441,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             *reinterpret_cast<uint32_t*>(P.xq + (size_t)t * H + g * kBlock + lane * 4) = quant4(x0, x1, x2, x3, s);
             if (lane == 0) P.xs[p] = s;
         }
+        if (tid == 0) MOE_STAMP(1);
         // router logits: CTA c owns experts c, c+G, ...; all 256 threads split H  (Section 3.3)
         for (int e = cta; e < E; e += G) {
             for (int t0 = 0; t0 < T; t0 += 8) {
@@ -350,6 +481,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
         }
     }
+    if (tid == 0) MOE_STAMP(2);
     // publish: generic writes of xq must be visible to the async proxy (TMA) of every CTA
     fence_proxy_async();
     __threadfence();
@@ -358,6 +490,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
     if (tid == 0) {
+        MOE_STAMP(3);
         const unsigned old = atomicAdd(P.ctrl + kRouteCnt, 1u);
         if (old == (unsigned)G - 1u) {
             P.ctrl[kRouteCnt] = 0u;
@@ -366,6 +499,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         }
         wt.flag(P.ctrl + kRouteReady, tag, 1);
         __threadfence();
+        MOE_STAMP(4);
     }
     __syncthreads();
     bool alive = (*(volatile unsigned*)(P.ctrl + kAbort) == 0);
@@ -375,74 +509,17 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
         for (int i = tid; i < T * KBu; i += kThreads) s_xs[i] = __ldcg(P.xs + i);
         __syncthreads();
-        constexpr int EPL = kMaxExperts / 32;
+        if (tid == 0) MOE_STAMP(5);
+        const bool wg = (cta == 0);
         for (int t = warp; t < T; t += kWarps) {
-            float key[EPL], val[EPL];
-            float mx = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < EPL; ++j) {
-                const int e = lane + 32 * j;
-                float l = (e < E) ? __ldcg(P.logits + (size_t)t * E + e) : -INFINITY;
-                val[j] = l;
-                mx = fmaxf(mx, l);
-            }
-            if (P.scoring == 0) {
-#pragma unroll
-                for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                float sum = 0.f;
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {
-                    const int e = lane + 32 * j;
-                    key[j] = val[j];
-                    val[j] = (e < E) ? expf(val[j] - mx) : 0.f;
-                    sum += val[j];
-                }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) val[j] = __fdiv_rn(val[j], sum);
-            } else {
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {
-                    const int e = lane + 32 * j;
-                    if (e < E) {
-                        val[j] = __fdiv_rn(1.0f, 1.0f + expf(-val[j]));
-                        key[j] = val[j] + (P.bias ? __ldg(P.bias + e) : 0.f);
-                    } else { val[j] = 0.f; key[j] = -INFINITY; }
-                }
-            }
-            float vsum = 0.f, myv = 0.f;
-            int myid = 0;
-            for (int k = 0; k < K; ++k) {
-                float bk = -INFINITY, bv = 0.f;
-                int bi = 0x7fffffff;
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {            // ascending index, strict '>' keeps the lowest index
-                    const int e = lane + 32 * j;
-                    if (e < E && key[j] > bk) { bk = key[j]; bi = e; bv = val[j]; }
-                }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) {
-                    const float ok = __shfl_xor_sync(0xffffffffu, bk, o);
-                    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                    if (ok > bk || (ok == bk && oi < bi)) { bk = ok; bi = oi; bv = ov; }
-                }
-                if (bi == 0x7fffffff) bi = 0;              // only reachable with NaN keys
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) if (lane + 32 * j == bi) key[j] = -INFINITY;
-                if (lane == k) { myid = bi; myv = bv; }
-                vsum += bv;
-            }
-            if (lane < K) {
-                const float w = (P.renorm ? __fdiv_rn(myv, vsum) : myv) * P.routed_scale;
-                s_ids[t * K + lane] = myid;
-                s_w[t * K + lane] = w;
-                atomicOr(&s_mask[myid], 1ull << t);
-                if (cta == 0) { P.ids[t * K + lane] = myid; P.wts[t * K + lane] = w; }
-            }
+            if (E <= 32) topk_token<1>(P, t, lane, s_ids, s_w, s_mask, wg);
+            else if (E <= 64) topk_token<2>(P, t, lane, s_ids, s_w, s_mask, wg);
+            else if (E <= 128) topk_token<4>(P, t, lane, s_ids, s_w, s_mask, wg);
+            else if (E <= 256) topk_token<8>(P, t, lane, s_ids, s_w, s_mask, wg);
+            else topk_token<16>(P, t, lane, s_ids, s_w, s_mask, wg);
         }
         __syncthreads();
+        if (tid == 0) MOE_STAMP(6);
         if (warp == 0) {                                   // active-expert list in ascending expert order
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
@@ -452,76 +529,110 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (on) s_act[base + __popc(b & ((1u << lane) - 1u))] = e;
                 base += __popc(b);
             }
-            if (lane == 0) misc[1] = (uint32_t)base;
+            if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
         }
-        fence_proxy_async();
         __syncthreads();
     }
     const int U = alive ? (int)misc[1] : 0;
-    const long long S_up = (long long)U * IB * KBu, S_dn = (long long)U * HB * KBd;
-    const long long up_lo = range_lo(S_up, cta, G), up_hi = range_lo(S_up, cta + 1, G);
-    const long long dn_lo = range_lo(S_dn, cta, G), dn_hi = range_lo(S_dn, cta + 1, G);
+    if (tid == 0) MOE_STAMP(7);
+    const int S_up = U * IB * KBu, S_dn = U * HB * KBd;     // k-steps of the two projections (host checks the range)
+    const int up_lo = range_lo(S_up, cta, G), up_hi = range_lo(S_up, cta + 1, G);
+    const int dn_lo = range_lo(S_dn, cta, G), dn_hi = range_lo(S_dn, cta + 1, G);
     const uint32_t stage_tx = (uint32_t)L.stage_bytes;
 
     // ------------------------------------------------------------------ role: TMA producer
     if (warp == 0) {
         if (lane == 0 && alive) {
-            // stage sequence: up k-steps contribute two stages (gate tile, up tile), down k-steps one.
-            const long long n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
-            long long a_cur = 0, b_cur = 0;      // stages whose weight tile / activation tile has been issued
+            // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.
+            // Every stage = weight tile + activation tile + the block scales its K block needs (a 16-byte chunk of
+            // the weight-scale array and, in the down phase, the N activation scales), all on one mbarrier.
+            // Weight tiles (cursor A) run ahead of activation tiles (cursor B): only the latter wait for the
+            // intermediate tile of the up projection to be published.
+            fence_proxy_async();                 // xq was written with ordinary stores by other CTAs
+            const int n_up_ks = up_hi - up_lo, n_up_st = 2 * n_up_ks, n_st = n_up_st + (dn_hi - dn_lo);
+            const uint32_t sc_base = smem_u32(smem + L.sc_off);
+            Walk aw, bw;
+            int a_cur = 0, a_st = 0, a_slot = 0, b_cur = 0, b_st = 0, b_slot = 0;
+            uint32_t a_ph = 1u;                  // parity to wait for on the empty barrier
+            if (n_up_ks > 0) { aw.init(up_lo, KBu, IB, s_act); bw = aw; }
+            else if (n_st > 0) { aw.init(dn_lo, KBd, HB, s_act); bw = aw; }
+            int ready_e = -1;                    // expert whose intermediate tile is known to be published
             uint32_t idle = 0;
+            bool stamped = false;
+            MOE_STAMP(8);
             while (b_cur < n_st && !wt.dead) {
                 bool progress = false;
-                if (a_cur < n_st && a_cur - b_cur < S) {
-                    const int st = (int)(a_cur % S);
-                    const uint32_t par = (uint32_t)((a_cur / S) & 1) ^ 1u;
-                    if (mbar_try_wait(bar_empty + 8 * st, par)) {
-                        const uint32_t dst = smem_u32(smem + (size_t)st * L.stage_bytes);
-                        mbar_expect_tx(bar_full + 8 * st, stage_tx);
-                        if (a_cur < n_up_st) {
-                            const long long s = up_lo + (a_cur >> 1);
-                            const int half = (int)(a_cur & 1), kb = (int)(s % KBu);
-                            const int unit = (int)(s / KBu), e = s_act[unit / IB], ib = unit % IB;
-                            tma_load_2d(dst, &tmW13, kb * kBlock, e * 2 * I + half * I + ib * kBlock, bar_full + 8 * st);
-                        } else {
-                            const long long s = dn_lo + (a_cur - n_up_st);
-                            const int ib = (int)(s % KBd), unit = (int)(s / KBd), e = s_act[unit / HB], hb = unit % HB;
-                            tma_load_2d(dst, &tmW2, ib * kBlock, e * H + hb * kBlock, bar_full + 8 * st);
-                        }
-                        ++a_cur;
-                        progress = true;
+                while (a_cur < n_st && a_cur - b_cur < S) {
+                    if (!mbar_try_wait(bar_empty + 8 * a_st, a_ph)) break;
+                    const uint32_t dst = smem_u32(smem + (size_t)a_st * L.stage_bytes);
+                    const uint32_t full = bar_full + 8 * a_st;
+                    const bool is_up = a_cur < n_up_st;
+                    const int half = is_up ? (a_cur & 1) : 0;
+                    const uint32_t slot = sc_base + (uint32_t)a_slot * L.sc_bytes + 16u * half;
+                    const float* sbase = is_up ? P.W13s : P.W2s;
+                    const size_t sbytes = is_up ? P.w13s_bytes : P.w2s_bytes;
+                    const int sidx = is_up ? ((aw.e * 2 * IB + half * IB + aw.mb) * KBu + aw.kb)
+                                           : ((aw.e * HB + aw.mb) * KBd + aw.kb);
+                    const size_t off16 = ((size_t)sidx * 4) & ~(size_t)15;
+                    const bool bulk = off16 + 16 <= sbytes;
+                    if (!bulk) {   // last, partial 16-byte chunk of the scale array: fetch the one value directly
+                        const float v = __ldg(sbase + sidx);
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((sidx & 3) * 4)), "f"(v) : "memory");
                     }
+                    mbar_expect_tx(full, stage_tx + (bulk ? 16u : 0u) + (is_up ? 0u : (uint32_t)(N * 4)));
+                    if (bulk) bulk_load(slot, (const char*)sbase + off16, 16u, full);
+                    if (is_up) tma_load_2d(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full);
+                    else tma_load_2d(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full);
+                    ++a_cur;
+                    if (++a_st == S) { a_st = 0; a_ph ^= 1u; }
+                    if (!is_up || half == 1) {
+                        if (++a_slot == kScaleSlots) a_slot = 0;
+                        if (a_cur == n_up_st) { if (a_cur < n_st) aw.init(dn_lo, KBd, HB, s_act); }
+                        else aw.next(s_act);
+                    }
+                    progress = true;
                 }
-                if (b_cur < a_cur) {
-                    const int st = (int)(b_cur % S);
-                    const uint32_t dst = smem_u32(smem + (size_t)st * L.stage_bytes + kATileBytes);
-                    if (b_cur < n_up_st) {
-                        const long long s = up_lo + (b_cur >> 1);
-                        tma_load_2d(dst, &tmXq, (int)(s % KBu) * kBlock, 0, bar_full + 8 * st);
-                        ++b_cur;
-                        progress = true;
+                while (b_cur < a_cur) {
+                    const uint32_t dst = smem_u32(smem + (size_t)b_st * L.stage_bytes + kATileBytes);
+                    const uint32_t full = bar_full + 8 * b_st;
+                    const bool is_up = b_cur < n_up_st;
+                    if (is_up) {
+                        tma_load_2d(dst, &tmXq, bw.kb * kBlock, 0, full);
                     } else {
-                        const long long s = dn_lo + (b_cur - n_up_st);
-                        const int ib = (int)(s % KBd), e = s_act[(int)(s / KBd) / HB];
-                        if (ld_acquire(P.hq_flag + e * IB + ib) == tag) {   // intermediate tile published (Section 3.2)
+                        if (bw.e != ready_e) {                   // intermediate tile published? (Section 3.2)
+                            if (ld_acquire(P.e_ready + bw.e) != tag) break;
                             fence_proxy_async();
-                            tma_load_2d(dst, &tmHq, ib * kBlock, e * N, bar_full + 8 * st);
-                            ++b_cur;
-                            progress = true;
+                            ready_e = bw.e;
                         }
+                        tma_load_2d(dst, &tmHq, bw.kb * kBlock, bw.e * N, full);
+                        bulk_load(sc_base + (uint32_t)b_slot * L.sc_bytes + 32u, P.hs + ((size_t)bw.e * IB + bw.kb) * N,
+                                  (uint32_t)(N * 4), full);
                     }
+                    const bool step_done = !is_up || (b_cur & 1);
+                    ++b_cur;
+                    if (++b_st == S) b_st = 0;
+                    if (step_done) {
+                        if (++b_slot == kScaleSlots) b_slot = 0;
+                        if (b_cur == n_up_st) { if (b_cur < n_st) bw.init(dn_lo, KBd, HB, s_act); }
+                        else bw.next(s_act);
+                    }
+                    progress = true;
                 }
+                if (!stamped) { MOE_STAMP(9); stamped = true; }
                 if (progress) idle = 0;
-                else if ((++idle & 127u) == 0) { if (wt.expired(2)) break; __nanosleep(32); }
+                else if ((++idle & 63u) == 0) { if (wt.expired(2)) break; __nanosleep(40); }
             }
             if (wt.dead) {
                 // give-up path: complete the byte count of half-armed stages, then wait for copies in flight
-                for (long long it = b_cur; it < a_cur; ++it) {
-                    const int st = (int)(it % S);
+                for (int it = b_cur; it < a_cur; ++it) {
+                    const int st = it % S;
                     tma_load_2d(smem_u32(smem + (size_t)st * L.stage_bytes + kATileBytes), &tmXq, 0, 0, bar_full + 8 * st);
+                    if (it >= n_up_st)
+                        bulk_load(sc_base + (uint32_t)((n_up_ks + it - n_up_st) % kScaleSlots) * L.sc_bytes + 32u, P.xq,
+                                  (uint32_t)(N * 4), bar_full + 8 * st);
                 }
-                for (long long it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it) {
-                    const int st = (int)(it % S);
+                for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it) {
+                    const int st = it % S;
                     for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * st, (uint32_t)((it / S) & 1)); ++i) {}
                 }
             }
@@ -532,17 +643,18 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     else if (warp == 1) {
         if (lane == 0 && alive) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
-            long long it = 0, ks = 0;
+            int st = 0, buf = 0;
+            uint32_t ph = 0, tph = 1u;           // full-barrier parity; tmem-empty parity
+            bool first = true;
             for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
-                const long long n_steps = phase == 0 ? (up_hi - up_lo) : (dn_hi - dn_lo);
+                const int n_steps = phase == 0 ? (up_hi - up_lo) : (dn_hi - dn_lo);
                 const int halves = phase == 0 ? 2 : 1;
-                for (long long s = 0; s < n_steps && !wt.dead; ++s, ++ks) {
-                    const int buf = (int)(ks & 1);
-                    if (!wt.mbar(bar_tempty + 8 * buf, (uint32_t)((ks >> 1) & 1) ^ 1u, 3)) break;
+                for (int s = 0; s < n_steps && !wt.dead; ++s) {
+                    if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
                     tc_fence_after();
-                    for (int half = 0; half < halves; ++half, ++it) {
-                        const int st = (int)(it % S);
-                        if (!wt.mbar(bar_full + 8 * st, (uint32_t)((it / S) & 1), 4)) break;
+                    for (int half = 0; half < halves; ++half) {
+                        if (!wt.mbar(bar_full + 8 * st, ph, 4)) break;
+                        if (first) { MOE_STAMP(10); first = false; }
                         tc_fence_after();
                         const uint32_t a_addr = smem_u32(smem + (size_t)st * L.stage_bytes);
                         const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(a_addr + kATileBytes);
@@ -551,9 +663,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         for (int k = 0; k < 4; ++k)
                             umma_f8(d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, k > 0 ? 1u : 0u);
                         umma_commit(bar_empty + 8 * st);      // smem stage reusable once these MMAs retire
+                        if (++st == S) { st = 0; ph ^= 1u; }
                     }
                     if (wt.dead) break;
                     umma_commit(bar_tfull + 8 * buf);          // accumulator of this K block complete
+                    if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
                 }
             }
             if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
@@ -568,68 +682,84 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-        long long ks = 0;
-        float accg[N], accu[N];
+        volatile uint32_t* s_giveup = misc + 3;
+        bool first_acc = true;
+        const float* sc_ring = (const float*)(smem + L.sc_off);
+        const int sc_floats = L.sc_bytes / 4;
+        constexpr int CH = TC < 16 ? TC : 16;                  // columns per TMEM load
+        int buf = 0, slot = 0;
+        uint32_t tph = 0;
+        float accg[TC], accu[TC];
 
         for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
             const bool up = (phase == 0);
-            const long long lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
+            const int lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
             const int KB = up ? KBu : KBd, MB = up ? IB : HB;  // K blocks per unit, row blocks per expert
-            const long long S_all = up ? S_up : S_dn;
+            const int S_all = up ? S_up : S_dn;
             float* part = up ? P.part_up : P.part_dn;
             unsigned* pflag = up ? P.pu_flag : P.pd_flag;
             const int pcols = up ? 2 * N : N;
+            if (!up && etid == 0) MOE_STAMP(12);
+            if (hi <= lo) continue;
+            Walk w;
+            w.init(lo, KB, MB, s_act);
 
-            for (long long s = lo; s < hi && !wt.dead; ++s, ++ks) {
-                const int kb = (int)(s % KB), unit = (int)(s / KB);
-                const int e = s_act[unit / MB], mb = unit % MB;
-                const unsigned long long mask = s_mask[e];
-                if (s == lo || kb == 0) {
+            for (int s = lo; s < hi && !wt.dead;) {
+                // ---- one piece: the k-steps [s, pend) of unit (e, mb), first K block kb0
+                const int e = w.e, mb = w.mb, kb0 = w.kb;
+                const int ustart = s - kb0, uend = ustart + KB;
+                const int pend = uend < hi ? uend : hi;
+                const int gi = up ? ((e * 2 * IB + mb) * KBu + kb0) : ((e * HB + mb) * KBd + kb0);
+                const int ui = (e * 2 * IB + IB + mb) * KBu + kb0;
+                const float* xs_p = s_xs + kb0;
 #pragma unroll
-                    for (int n = 0; n < N; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
-                }
-                // block scales of this K block
-                float wsg, wsu = 0.f;
-                if (up) {
-                    wsg = __ldg(P.W13s + ((size_t)e * 2 * IB + mb) * KBu + kb);
-                    wsu = __ldg(P.W13s + ((size_t)e * 2 * IB + IB + mb) * KBu + kb);
-                } else {
-                    wsg = __ldg(P.W2s + ((size_t)e * HB + mb) * KBd + kb);
-                }
-                const int buf = (int)(ks & 1);
-                if (!epi_all(wt.mbar(bar_tfull + 8 * buf, (uint32_t)((ks >> 1) & 1), 5))) { wt.dead = true; break; }
-                tc_fence_after();
-                const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
+                for (int n = 0; n < TC; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
+
+                for (int i = 0; i < pend - s; ++i) {
+                    // A wait that runs out is recorded and the warp keeps walking in lockstep with the others;
+                    // the piece end below turns the record into a uniform decision to stop.
+                    if (!wt.mbar(bar_tfull + 8 * buf, tph, 5)) *s_giveup = 1u;
+                    tc_fence_after();
+                    if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
+                    const float* rec = sc_ring + slot * sc_floats;      // scale record that arrived with the stage
+                    const float wsg = rec[(gi + i) & 3];
+                    const float wsu = up ? rec[4 + ((ui + i) & 3)] : 0.f;
+                    const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
 #pragma unroll
-                for (int c = 0; c < N; c += 16) {
-                    float dg[16], du[16];
-                    tmem_ld16(tcol + c, dg);
-                    if (up) tmem_ld16(tcol + N + c, du);
-                    tmem_ld_wait();
+                    for (int c = 0; c < TC; c += CH) {
+                        float dg[CH], du[CH];
+                        tmem_ld<CH>(tcol + c, dg);
+                        if (up) tmem_ld<CH>(tcol + N + c, du);
+                        tmem_ld_wait();
+                        if (c + CH == TC) {                             // accumulator is in registers: free the buffer
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                        }
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int n = c + j;
-                        if (n < T) {
-                            const float as = up ? s_xs[n * KBu + kb]
-                                                : (((mask >> n) & 1ull) ? __ldcg(P.hs + ((size_t)e * N + n) * IB + kb) : 0.f);
+                        for (int j = 0; j < CH; ++j) {
+                            const int n = c + j;
+                            const float as = up ? xs_p[n * KBu + i] : rec[8 + n];
                             accg[n] = fmaf(dg[j], wsg * as, accg[n]);
                             if (up) accu[n] = fmaf(du[j], wsu * as, accu[n]);
                         }
                     }
+                    if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
+                    if (++slot == kScaleSlots) slot = 0;
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                const bool unit_done = (pend == uend);
+                s = pend;
+                if (s < hi) { if (unit_done) w.init(s, KB, MB, s_act); }
+                epi_bar();
+                if (*s_giveup) { wt.dead = true; break; }
+                const unsigned long long mask = s_mask[e];
 
-                if (kb != KB - 1 && s != hi - 1) continue;
                 // ---- end of this CTA's piece of the unit: combine split-K partials, then the epilogue
-                const long long ustart = (long long)unit * KB, uend = ustart + KB;
-                const long long pstart = ustart > lo ? ustart : lo;
-                if (pstart != ustart) {
+                if (ustart < lo) {
                     // not the owner: park the partial accumulator, [column][row] so rows are contiguous
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
-                    for (int n = 0; n < N; ++n)
+                    for (int n = 0; n < TC; ++n)
                         if (n < T) {
                             __stcg(dst + n * kBlock + row, accg[n]);
                             if (up) __stcg(dst + (N + n) * kBlock + row, accu[n]);
@@ -639,87 +769,107 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (etid == 0) st_release(pflag + cta, tag);
                     continue;
                 }
-                if (s + 1 < uend) {
-                    // owner of a unit that continues in later CTAs: add their partials in CTA order
-                    for (int c = cta + 1; c < G; ++c) {
-                        const long long clo = range_lo(S_all, c, G), chi = range_lo(S_all, c + 1, G);
-                        if (clo >= uend) break;
-                        if (chi == clo) continue;
-                        const bool got = (etid == 0) ? wt.flag(pflag + c, tag, 6) : true;
-                        if (!epi_all(got)) { wt.dead = true; break; }
+                if (!unit_done) {
+                    // owner of a unit that continues in later CTAs: wait for all of them at once (one thread per
+                    // contributor), then add their partials in CTA order
+                    int c_end = cta + 1;
+                    bool got = true;
+                    for (int base = cta + 1; base < G; base += kEpiThreads) {
+                        const int c = base + etid;
+                        if (c < G) {
+                            const int clo = range_lo(S_all, c, G), chi = range_lo(S_all, c + 1, G);
+                            if (clo < uend && chi > clo) got = wt.flag(pflag + c, tag, 6) && got;
+                        }
+                        if (range_lo(S_all, min(base + kEpiThreads, G), G) >= uend) break;
+                    }
+                    while (c_end < G && range_lo(S_all, c_end, G) < uend) ++c_end;
+                    if (!epi_all(got)) { wt.dead = true; break; }
+                    for (int c = cta + 1; c < c_end; ++c) {
+                        if (range_lo(S_all, c + 1, G) == range_lo(S_all, c, G)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
-                        for (int n = 0; n < N; ++n)
+                        for (int n = 0; n < TC; ++n)
                             if (n < T) {
                                 accg[n] += __ldcg(src + n * kBlock + row);
                                 if (up) accu[n] += __ldcg(src + (N + n) * kBlock + row);
                             }
                     }
-                    if (wt.dead) break;
                 }
                 if (up) {
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
-                    for (int n = 0; n < N; ++n) {
+                    for (int n = 0; n < TC; ++n) {
                         float a = 0.f;
                         if (n < T && ((mask >> n) & 1ull)) {
                             const float g = accg[n];
                             a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
                         }
                         accg[n] = a;
-                        float m = fabsf(a);
+                        if (n < T) {
+                            float m = fabsf(a);
 #pragma unroll
-                        for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                        if (lane == 0) s_red[q * N + n] = m;
+                            for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                            if (lane == 0) s_red[q * N + n] = m;
+                        }
                     }
                     epi_bar();
 #pragma unroll
-                    for (int n = 0; n < N; ++n) {
+                    for (int n = 0; n < TC; ++n) {
                         if (n < T && ((mask >> n) & 1ull)) {
                             const float amax = fmaxf(fmaxf(s_red[n], s_red[N + n]), fmaxf(s_red[2 * N + n], s_red[3 * N + n]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
                             const float2 v = make_float2(__fdiv_rn(accg[n], sc), 0.f);
                             const uint8_t code = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
                             P.hq[((size_t)e * N + n) * I + mb * kBlock + row] = code;
-                            if (row == 0) P.hs[((size_t)e * N + n) * IB + mb] = sc;
+                            if (row == 0) P.hs[((size_t)e * IB + mb) * N + n] = sc;
                         }
                     }
                     fence_proxy_async();
                     __threadfence();
                     epi_bar();
-                    if (etid == 0) st_release(P.hq_flag + e * IB + mb, tag);
+                    if (etid == 0) {
+                        const unsigned old = atomicAdd(P.e_cnt + e, 1u);
+                        if (old == (unsigned)IB - 1u) {        // last I-block of this expert: publish the tile
+                            P.e_cnt[e] = 0u;
+                            __threadfence();
+                            st_release(P.e_ready + e, tag);
+                        }
+                    }
                 } else {
-                    // per-slot result, then the deterministic slot-ordered reduction by the last arriver
+                    // per-slot result of this expert for its routed tokens
 #pragma unroll
-                    for (int n = 0; n < N; ++n) {
+                    for (int n = 0; n < TC; ++n) {
                         if (n < T && ((mask >> n) & 1ull)) {
-                            int slot = 0;
-                            for (int j = 0; j < K; ++j) if (s_ids[n * K + j] == e) slot = j;
-                            __stcg(P.y + ((size_t)n * K + slot) * H + mb * kBlock + row, accg[n]);
+                            int sl = 0;
+                            for (int j = 0; j < K; ++j) if (s_ids[n * K + j] == e) sl = j;
+                            __stcg(P.y + ((size_t)n * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
                     __threadfence();
                     epi_bar();
-                    if (etid == 0) {
-                        const unsigned old = atomicAdd(P.hb_cnt + mb, 1u);
-                        const unsigned last = (old == (unsigned)U - 1u) ? 1u : 0u;
-                        if (last) P.hb_cnt[mb] = 0u;
-                        misc[2] = last;
-                        __threadfence();
-                    }
-                    epi_bar();
-                    if (misc[2]) {
-                        for (int t = 0; t < T; ++t) {
-                            float acc = 0.f;
-                            for (int j = 0; j < K; ++j)
-                                acc = fmaf(s_w[t * K + j], __ldcg(P.y + ((size_t)t * K + j) * H + mb * kBlock + row), acc);
-                            P.out[(size_t)t * H + mb * kBlock + row] = __float2bfloat16_rn(acc);
-                        }
-                    }
-                    epi_bar();
+                    if (etid == 0) st_release(P.dn_done + e * HB + mb, tag);
                 }
             }
         }
+        if (etid == 0) MOE_STAMP(13);
+        // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block) over all CTAs
+        for (int task = cta; task < T * HB && !wt.dead; task += G) {
+            const int t = task / HB, hb = task - t * HB;
+            bool got = true;
+            if (etid < K) got = wt.flag(P.dn_done + s_ids[t * K + etid] * HB + hb, tag, 7);
+            if (!epi_all(got)) { wt.dead = true; break; }
+            float acc = 0.f;
+            const float* yp = P.y + (size_t)t * K * H + hb * kBlock + row;
+            for (int j0 = 0; j0 < K; j0 += 8) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = (j0 + j < K) ? __ldcg(yp + (size_t)(j0 + j) * H) : 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) if (j0 + j < K) acc = fmaf(s_w[t * K + j0 + j], v[j], acc);
+            }
+            P.out[(size_t)t * H + hb * kBlock + row] = __float2bfloat16_rn(acc);
+        }
+        if (etid == 0) MOE_STAMP(14);
     }
 
     // ------------------------------------------------------------------ teardown
@@ -728,6 +878,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
     if (tid == 0) {
+        MOE_STAMP(15);
         __threadfence();
         const unsigned old = atomicAdd(P.ctrl + kExitCnt, 1u);
         if (old == (unsigned)G - 1u) {          // last CTA out: open the next epoch
