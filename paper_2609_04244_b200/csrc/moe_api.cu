@@ -106,7 +106,7 @@ struct moe_plan {
 
     int stages_for(int N, int T) const {
         for (int s = moe::kMaxStages; s >= 2; --s) {
-            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, s);
+            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s);
             if (L.total + 1024 <= smem_optin) return s;
         }
         return 0;
@@ -163,7 +163,7 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
     const int stages = p->stages_for(N, T);
     if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, stages);
+    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages);
     uint8_t* w = static_cast<uint8_t*>(ws);
 
     CUtensorMap m13, m2, mx, mh;
@@ -200,8 +200,6 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
     P.y = reinterpret_cast<float*>(w + L.y);
     P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
-    P.w13s_bytes = (size_t)p->E * (2 * p->I / 128) * (p->H / 128) * 4;
-    P.w2s_bytes = (size_t)p->E * (p->H / 128) * (p->I / 128) * 4;
 
     const int smem_bytes = SL.total + 1024;
     if (T == 1) return launch<16, 1>(p, m13, m2, mx, mh, P, smem_bytes, stream);
@@ -265,7 +263,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
-    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, st).total + 1024;
+    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, I, st).total + 1024;
     const int optin = p->smem_optin;
     if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) ||
         !resident<16, 8>(optin, smem) || !resident<16, 4>(optin, smem) || !resident<16, 2>(optin, smem) ||
@@ -365,7 +363,7 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
     if (grid) *grid = plan->sms;
     if (stages) *stages = st;
     if (n_hw) *n_hw = N;
-    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, st).total + 1024;
+    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st).total + 1024;
     return MOE_OK;
 }
 

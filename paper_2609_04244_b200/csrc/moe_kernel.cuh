@@ -8,11 +8,11 @@
 //             equal contiguous ranges, one per CTA (split-K across CTAs, partial
 //             accumulators exchanged through L2, summed in fixed order)
 //   phase D : down projection, same scheme over (active expert, 128-row block of
-//             H, 128-wide K block of I); input tiles wait on per-(expert,block)
-//             readiness flags published by phase U (Section 3.2, readiness-based
+//             H, 128-wide K block of I); its activation tiles wait on a per-expert
+//             readiness flag published by phase U (Section 3.2, readiness-based
 //             handoff)
-//   reduce  : the CTA that completes the last expert of a 128-row output block
-//             sums the per-slot results in slot order (deterministic)
+//   reduce  : (token, 128-row block) tasks spread over all CTAs sum the per-slot
+//             results in slot order (deterministic, no float atomics)
 //
 // Warp roles (Section 3.3, warp specialisation): warp 0 = TMA producer, warp 1 =
 // tcgen05 MMA issuer, warps 4..7 = accumulator/epilogue warps (one TMEM lane
@@ -41,8 +41,8 @@ constexpr int kATileBytes = kBlock * kBlock;  // 16 KiB of FP8
 constexpr int kMaxTopK = 32;
 constexpr int kMaxExperts = 512;
 constexpr int kMaxTokens = 64;
-constexpr int kTmemBufs = 4;                     // accumulator buffers in TMEM (one K block each)
-constexpr int kScaleSlots = kMaxStages + 8;   // ring of per-k-step scale records, deeper than any producer lead
+constexpr int kTmemBufs = 4;         // accumulator buffers in TMEM (one K block each)
+constexpr int kStampsPerCta = 16;
 
 // control words at the head of the workspace
 enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kRouteReady = 4, kExitCnt = 5, kCtrlWords = 64 };
@@ -76,8 +76,7 @@ struct Params {
     unsigned* pu_flag;  // [grid]
     unsigned* pd_flag;  // [grid]
     float* y;           // [T,K,H]
-    size_t w13s_bytes, w2s_bytes;   // sizes of the block-scale arrays (bound for 16-byte scale fetches)
-    unsigned long long* stamps;     // [grid][8] globaltimer stamps of the phases of the last launch (diagnostics)
+    unsigned long long* stamps;     // [grid][16] globaltimer stamps of the phases of the last launch (diagnostics)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -116,16 +115,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
-// plain bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16), completes on an mbarrier
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-        : "memory");
-}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -202,7 +195,7 @@ __device__ __forceinline__ bool epi_all(bool ok) {
     return r != 0;
 }
 
-#define MOE_STAMP(i) do { P.stamps[(size_t)blockIdx.x * 16 + (i)] = gtime(); } while (0)
+#define MOE_STAMP(i) do { P.stamps[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
 
 // K-major, 128-byte swizzled operand tile (rows of 128 bytes, 8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
@@ -248,24 +241,23 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, xs_off, red_off, misc_off, sc_off, sc_bytes, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, xs_off, hs_off, red_off, misc_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int stages) {
+__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages) {
     SmemLayout L;
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
     int o = stages * L.stage_bytes;
     L.bar_off = o;  o += (2 * kMaxStages + 16) * 8;
     L.misc_off = o; o += 64;
-    L.sc_bytes = 32 + N * 4;                   // [16 B gate/down weight-scale chunk][16 B up chunk][N activation scales]
-    L.sc_off = o;   o += kScaleSlots * L.sc_bytes;
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
     L.act_off = o;  o += (E + 1) * 4;
-    L.xs_off = o;   o += T * (H / kBlock) * 4;
-    L.red_off = o;  o += kWarps * 64 * 4;      // cross-warp reduction scratch (>= 4*64 floats for amax, 8*8 for logits)
+    L.xs_off = o;   o += T * (H / kBlock) * 4;      // input activation scales [T][H/128]
+    L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]
+    L.red_off = o;  o += kWarps * 64 * 4;           // cross-warp reduction scratch
     L.total = o;
     return L;
 }
@@ -299,12 +291,11 @@ __device__ __forceinline__ uint32_t orderable(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-struct Params;
 // Scores and top-k of one token by one warp (Section 4.1 routing policies): softmax over all experts or
 // sigmoid plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots are in
 // (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
-template <int EPL, class ParamsT>
-__device__ __forceinline__ void topk_token(const ParamsT& P, int t, int lane, int* s_ids, float* s_w,
+template <int EPL>
+__device__ __forceinline__ void topk_token(const Params& P, int t, int lane, int* s_ids, float* s_w,
                                            unsigned long long* s_mask, bool write_global) {
     const int E = P.E, K = P.K;
     const float* lg = P.logits + (size_t)t * E;
@@ -324,7 +315,8 @@ __device__ __forceinline__ void topk_token(const ParamsT& P, int t, int lane, in
         for (int j = 0; j < EPL; ++j) {
             const int e = lane + 32 * j;
             ok[j] = (e < E) ? orderable(l[j]) : 0u;
-            sum += (e < E) ? expf(l[j] - mx) : 0.f;
+            l[j] = (e < E) ? expf(l[j] - mx) : 0.f;
+            sum += l[j];
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -333,29 +325,29 @@ __device__ __forceinline__ void topk_token(const ParamsT& P, int t, int lane, in
         for (int j = 0; j < EPL; ++j) {
             const int e = lane + 32 * j;
             if (e < E) {
-                const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l[j]));
-                ok[j] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
-            } else ok[j] = 0u;
+                l[j] = __fdiv_rn(1.0f, 1.0f + expf(-l[j]));
+                ok[j] = orderable(l[j] + (P.bias ? __ldg(P.bias + e) : 0.f));
+            } else { ok[j] = 0u; l[j] = 0.f; }
         }
+        sum = 1.0f;
     }
+    // l[] now holds the unnormalised score of each expert (exp(logit - max) or the sigmoid)
     int myid = 0;
+    float v = 0.f;
     for (int k = 0; k < K; ++k) {
         uint32_t best = 0u;
         int bj = 0;
+        float bv = 0.f;
 #pragma unroll
-        for (int j = 0; j < EPL; ++j) if (ok[j] > best) { best = ok[j]; bj = j; }   // strict '>' keeps the lowest index
+        for (int j = 0; j < EPL; ++j) if (ok[j] > best) { best = ok[j]; bj = j; bv = l[j]; }   // strict '>' keeps the lowest index
         const uint32_t wmax = __reduce_max_sync(0xffffffffu, best);
         const uint32_t cand = (best == wmax && best != 0u) ? (uint32_t)(lane + 32 * bj) : 0xFFFFFFFFu;
         uint32_t win = __reduce_min_sync(0xffffffffu, cand);
         if (win == 0xFFFFFFFFu) win = (uint32_t)k;                                     // only with NaN logits
+        const float wv = __shfl_sync(0xffffffffu, bv, (int)(win & 31u));
 #pragma unroll
         for (int j = 0; j < EPL; ++j) if ((uint32_t)(lane + 32 * j) == win) ok[j] = 0u;
-        if (lane == k) myid = (int)win;
-    }
-    float v = 0.f;
-    if (lane < K) {
-        const float lv = __ldcg(lg + myid);
-        v = (P.scoring == 0) ? __fdiv_rn(expf(lv - mx), sum) : __fdiv_rn(1.0f, 1.0f + expf(-lv));
+        if (lane == k) { myid = (int)win; v = __fdiv_rn(wv, sum); }
     }
     float vsum = v;
 #pragma unroll
@@ -378,10 +370,33 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
     return lo | (hi << 16);
 }
 
+// dot products of one router row with up to 8 tokens, this thread's share of H (16-byte chunks strided by the block)
+__device__ __forceinline__ void router_partial(const Params& P, int e, int t0, int tid, float* acc) {
+    const int H = P.H, T = P.T;
+    const uint4* wrow = reinterpret_cast<const uint4*>(P.Wr + (size_t)e * H);
+#pragma unroll 2
+    for (int c = tid; c < H / 8; c += kThreads) {
+        const uint4 wv = __ldg(wrow + c);
+        const uint32_t wr[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (t0 + j < T) {
+                const uint4 xv = __ldg(reinterpret_cast<const uint4*>(P.hidden + (size_t)(t0 + j) * H) + c);
+                const uint32_t xr[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    acc[j] = fmaf(__uint_as_float(wr[q] << 16), __uint_as_float(xr[q] << 16), acc[j]);
+                    acc[j] = fmaf(__uint_as_float(wr[q] & 0xFFFF0000u), __uint_as_float(xr[q] & 0xFFFF0000u), acc[j]);
+                }
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // the kernel
-// ---------------------------------------------------------------------------------------------
 // N  = MMA N (token tile, 16/32/64); TC = token columns the accumulator warps actually read (power of two >= T).
+// ---------------------------------------------------------------------------------------------
 template <int N, int TC>
 __global__ void __launch_bounds__(kThreads, 1)
 moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
@@ -395,7 +410,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock, KBd = IB;
     const int S = P.stages;
-    const SmemLayout L = smem_layout(N, T, K, E, H, S);
+    const SmemLayout L = smem_layout(N, T, K, E, H, I, S);
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
@@ -407,6 +422,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
     int* s_act = (int*)(smem + L.act_off);
     float* s_xs = (float*)(smem + L.xs_off);
+    float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
 
     Waiter wt;
@@ -419,11 +435,13 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
         for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
-        misc[3] = 0u;
         mbar_init(bar_drain, 1);
+        misc[3] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
+    for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
+    if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
     // ------------------------------------------------------------------ phase R: quantise + logits
     {
@@ -442,40 +460,31 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (lane == 0) P.xs[p] = s;
         }
         if (tid == 0) MOE_STAMP(1);
-        // router logits: CTA c owns experts c, c+G, ...; all 256 threads split H  (Section 3.3)
-        for (int e = cta; e < E; e += G) {
+        // router logits: CTA c owns experts c, c+G, ...; two experts at a time, all 256 threads split H  (Section 3.3)
+        for (int e0 = cta; e0 < E; e0 += 2 * G) {
+            const int e1 = e0 + G;
+            const bool two = e1 < E;
             for (int t0 = 0; t0 < T; t0 += 8) {
-                float acc[8];
+                float acc0[8], acc1[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-                for (int c = tid; c < H / 8; c += kThreads) {
-                    const uint4 wv = __ldg(reinterpret_cast<const uint4*>(P.Wr + (size_t)e * H) + c);
-                    const uint32_t wr[4] = {wv.x, wv.y, wv.z, wv.w};
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (t0 + j < T) {
-                            const uint4 xv = __ldg(reinterpret_cast<const uint4*>(P.hidden + (size_t)(t0 + j) * H) + c);
-                            const uint32_t xr[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                acc[j] = fmaf(__uint_as_float(wr[q] << 16), __uint_as_float(xr[q] << 16), acc[j]);
-                                acc[j] = fmaf(__uint_as_float(wr[q] & 0xFFFF0000u), __uint_as_float(xr[q] & 0xFFFF0000u), acc[j]);
-                            }
-                        }
-                    }
-                }
+                for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+                router_partial(P, e0, t0, tid, acc0);
+                if (two) router_partial(P, e1, t0, tid, acc1);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
 #pragma unroll
-                    for (int o = 16; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-                    if (lane == 0) s_red[warp * 8 + j] = acc[j];
+                    for (int o = 16; o; o >>= 1) {
+                        acc0[j] += __shfl_xor_sync(0xffffffffu, acc0[j], o);
+                        acc1[j] += __shfl_xor_sync(0xffffffffu, acc1[j], o);
+                    }
+                    if (lane == 0) { s_red[warp * 16 + j] = acc0[j]; s_red[warp * 16 + 8 + j] = acc1[j]; }
                 }
                 __syncthreads();
-                if (tid < 8 && t0 + tid < T) {
+                if (tid < 16 && t0 + (tid & 7) < T && (tid < 8 || two)) {
                     float v = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kWarps; ++w) v += s_red[w * 8 + tid];
-                    P.logits[(size_t)(t0 + tid) * E + e] = v;
+                    for (int w = 0; w < kWarps; ++w) v += s_red[w * 16 + tid];
+                    P.logits[(size_t)(t0 + (tid & 7)) * E + (tid < 8 ? e0 : e1)] = v;
                 }
                 __syncthreads();
             }
@@ -506,10 +515,6 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     // ------------------------------------------------------------------ top-k + routing metadata (every CTA)
     if (alive) {
-        for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
-        for (int i = tid; i < T * KBu; i += kThreads) s_xs[i] = __ldcg(P.xs + i);
-        __syncthreads();
-        if (tid == 0) MOE_STAMP(5);
         const bool wg = (cta == 0);
         for (int t = warp; t < T; t += kWarps) {
             if (E <= 32) topk_token<1>(P, t, lane, s_ids, s_w, s_mask, wg);
@@ -518,6 +523,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             else if (E <= 256) topk_token<8>(P, t, lane, s_ids, s_w, s_mask, wg);
             else topk_token<16>(P, t, lane, s_ids, s_w, s_mask, wg);
         }
+        for (int i = tid; i < T * KBu; i += kThreads) s_xs[i] = __ldcg(P.xs + i);
         __syncthreads();
         if (tid == 0) MOE_STAMP(6);
         if (warp == 0) {                                   // active-expert list in ascending expert order
@@ -538,23 +544,20 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int S_up = U * IB * KBu, S_dn = U * HB * KBd;     // k-steps of the two projections (host checks the range)
     const int up_lo = range_lo(S_up, cta, G), up_hi = range_lo(S_up, cta + 1, G);
     const int dn_lo = range_lo(S_dn, cta, G), dn_hi = range_lo(S_dn, cta + 1, G);
-    const uint32_t stage_tx = (uint32_t)L.stage_bytes;
 
     // ------------------------------------------------------------------ role: TMA producer
     if (warp == 0) {
         if (lane == 0 && alive) {
             // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.
-            // Every stage = weight tile + activation tile + the block scales its K block needs (a 16-byte chunk of
-            // the weight-scale array and, in the down phase, the N activation scales), all on one mbarrier.
-            // Weight tiles (cursor A) run ahead of activation tiles (cursor B): only the latter wait for the
-            // intermediate tile of the up projection to be published.
+            // A stage = one 128x128 weight tile + one Nx128 activation tile on one mbarrier; the up tile of a
+            // k-step reuses the activation tile of its gate stage.  Weight tiles (cursor A) run ahead of
+            // activation tiles (cursor B): only the latter wait for the up projection's intermediate tile.
             fence_proxy_async();                 // xq was written with ordinary stores by other CTAs
-            const int n_up_ks = up_hi - up_lo, n_up_st = 2 * n_up_ks, n_st = n_up_st + (dn_hi - dn_lo);
-            const uint32_t sc_base = smem_u32(smem + L.sc_off);
+            const int n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
             Walk aw, bw;
-            int a_cur = 0, a_st = 0, a_slot = 0, b_cur = 0, b_st = 0, b_slot = 0;
+            int a_cur = 0, a_st = 0, b_cur = 0, b_st = 0;
             uint32_t a_ph = 1u;                  // parity to wait for on the empty barrier
-            if (n_up_ks > 0) { aw.init(up_lo, KBu, IB, s_act); bw = aw; }
+            if (n_up_st > 0) { aw.init(up_lo, KBu, IB, s_act); bw = aw; }
             else if (n_st > 0) { aw.init(dn_lo, KBd, HB, s_act); bw = aw; }
             int ready_e = -1;                    // expert whose intermediate tile is known to be published
             uint32_t idle = 0;
@@ -566,38 +569,30 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (!mbar_try_wait(bar_empty + 8 * a_st, a_ph)) break;
                     const uint32_t dst = smem_u32(smem + (size_t)a_st * L.stage_bytes);
                     const uint32_t full = bar_full + 8 * a_st;
-                    const bool is_up = a_cur < n_up_st;
-                    const int half = is_up ? (a_cur & 1) : 0;
-                    const uint32_t slot = sc_base + (uint32_t)a_slot * L.sc_bytes + 16u * half;
-                    const float* sbase = is_up ? P.W13s : P.W2s;
-                    const size_t sbytes = is_up ? P.w13s_bytes : P.w2s_bytes;
-                    const int sidx = is_up ? ((aw.e * 2 * IB + half * IB + aw.mb) * KBu + aw.kb)
-                                           : ((aw.e * HB + aw.mb) * KBd + aw.kb);
-                    const size_t off16 = ((size_t)sidx * 4) & ~(size_t)15;
-                    const bool bulk = off16 + 16 <= sbytes;
-                    if (!bulk) {   // last, partial 16-byte chunk of the scale array: fetch the one value directly
-                        const float v = __ldg(sbase + sidx);
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot + (uint32_t)((sidx & 3) * 4)), "f"(v) : "memory");
+                    if (a_cur < n_up_st) {
+                        const int half = a_cur & 1;
+                        mbar_expect_tx(full, (uint32_t)kATileBytes + (half ? 0u : (uint32_t)(N * kBlock)));
+                        tma_load_2d(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full);
+                        ++a_cur;
+                        if (half) { if (a_cur == n_up_st) { if (a_cur < n_st) aw.init(dn_lo, KBd, HB, s_act); } else aw.next(s_act); }
+                    } else {
+                        mbar_expect_tx(full, (uint32_t)(kATileBytes + N * kBlock));
+                        tma_load_2d(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full);
+                        ++a_cur;
+                        aw.next(s_act);
                     }
-                    mbar_expect_tx(full, stage_tx + (bulk ? 16u : 0u) + (is_up ? 0u : (uint32_t)(N * 4)));
-                    if (bulk) bulk_load(slot, (const char*)sbase + off16, 16u, full);
-                    if (is_up) tma_load_2d(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full);
-                    else tma_load_2d(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full);
-                    ++a_cur;
                     if (++a_st == S) { a_st = 0; a_ph ^= 1u; }
-                    if (!is_up || half == 1) {
-                        if (++a_slot == kScaleSlots) a_slot = 0;
-                        if (a_cur == n_up_st) { if (a_cur < n_st) aw.init(dn_lo, KBd, HB, s_act); }
-                        else aw.next(s_act);
-                    }
                     progress = true;
                 }
                 while (b_cur < a_cur) {
                     const uint32_t dst = smem_u32(smem + (size_t)b_st * L.stage_bytes + kATileBytes);
                     const uint32_t full = bar_full + 8 * b_st;
-                    const bool is_up = b_cur < n_up_st;
-                    if (is_up) {
-                        tma_load_2d(dst, &tmXq, bw.kb * kBlock, 0, full);
+                    if (b_cur < n_up_st) {
+                        if ((b_cur & 1) == 0) {
+                            tma_load_2d(dst, &tmXq, bw.kb * kBlock, 0, full);
+                        } else {
+                            if (b_cur + 1 == n_up_st) { if (b_cur + 1 < n_st) bw.init(dn_lo, KBd, HB, s_act); } else bw.next(s_act);
+                        }
                     } else {
                         if (bw.e != ready_e) {                   // intermediate tile published? (Section 3.2)
                             if (ld_acquire(P.e_ready + bw.e) != tag) break;
@@ -605,17 +600,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             ready_e = bw.e;
                         }
                         tma_load_2d(dst, &tmHq, bw.kb * kBlock, bw.e * N, full);
-                        bulk_load(sc_base + (uint32_t)b_slot * L.sc_bytes + 32u, P.hs + ((size_t)bw.e * IB + bw.kb) * N,
-                                  (uint32_t)(N * 4), full);
+                        bw.next(s_act);
                     }
-                    const bool step_done = !is_up || (b_cur & 1);
                     ++b_cur;
                     if (++b_st == S) b_st = 0;
-                    if (step_done) {
-                        if (++b_slot == kScaleSlots) b_slot = 0;
-                        if (b_cur == n_up_st) { if (b_cur < n_st) bw.init(dn_lo, KBd, HB, s_act); }
-                        else bw.next(s_act);
-                    }
                     progress = true;
                 }
                 if (!stamped) { MOE_STAMP(9); stamped = true; }
@@ -625,11 +613,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (wt.dead) {
                 // give-up path: complete the byte count of half-armed stages, then wait for copies in flight
                 for (int it = b_cur; it < a_cur; ++it) {
+                    if (it < n_up_st && (it & 1)) continue;
                     const int st = it % S;
                     tma_load_2d(smem_u32(smem + (size_t)st * L.stage_bytes + kATileBytes), &tmXq, 0, 0, bar_full + 8 * st);
-                    if (it >= n_up_st)
-                        bulk_load(sc_base + (uint32_t)((n_up_ks + it - n_up_st) % kScaleSlots) * L.sc_bytes + 32u, P.xq,
-                                  (uint32_t)(N * 4), bar_full + 8 * st);
                 }
                 for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it) {
                     const int st = it % S;
@@ -643,32 +629,44 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     else if (warp == 1) {
         if (lane == 0 && alive) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
+            const uint32_t ring = smem_u32(smem);
             int st = 0, buf = 0;
             uint32_t ph = 0, tph = 1u;           // full-barrier parity; tmem-empty parity
             bool first = true;
-            for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
-                const int n_steps = phase == 0 ? (up_hi - up_lo) : (dn_hi - dn_lo);
-                const int halves = phase == 0 ? 2 : 1;
-                for (int s = 0; s < n_steps && !wt.dead; ++s) {
-                    if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
-                    tc_fence_after();
-                    for (int half = 0; half < halves; ++half) {
-                        if (!wt.mbar(bar_full + 8 * st, ph, 4)) break;
-                        if (first) { MOE_STAMP(10); first = false; }
-                        tc_fence_after();
-                        const uint32_t a_addr = smem_u32(smem + (size_t)st * L.stage_bytes);
-                        const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(a_addr + kATileBytes);
-                        const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N + half * N);
+            const int n_up = up_hi - up_lo, n_dn = dn_hi - dn_lo;
+            for (int s = 0; s < n_up + n_dn && !wt.dead; ++s) {
+                const bool up = s < n_up;
+                if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
+                const int st0 = st;
+                const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)L.stage_bytes;
+                if (!wt.mbar(bar_full + 8 * st0, ph, 4)) break;
+                if (++st == S) { st = 0; ph ^= 1u; }
+                const uint64_t b_desc = make_smem_desc(a0 + kATileBytes);
+                const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
+                if (first) { MOE_STAMP(10); first = false; }
+                tc_fence_after();
+                {
+                    const uint64_t a_desc = make_smem_desc(a0);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_f8(d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, k > 0 ? 1u : 0u);
-                        umma_commit(bar_empty + 8 * st);      // smem stage reusable once these MMAs retire
-                        if (++st == S) { st = 0; ph ^= 1u; }
-                    }
-                    if (wt.dead) break;
-                    umma_commit(bar_tfull + 8 * buf);          // accumulator of this K block complete
-                    if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
+                    for (int k = 0; k < 4; ++k)
+                        umma_f8(d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, k > 0 ? 1u : 0u);
                 }
+                if (up) {                                      // up tile of the same K block, same activation tile
+                    const int st1 = st;
+                    if (!wt.mbar(bar_full + 8 * st1, ph, 4)) break;
+                    if (++st == S) { st = 0; ph ^= 1u; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_smem_desc(ring + (uint32_t)st1 * (uint32_t)L.stage_bytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_f8(d + N, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, k > 0 ? 1u : 0u);
+                    umma_commit(bar_empty + 8 * st0);          // both stages reusable once all eight MMAs retire
+                    umma_commit(bar_empty + 8 * st1);
+                } else {
+                    umma_commit(bar_empty + 8 * st0);
+                }
+                umma_commit(bar_tfull + 8 * buf);              // accumulator of this K block complete
+                if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
             }
             if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
                 umma_commit(bar_drain);
@@ -684,10 +682,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         volatile uint32_t* s_giveup = misc + 3;
         bool first_acc = true;
-        const float* sc_ring = (const float*)(smem + L.sc_off);
-        const int sc_floats = L.sc_bytes / 4;
         constexpr int CH = TC < 16 ? TC : 16;                  // columns per TMEM load
-        int buf = 0, slot = 0;
+        int buf = 0, hs_e = -1;
         uint32_t tph = 0;
         float accg[TC], accu[TC];
 
@@ -704,26 +700,55 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             Walk w;
             w.init(lo, KB, MB, s_act);
 
+            // Block scales of the weight tiles: lane l of every warp holds the scales of k-step (32*block + l) of
+            // this CTA's range and hands them out by shuffle; the next block of 32 is fetched one block ahead.
+            auto fetch_scales = [&](int sidx, float& g, float& u2) {
+                g = 0.f; u2 = 0.f;
+                if (sidx < hi) {
+                    const int unit = sidx / KB, kb = sidx - unit * KB, uu = unit / MB, mb = unit - uu * MB, e = s_act[uu];
+                    if (up) {
+                        g = __ldg(P.W13s + ((size_t)e * 2 * IB + mb) * KBu + kb);
+                        u2 = __ldg(P.W13s + ((size_t)e * 2 * IB + IB + mb) * KBu + kb);
+                    } else {
+                        g = __ldg(P.W2s + ((size_t)e * HB + mb) * KBd + kb);
+                    }
+                }
+            };
+            float sg_cur, su_cur, sg_nxt, su_nxt;
+            fetch_scales(lo + lane, sg_cur, su_cur);
+            fetch_scales(lo + 32 + lane, sg_nxt, su_nxt);
+
             for (int s = lo; s < hi && !wt.dead;) {
                 // ---- one piece: the k-steps [s, pend) of unit (e, mb), first K block kb0
                 const int e = w.e, mb = w.mb, kb0 = w.kb;
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
-                const int gi = up ? ((e * 2 * IB + mb) * KBu + kb0) : ((e * HB + mb) * KBd + kb0);
-                const int ui = (e * 2 * IB + IB + mb) * KBu + kb0;
-                const float* xs_p = s_xs + kb0;
+                if (!up && e != hs_e) {
+                    // activation scales of this expert's intermediate tile -> shared memory (once per expert)
+                    const bool got = (etid == 0) ? wt.flag(P.e_ready + e, tag, 8) : true;
+                    if (!epi_all(got)) { wt.dead = true; break; }
+                    for (int i = etid; i < IB * N; i += kEpiThreads) s_hs[i] = __ldcg(P.hs + (size_t)e * IB * N + i);
+                    hs_e = e;
+                    epi_bar();
+                }
+                const float* as_p = up ? (s_xs + kb0) : (s_hs + kb0 * N);
+                const int as_tok = up ? KBu : 1, as_step = up ? 1 : N;
 #pragma unroll
                 for (int n = 0; n < TC; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
                 for (int i = 0; i < pend - s; ++i) {
+                    const int j = (s + i - lo) & 31;
+                    if (j == 0 && s + i != lo) {
+                        sg_cur = sg_nxt; su_cur = su_nxt;
+                        fetch_scales(s + i + 32 + lane, sg_nxt, su_nxt);
+                    }
+                    const float wsg = __shfl_sync(0xffffffffu, sg_cur, j);
+                    const float wsu = __shfl_sync(0xffffffffu, su_cur, j);
                     // A wait that runs out is recorded and the warp keeps walking in lockstep with the others;
                     // the piece end below turns the record into a uniform decision to stop.
                     if (!wt.mbar(bar_tfull + 8 * buf, tph, 5)) *s_giveup = 1u;
                     tc_fence_after();
                     if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
-                    const float* rec = sc_ring + slot * sc_floats;      // scale record that arrived with the stage
-                    const float wsg = rec[(gi + i) & 3];
-                    const float wsu = up ? rec[4 + ((ui + i) & 3)] : 0.f;
                     const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
 #pragma unroll
                     for (int c = 0; c < TC; c += CH) {
@@ -737,19 +762,18 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
                         }
 #pragma unroll
-                        for (int j = 0; j < CH; ++j) {
-                            const int n = c + j;
-                            const float as = up ? xs_p[n * KBu + i] : rec[8 + n];
-                            accg[n] = fmaf(dg[j], wsg * as, accg[n]);
-                            if (up) accu[n] = fmaf(du[j], wsu * as, accu[n]);
+                        for (int jj = 0; jj < CH; ++jj) {
+                            const int n = c + jj;
+                            const float as = as_p[n * as_tok + i * as_step];
+                            accg[n] = fmaf(dg[jj], wsg * as, accg[n]);
+                            if (up) accu[n] = fmaf(du[jj], wsu * as, accu[n]);
                         }
                     }
                     if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
-                    if (++slot == kScaleSlots) slot = 0;
                 }
                 const bool unit_done = (pend == uend);
                 s = pend;
-                if (s < hi) { if (unit_done) w.init(s, KB, MB, s_act); }
+                if (s < hi && unit_done) w.init(s, KB, MB, s_act);
                 epi_bar();
                 if (*s_giveup) { wt.dead = true; break; }
                 const unsigned long long mask = s_mask[e];
@@ -841,7 +865,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     for (int n = 0; n < TC; ++n) {
                         if (n < T && ((mask >> n) & 1ull)) {
                             int sl = 0;
-                            for (int j = 0; j < K; ++j) if (s_ids[n * K + j] == e) sl = j;
+                            for (int jj = 0; jj < K; ++jj) if (s_ids[n * K + jj] == e) sl = jj;
                             __stcg(P.y + ((size_t)n * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
