@@ -54,7 +54,7 @@ bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t ctrl, e_cnt, e_ready, dn_done, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
+    size_t ctrl, e_cnt, dn_done, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
     size_t stamps, logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, total;
 };
 
@@ -83,8 +83,7 @@ struct moe_plan {
         WsLayout L;
         size_t o = 0;
         L.ctrl = o;     o += moe::kCtrlWords * 4;
-        L.e_cnt = o;    o += align_up((size_t)E * 4, 256);
-        L.e_ready = o;  o += align_up((size_t)E * 4, 256);
+        L.e_cnt = o;    o += align_up((size_t)2 * E * 4, 256);
         L.dn_done = o;  o += align_up((size_t)E * (H / 128) * 4, 256);
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
@@ -192,7 +191,6 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.hq = w + L.hq;
     P.hs = reinterpret_cast<float*>(w + L.hs);
     P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
-    P.e_ready = reinterpret_cast<unsigned*>(w + L.e_ready);
     P.dn_done = reinterpret_cast<unsigned*>(w + L.dn_done);
     P.part_up = reinterpret_cast<float*>(w + L.part_up);
     P.part_dn = reinterpret_cast<float*>(w + L.part_dn);

@@ -45,7 +45,8 @@ constexpr int kTmemBufs = 4;         // accumulator buffers in TMEM (one K block
 constexpr int kStampsPerCta = 16;
 
 // control words at the head of the workspace
-enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kRouteReady = 4, kExitCnt = 5, kCtrlWords = 64 };
+// (the two arrival counters are used by alternate launches: a launch counts in one and clears the other)
+enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kExitCnt = 5, kCtrlWords = 64 };
 // device status codes
 enum DevStatus { kDevOk = 0, kDevTimeout = 1 };
 
@@ -68,8 +69,7 @@ struct Params {
     float* xs;          // [T,H/128]
     uint8_t* hq;        // [E,N,I]
     float* hs;          // [E,I/128,N]
-    unsigned* e_cnt;    // [E]   published I-blocks of an expert's intermediate tile
-    unsigned* e_ready;  // [E]   == tag once the whole intermediate tile of the expert is published
+    unsigned* e_cnt;    // [2][E] published I-blocks of an expert's intermediate tile (one row per launch parity)
     unsigned* dn_done;  // [E,H/128] == tag once the expert's down-projection rows of that block are stored
     float* part_up;     // [grid][2N][128]
     float* part_dn;     // [grid][N][128]
@@ -114,6 +114,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
+}
+// same, with an L2 eviction-priority hint (weights are read exactly once per step: evict them first, so that the
+// small hot data -- flags, partial sums, activation tiles, the kernel's own instructions -- stays in L2)
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -173,6 +186,9 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -291,74 +307,93 @@ __device__ __forceinline__ uint32_t orderable(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Scores and top-k of one token by one warp (Section 4.1 routing policies): softmax over all experts or
-// sigmoid plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots are in
-// (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
-template <int EPL>
-__device__ __forceinline__ void topk_token(const Params& P, int t, int lane, int* s_ids, float* s_w,
-                                           unsigned long long* s_mask, bool write_global) {
-    const int E = P.E, K = P.K;
-    const float* lg = P.logits + (size_t)t * E;
-    uint32_t ok[EPL];
-    float l[EPL];
-    float mx = -INFINITY, sum = 0.f;
-#pragma unroll
-    for (int j = 0; j < EPL; ++j) {
-        const int e = lane + 32 * j;
-        l[j] = (e < E) ? __ldcg(lg + e) : -INFINITY;
-        mx = fmaxf(mx, l[j]);
-    }
-    if (P.scoring == 0) {
-#pragma unroll
-        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-#pragma unroll
-        for (int j = 0; j < EPL; ++j) {
-            const int e = lane + 32 * j;
-            ok[j] = (e < E) ? orderable(l[j]) : 0u;
-            l[j] = (e < E) ? expf(l[j] - mx) : 0.f;
-            sum += l[j];
+// Scores and top-k for a few tokens at a time by the whole CTA (Section 4.1 routing policies): softmax over all
+// experts or sigmoid plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots
+// are in (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
+// Selection is by rank in two levels: a warp ranks the 32 experts of one segment against each other by shuffles
+// and keeps the best min(K,32) as candidates; then every candidate counts the candidates of its token that beat
+// it (larger key, or equal key and lower index) and takes that slot if the count is below K.
+// The softmax key is the logit itself; its normaliser is only summed when the weights are not renormalised
+// (it cancels otherwise), with the largest logit -- slot 0 -- as the shift.
+// Shared-memory scratch per token: E keys, E scores, ceil(E/32) * min(K,32) 64-bit candidates.
+__device__ __forceinline__ int route_scratch_words(int E, int K) { return 2 * E + 2 * ((E + 31) / 32) * (K < 32 ? K : 32); }
+
+__device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int tid, uint32_t* scratch, int* s_ids,
+                                             float* s_w, unsigned long long* s_mask, bool write_global) {
+    const int E = P.E, K = P.K, warp = tid >> 5, lane = tid & 31;
+    const int nseg = (E + 31) / 32, Kc = K < 32 ? K : 32, C = nseg * Kc;
+    uint32_t* s_key = scratch;
+    float* s_val = reinterpret_cast<float*>(scratch + nt * E);
+    // candidates are packed as (key << 32 | ~index): "a beats b" is then one 64-bit compare
+    unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
+    const bool softmax = (P.scoring == 0);
+    for (int p = tid; p < nt * E; p += kThreads) {
+        const float l = __ldcg(P.logits + (size_t)t0 * E + p);
+        if (softmax) {
+            s_val[p] = l;
+            s_key[p] = orderable(l);
+        } else {
+            const int e = p % E;
+            const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
+            s_val[p] = sg;
+            s_key[p] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
         }
+    }
+    __syncthreads();
+    for (int seg = warp; seg < nt * nseg; seg += kWarps) {  // level 1: rank inside a 32-expert segment
+        const int t = seg / nseg, sg = seg - t * nseg, e = sg * 32 + lane;
+        const uint32_t my = (e < E) ? s_key[t * E + e] : 0u;
+        int lr = 0;
 #pragma unroll
-        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    } else {
-#pragma unroll
-        for (int j = 0; j < EPL; ++j) {
-            const int e = lane + 32 * j;
-            if (e < E) {
-                l[j] = __fdiv_rn(1.0f, 1.0f + expf(-l[j]));
-                ok[j] = orderable(l[j] + (P.bias ? __ldg(P.bias + e) : 0.f));
-            } else { ok[j] = 0u; l[j] = 0.f; }
+        for (int i = 0; i < 32; ++i) {
+            const uint32_t ko = __shfl_sync(0xffffffffu, my, i);
+            lr += (int)(ko > my) | ((int)(ko == my) & (int)(i < lane));
         }
-        sum = 1.0f;
+        if (lr < Kc) cand[t * C + sg * Kc + lr] = ((unsigned long long)my << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)e);
     }
-    // l[] now holds the unnormalised score of each expert (exp(logit - max) or the sigmoid)
-    int myid = 0;
-    float v = 0.f;
-    for (int k = 0; k < K; ++k) {
-        uint32_t best = 0u;
-        int bj = 0;
-        float bv = 0.f;
+    __syncthreads();
+    for (int p = tid; p < nt * C; p += kThreads) {          // level 2: rank among the token's candidates
+        const int t = p / C;
+        const unsigned long long* ck = cand + t * C;
+        const unsigned long long my = cand[p];
+        const int me = (int)(0xFFFFFFFFu - (uint32_t)my);
+        int rank = 0;
+        for (int o0 = 0; o0 < C; o0 += 8) {
+            unsigned long long v[8];
 #pragma unroll
-        for (int j = 0; j < EPL; ++j) if (ok[j] > best) { best = ok[j]; bj = j; bv = l[j]; }   // strict '>' keeps the lowest index
-        const uint32_t wmax = __reduce_max_sync(0xffffffffu, best);
-        const uint32_t cand = (best == wmax && best != 0u) ? (uint32_t)(lane + 32 * bj) : 0xFFFFFFFFu;
-        uint32_t win = __reduce_min_sync(0xffffffffu, cand);
-        if (win == 0xFFFFFFFFu) win = (uint32_t)k;                                     // only with NaN logits
-        const float wv = __shfl_sync(0xffffffffu, bv, (int)(win & 31u));
+            for (int j = 0; j < 8; ++j) v[j] = (o0 + j < C) ? ck[o0 + j] : 0ull;
 #pragma unroll
-        for (int j = 0; j < EPL; ++j) if ((uint32_t)(lane + 32 * j) == win) ok[j] = 0u;
-        if (lane == k) { myid = (int)win; v = __fdiv_rn(wv, sum); }
+            for (int j = 0; j < 8; ++j) rank += (int)(v[j] > my);
+        }
+        if (rank < K && me < E) { s_ids[(t0 + t) * K + rank] = me; s_w[(t0 + t) * K + rank] = s_val[t * E + me]; }
     }
-    float vsum = v;
+    __syncthreads();
+    if (warp < nt) {                                       // weights of the selected experts, one warp per token
+        const int t = t0 + warp;
+        float v = (lane < K) ? s_w[t * K + lane] : 0.f;
+        float total = 1.0f;
+        if (softmax) {
+            const float mx = __shfl_sync(0xffffffffu, v, 0);          // slot 0 holds the largest logit
+            v = (lane < K) ? expf(v - mx) : 0.f;
+            if (!P.renorm) {
+                total = 0.f;
+                for (int e = lane; e < E; e += 32) total += expf(s_val[warp * E + e] - mx);
 #pragma unroll
-    for (int o = 16; o; o >>= 1) vsum += __shfl_xor_sync(0xffffffffu, vsum, o);
-    if (lane < K) {
-        const float w = (P.renorm ? __fdiv_rn(v, vsum) : v) * P.routed_scale;
-        s_ids[t * K + lane] = myid;
-        s_w[t * K + lane] = w;
-        atomicOr(&s_mask[myid], 1ull << t);
-        if (write_global) { P.ids[t * K + lane] = myid; P.wts[t * K + lane] = w; }
+                for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+            }
+        }
+        float vsum = v;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) vsum += __shfl_xor_sync(0xffffffffu, vsum, o);
+        if (lane < K) {
+            const int id = s_ids[t * K + lane];
+            const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
+            s_w[t * K + lane] = w;
+            atomicOr(&s_mask[id], 1ull << t);
+            if (write_global) { P.ids[t * K + lane] = id; P.wts[t * K + lane] = w; }
+        }
     }
+    __syncthreads();
 }
 
 // quantise 4 floats with scale s into 4 E4M3 bytes (memory order x0..x3)
@@ -370,14 +405,16 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
     return lo | (hi << 16);
 }
 
-// dot products of one router row with up to 8 tokens, this thread's share of H (16-byte chunks strided by the block)
-__device__ __forceinline__ void router_partial(const Params& P, int e, int t0, int tid, float* acc) {
+// dot products of two router rows (e0 and, if `two`, e1) with up to 8 tokens: this thread's share of H
+// (16-byte chunks strided by the block); both rows travel together so that all loads are in flight at once
+__device__ __forceinline__ void router_partial(const Params& P, int e0, int e1, bool two, int t0, int tid, float* acc0, float* acc1) {
     const int H = P.H, T = P.T;
-    const uint4* wrow = reinterpret_cast<const uint4*>(P.Wr + (size_t)e * H);
-#pragma unroll 2
+    const uint4* w0 = reinterpret_cast<const uint4*>(P.Wr + (size_t)e0 * H);
+    const uint4* w1 = reinterpret_cast<const uint4*>(P.Wr + (size_t)(two ? e1 : e0) * H);
+#pragma unroll 4
     for (int c = tid; c < H / 8; c += kThreads) {
-        const uint4 wv = __ldg(wrow + c);
-        const uint32_t wr[4] = {wv.x, wv.y, wv.z, wv.w};
+        const uint4 a = __ldg(w0 + c), b = __ldg(w1 + c);
+        const uint32_t ar[4] = {a.x, a.y, a.z, a.w}, br[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             if (t0 + j < T) {
@@ -385,8 +422,11 @@ __device__ __forceinline__ void router_partial(const Params& P, int e, int t0, i
                 const uint32_t xr[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    acc[j] = fmaf(__uint_as_float(wr[q] << 16), __uint_as_float(xr[q] << 16), acc[j]);
-                    acc[j] = fmaf(__uint_as_float(wr[q] & 0xFFFF0000u), __uint_as_float(xr[q] & 0xFFFF0000u), acc[j]);
+                    const float xl = __uint_as_float(xr[q] << 16), xh = __uint_as_float(xr[q] & 0xFFFF0000u);
+                    acc0[j] = fmaf(__uint_as_float(ar[q] << 16), xl, acc0[j]);
+                    acc0[j] = fmaf(__uint_as_float(ar[q] & 0xFFFF0000u), xh, acc0[j]);
+                    acc1[j] = fmaf(__uint_as_float(br[q] << 16), xl, acc1[j]);
+                    acc1[j] = fmaf(__uint_as_float(br[q] & 0xFFFF0000u), xh, acc1[j]);
                 }
             }
         }
@@ -416,7 +456,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kTmemBufs);
     const uint32_t bar_drain = smem_u32(bars + 2 * kMaxStages + 2 * kTmemBufs);
-    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [3] give-up flag of the accumulator warps
+    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] routing published, [3] give-up flag of the accumulator warps
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
@@ -429,6 +469,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     wt.init(P.ctrl, P.timeout_ns);
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
     if (tid == 0) MOE_STAMP(0);
+    const unsigned par = tag & 1u;
+    unsigned* e_cnt = P.e_cnt + par * E;                    // counters of this launch
+    for (int e = cta * kThreads + tid; e < E; e += G * kThreads) P.e_cnt[(par ^ 1u) * E + e] = 0u;
+    if (cta == 0 && tid == 0) P.ctrl[kRouteCnt + (par ^ 1u)] = 0u;
 
     constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
@@ -468,8 +512,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 float acc0[8], acc1[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
-                router_partial(P, e0, t0, tid, acc0);
-                if (two) router_partial(P, e1, t0, tid, acc1);
+                router_partial(P, e0, e1, two, t0, tid, acc0, acc1);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
 #pragma unroll
@@ -493,38 +536,28 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (tid == 0) MOE_STAMP(2);
     // publish: generic writes of xq must be visible to the async proxy (TMA) of every CTA
     fence_proxy_async();
-    __threadfence();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
     if (tid == 0) {
         MOE_STAMP(3);
-        const unsigned old = atomicAdd(P.ctrl + kRouteCnt, 1u);
-        if (old == (unsigned)G - 1u) {
-            P.ctrl[kRouteCnt] = 0u;
-            __threadfence();
-            st_release(P.ctrl + kRouteReady, tag);
-        }
-        wt.flag(P.ctrl + kRouteReady, tag, 1);
-        __threadfence();
+        red_release_add(P.ctrl + kRouteCnt + par, 1u);      // all CTAs' logits and xq published once this reaches G
+        const bool ok = wt.flag(P.ctrl + kRouteCnt + par, (unsigned)G, 1);
+        misc[2] = ok ? 1u : 0u;
         MOE_STAMP(4);
     }
     __syncthreads();
-    bool alive = (*(volatile unsigned*)(P.ctrl + kAbort) == 0);
+    const bool alive = (misc[2] != 0u);
 
     // ------------------------------------------------------------------ top-k + routing metadata (every CTA)
     if (alive) {
-        const bool wg = (cta == 0);
-        for (int t = warp; t < T; t += kWarps) {
-            if (E <= 32) topk_token<1>(P, t, lane, s_ids, s_w, s_mask, wg);
-            else if (E <= 64) topk_token<2>(P, t, lane, s_ids, s_w, s_mask, wg);
-            else if (E <= 128) topk_token<4>(P, t, lane, s_ids, s_w, s_mask, wg);
-            else if (E <= 256) topk_token<8>(P, t, lane, s_ids, s_w, s_mask, wg);
-            else topk_token<16>(P, t, lane, s_ids, s_w, s_mask, wg);
-        }
         for (int i = tid; i < T * KBu; i += kThreads) s_xs[i] = __ldcg(P.xs + i);
-        __syncthreads();
+        // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
+        int chunk = (S * L.stage_bytes) / (4 * route_scratch_words(E, K));
+        chunk = chunk < kWarps ? chunk : kWarps;
+        for (int t0 = 0; t0 < T; t0 += chunk)
+            route_tokens(P, t0, min(chunk, T - t0), tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0);
         if (tid == 0) MOE_STAMP(6);
         if (warp == 0) {                                   // active-expert list in ascending expert order
             int base = 0;
@@ -553,6 +586,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             // k-step reuses the activation tile of its gate stage.  Weight tiles (cursor A) run ahead of
             // activation tiles (cursor B): only the latter wait for the up projection's intermediate tile.
             fence_proxy_async();                 // xq was written with ordinary stores by other CTAs
+            const uint64_t stream_once = l2_policy_evict_first();
             const int n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
             Walk aw, bw;
             int a_cur = 0, a_st = 0, b_cur = 0, b_st = 0;
@@ -572,12 +606,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (a_cur < n_up_st) {
                         const int half = a_cur & 1;
                         mbar_expect_tx(full, (uint32_t)kATileBytes + (half ? 0u : (uint32_t)(N * kBlock)));
-                        tma_load_2d(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full);
+                        tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
                         ++a_cur;
                         if (half) { if (a_cur == n_up_st) { if (a_cur < n_st) aw.init(dn_lo, KBd, HB, s_act); } else aw.next(s_act); }
                     } else {
                         mbar_expect_tx(full, (uint32_t)(kATileBytes + N * kBlock));
-                        tma_load_2d(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full);
+                        tma_load_2d_hint(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full, stream_once);
                         ++a_cur;
                         aw.next(s_act);
                     }
@@ -595,7 +629,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         }
                     } else {
                         if (bw.e != ready_e) {                   // intermediate tile published? (Section 3.2)
-                            if (ld_acquire(P.e_ready + bw.e) != tag) break;
+                            if (ld_acquire(e_cnt + bw.e) != (unsigned)IB) break;
                             fence_proxy_async();
                             ready_e = bw.e;
                         }
@@ -725,7 +759,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int pend = uend < hi ? uend : hi;
                 if (!up && e != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert)
-                    const bool got = (etid == 0) ? wt.flag(P.e_ready + e, tag, 8) : true;
+                    const bool got = (etid == 0) ? wt.flag(e_cnt + e, (unsigned)IB, 8) : true;
                     if (!epi_all(got)) { wt.dead = true; break; }
                     for (int i = etid; i < IB * N; i += kEpiThreads) s_hs[i] = __ldcg(P.hs + (size_t)e * IB * N + i);
                     hs_e = e;
@@ -788,7 +822,6 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             __stcg(dst + n * kBlock + row, accg[n]);
                             if (up) __stcg(dst + (N + n) * kBlock + row, accu[n]);
                         }
-                    __threadfence();
                     epi_bar();
                     if (etid == 0) st_release(pflag + cta, tag);
                     continue;
@@ -849,16 +882,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         }
                     }
                     fence_proxy_async();
-                    __threadfence();
                     epi_bar();
-                    if (etid == 0) {
-                        const unsigned old = atomicAdd(P.e_cnt + e, 1u);
-                        if (old == (unsigned)IB - 1u) {        // last I-block of this expert: publish the tile
-                            P.e_cnt[e] = 0u;
-                            __threadfence();
-                            st_release(P.e_ready + e, tag);
-                        }
-                    }
+                    if (etid == 0) red_release_add(e_cnt + e, 1u);   // the expert's tile is complete at count == I/128
                 } else {
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
@@ -869,7 +894,6 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             __stcg(P.y + ((size_t)n * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
-                    __threadfence();
                     epi_bar();
                     if (etid == 0) st_release(P.dn_done + e * HB + mb, tag);
                 }
