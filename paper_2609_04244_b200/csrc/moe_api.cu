@@ -72,6 +72,7 @@ struct moe_plan {
     float routed_scale;
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
+    int split_slack_kib = 100;
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
@@ -176,6 +177,7 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.T = T; P.H = p->H; P.E = p->E; P.I = p->I; P.K = p->K; P.scoring = p->scoring; P.renorm = p->renorm;
     P.routed_scale = p->routed_scale;
     P.stages = stages;
+    P.split_slack_kib = p->split_slack_kib;
     P.timeout_ns = p->timeout_ns;
     P.hidden = static_cast<const __nv_bfloat16*>(hidden);
     P.Wr = static_cast<const __nv_bfloat16*>(Wr);

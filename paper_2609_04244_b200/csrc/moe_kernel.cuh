@@ -54,6 +54,7 @@ struct Params {
     int T, H, E, I, K, scoring, renorm;
     float routed_scale;
     int stages;
+    int split_slack_kib;            // see range_quantum()
     unsigned long long timeout_ns;
     const __nv_bfloat16* hidden;
     const __nv_bfloat16* Wr;
@@ -279,7 +280,17 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
 }
 
 // per-phase split of a linear k-step list into contiguous per-CTA ranges
-__device__ __forceinline__ int range_lo(int S, int c, int G) { return (int)(((long long)S * c) / G); }
+// (q = 1: equal k-step counts, units may be split between neighbouring CTAs; q = K blocks per unit: whole units only)
+__device__ __forceinline__ int range_lo(int S, int c, int G, int q) { return (int)(((unsigned)(S / q) * (unsigned)c) / (unsigned)G) * q; }
+
+// Split a projection's units across CTAs (split-K, partial sums exchanged through L2) or keep units whole?
+// Whole units cost no exchange but load the busiest CTA with ceil(units/G) units; take them when that surplus,
+// in KiB of weight tiles, stays below `slack_kib` (what an exchange costs in streaming time).
+__device__ __forceinline__ int range_quantum(int units, int KB, int G, int kstep_kib, int slack_kib) {
+    const int whole = ((units + G - 1) / G) * KB * kstep_kib;
+    const int split = (int)(((long long)units * KB * kstep_kib + G - 1) / G);
+    return (whole - split <= slack_kib) ? KB : 1;
+}
 
 // position inside the linear k-step list of one projection: k-step -> (K block, row block, active expert)
 struct Walk {
@@ -575,8 +586,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int U = alive ? (int)misc[1] : 0;
     if (tid == 0) MOE_STAMP(7);
     const int S_up = U * IB * KBu, S_dn = U * HB * KBd;     // k-steps of the two projections (host checks the range)
-    const int up_lo = range_lo(S_up, cta, G), up_hi = range_lo(S_up, cta + 1, G);
-    const int dn_lo = range_lo(S_dn, cta, G), dn_hi = range_lo(S_dn, cta + 1, G);
+    const int q_up = range_quantum(U * IB, KBu, G, 32, P.split_slack_kib), q_dn = range_quantum(U * HB, KBd, G, 16, P.split_slack_kib);
+    const int up_lo = range_lo(S_up, cta, G, q_up), up_hi = range_lo(S_up, cta + 1, G, q_up);
+    const int dn_lo = range_lo(S_dn, cta, G, q_dn), dn_hi = range_lo(S_dn, cta + 1, G, q_dn);
 
     // ------------------------------------------------------------------ role: TMA producer
     if (warp == 0) {
@@ -725,7 +737,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const bool up = (phase == 0);
             const int lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
             const int KB = up ? KBu : KBd, MB = up ? IB : HB;  // K blocks per unit, row blocks per expert
-            const int S_all = up ? S_up : S_dn;
+            const int S_all = up ? S_up : S_dn, q_all = up ? q_up : q_dn;
             float* part = up ? P.part_up : P.part_dn;
             unsigned* pflag = up ? P.pu_flag : P.pd_flag;
             const int pcols = up ? 2 * N : N;
@@ -834,15 +846,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     for (int base = cta + 1; base < G; base += kEpiThreads) {
                         const int c = base + etid;
                         if (c < G) {
-                            const int clo = range_lo(S_all, c, G), chi = range_lo(S_all, c + 1, G);
+                            const int clo = range_lo(S_all, c, G, q_all), chi = range_lo(S_all, c + 1, G, q_all);
                             if (clo < uend && chi > clo) got = wt.flag(pflag + c, tag, 6) && got;
                         }
-                        if (range_lo(S_all, min(base + kEpiThreads, G), G) >= uend) break;
+                        if (range_lo(S_all, min(base + kEpiThreads, G), G, q_all) >= uend) break;
                     }
-                    while (c_end < G && range_lo(S_all, c_end, G) < uend) ++c_end;
+                    while (c_end < G && range_lo(S_all, c_end, G, q_all) < uend) ++c_end;
                     if (!epi_all(got)) { wt.dead = true; break; }
                     for (int c = cta + 1; c < c_end; ++c) {
-                        if (range_lo(S_all, c + 1, G) == range_lo(S_all, c, G)) continue;
+                        if (range_lo(S_all, c + 1, G, q_all) == range_lo(S_all, c, G, q_all)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TC; ++n)
