@@ -100,6 +100,30 @@ int moe_forward(moe_plan_t plan, int T,
                 void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream);
 
 /*
+ * moe_forward_noalloc: moe_forward for callers that cannot give the library device memory.  (The paper has no
+ * counterpart: this entry point exists only for integration.)  Some hosts of this library may not call cudaMalloc
+ * at the point where they run a decode step -- for instance code running inside a memory pool that owns the whole
+ * device, or a runtime whose allocator is not reentrant from the thread that launches kernels -- and so they have
+ * no scratch buffer to hand over.  Here the scratch is a fixed array of MOE_NOALLOC_SCRATCH_BYTES (24 MiB) that is
+ * part of the library's device image: every GPU that loads the library holds these 24 MiB until the process exits.
+ *   - Same tensor arguments as moe_forward; there is no workspace argument.  1 <= T <= 64.
+ *   - A layer shape whose scratch for T tokens exceeds the array is rejected with MOE_ERR_WORKSPACE and a message
+ *     giving both sizes (the five benchmark shapes fit for T <= 16).
+ *   - The plan's device must be the current device.  The FIRST call on a device looks up the array's device
+ *     address (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *   - The call itself allocates nothing: no cudaMalloc/cudaFree, no descriptor cache; TMA descriptors are built on
+ *     the stack.  It enqueues one small memset (control words and flags, which must start from zero because the
+ *     array keeps the previous call's contents) and the kernel, both on `stream`.
+ *   - All calls on a device share the one array: calls that overlap on the GPU (different streams without an
+ *     ordering between them, or different host threads) race.  Order them.
+ */
+int moe_forward_noalloc(moe_plan_t plan, int T,
+                        const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                        const void* W13_fp8, const float* W13_scale,
+                        const void* W2_fp8, const float* W2_scale,
+                        void* out_bf16, moe_stream_t stream);
+
+/*
  * moe_forward_debug: moe_forward, then copies (device to device, on `stream`) the routing and input
  * quantisation results of the step into caller buffers; any of them may be NULL.  Requires T <= 64.
  *   topk_ids [T,top_k] int32 (slot order: key descending, index ascending)   topk_w [T,top_k] fp32

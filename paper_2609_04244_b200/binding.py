@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_noalloc", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -54,6 +54,8 @@ def load_library():
     lib.moe_workspace_init.argtypes = [vp, vp, sz, vp]
     lib.moe_forward.restype = i
     lib.moe_forward.argtypes = [vp, i] + [vp] * 9 + [sz, vp]
+    lib.moe_forward_noalloc.restype = i
+    lib.moe_forward_noalloc.argtypes = [vp, i] + [vp] * 8 + [vp]
     lib.moe_forward_debug.restype = i
     lib.moe_forward_debug.argtypes = [vp, i] + [vp] * 9 + [sz, vp] + [vp] * 5
     lib.moe_sync_status.restype = i
@@ -112,6 +114,16 @@ def moe_forward(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, worksp
     _check(load_library().moe_forward(plan, T, _p(hidden), _p(Wr), _p(sel_bias), _p(W13q), _p(W13s), _p(W2q), _p(W2s),
                                       _p(out), _p(workspace), workspace.numel() * workspace.element_size(),
                                       _stream(stream)))
+
+
+def moe_forward_noalloc(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, stream=None) -> None:
+    """One decode step using the library's built-in scratch array instead of a caller workspace.
+
+    For callers that cannot allocate device memory where they run the step; see include/moe_b200.h for the size
+    limit, the first-call set-up and the rule that calls sharing a device must not overlap.
+    """
+    _check(load_library().moe_forward_noalloc(plan, T, _p(hidden), _p(Wr), _p(sel_bias), _p(W13q), _p(W13s), _p(W2q),
+                                              _p(W2s), _p(out), _stream(stream)))
 
 
 def moe_forward_debug(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, workspace, stream=None,

@@ -313,6 +313,99 @@ int moe_forward(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_
     return MOE_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Entry point for callers that must not allocate: the scratch lives in a fixed array in the device image.
+// ---------------------------------------------------------------------------------------------------------------
+#define MOE_NOALLOC_SCRATCH_BYTES (24u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MOE_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[64] = {nullptr};   // device address of g_noalloc_scratch, per device ordinal
+}  // namespace
+
+int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
+                        const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
+                        void* out_bf16, moe_stream_t stream) {
+    if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (T < 1 || T > moe::kMaxTokens)
+        return fail(MOE_ERR_ARG, "moe_forward_noalloc handles 1..%d tokens per call (got %d)", moe::kMaxTokens, T);
+    const WsLayout L = plan->layout(T);
+    if (L.total > MOE_NOALLOC_SCRATCH_BYTES)
+        return fail(MOE_ERR_WORKSPACE, "this shape with T=%d needs %zu bytes of scratch; the built-in array holds %u",
+                    T, L.total, (unsigned)MOE_NOALLOC_SCRATCH_BYTES);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != plan->device || dev < 0 || dev >= 64)
+        return fail(MOE_ERR_ARG, "the plan's device must be the current device");
+    void* ws = nullptr;
+    {
+        // First call on this device: resolve the array's device address.  In host code the array's name is only a
+        // handle, so the address has to come from the runtime, with the owning device current.
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        if (!g_noalloc_ptr[dev]) {
+            void* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+            if (e != cudaSuccess || !ptr)
+                return fail(MOE_ERR_CUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            g_noalloc_ptr[dev] = ptr;
+        }
+        ws = g_noalloc_ptr[dev];
+    }
+    int rc = check_forward_args(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, ws);
+    if (rc != MOE_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the previous call left: start every call from cleared control words and flags.
+    if (cudaMemsetAsync(ws, 0, L.flags_end, s) != cudaSuccess)
+        return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
+
+    const int N = plan->n_hw(T);
+    const int stages = plan->stages_for(N, T);
+    if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
+    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages);
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    CUtensorMap m13, m2, mx, mh;       // encoded on the stack: no descriptor cache, nothing allocated
+    if (!encode_2d(&m13, W13_fp8, (uint64_t)plan->E * 2 * plan->I, plan->H, 128) ||
+        !encode_2d(&m2, W2_fp8, (uint64_t)plan->E * plan->H, plan->I, 128) ||
+        !encode_2d(&mx, w + L.xq, moe::kMaxTokens, plan->H, N) ||
+        !encode_2d(&mh, w + L.hq, (uint64_t)plan->E * N, plan->I, N))
+        return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    moe::Params P;
+    P.T = T; P.H = plan->H; P.E = plan->E; P.I = plan->I; P.K = plan->K; P.scoring = plan->scoring; P.renorm = plan->renorm;
+    P.routed_scale = plan->routed_scale;
+    P.stages = stages;
+    P.split_slack_kib = plan->split_slack_kib;
+    P.timeout_ns = plan->timeout_ns;
+    P.hidden = static_cast<const __nv_bfloat16*>(hidden_bf16);
+    P.Wr = static_cast<const __nv_bfloat16*>(Wr_bf16);
+    P.bias = (plan->scoring == MOE_SCORE_SIGMOID_BIAS) ? sel_bias : nullptr;
+    P.W13s = W13_scale; P.W2s = W2_scale;
+    P.out = static_cast<__nv_bfloat16*>(out_bf16);
+    P.ctrl = reinterpret_cast<unsigned*>(w + L.ctrl);
+    P.logits = reinterpret_cast<float*>(w + L.logits);
+    P.ids = reinterpret_cast<int*>(w + L.ids);
+    P.wts = reinterpret_cast<float*>(w + L.wts);
+    P.xq = w + L.xq;
+    P.xs = reinterpret_cast<float*>(w + L.xs);
+    P.hq = w + L.hq;
+    P.hs = reinterpret_cast<float*>(w + L.hs);
+    P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
+    P.dn_done = reinterpret_cast<unsigned*>(w + L.dn_done);
+    P.part_up = reinterpret_cast<float*>(w + L.part_up);
+    P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
+    P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
+    P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
+    P.y = reinterpret_cast<float*>(w + L.y);
+    P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
+    const int smem_bytes = SL.total + 1024;
+    if (T == 1) return launch<16, 1>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    if (T == 2) return launch<16, 2>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    if (T <= 4) return launch<16, 4>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    if (T <= 8) return launch<16, 8>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    if (T <= 16) return launch<16, 16>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    if (T <= 32) return launch<32, 32>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    return launch<64, 64>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+}
+
 int moe_forward_debug(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,
                       const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
                       void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream,
