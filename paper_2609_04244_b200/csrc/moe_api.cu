@@ -3,6 +3,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -73,6 +74,7 @@ struct moe_plan {
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
     int split_slack_kib = 100;
+    int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
@@ -105,7 +107,7 @@ struct moe_plan {
     }
 
     int stages_for(int N, int T) const {
-        for (int s = moe::kMaxStages; s >= 2; --s) {
+        for (int s = (stages_cap > 0 && stages_cap < moe::kMaxStages) ? stages_cap : moe::kMaxStages; s >= 2; --s) {
             const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s);
             if (L.total + 1024 <= smem_optin) return s;
         }
@@ -260,6 +262,9 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     p->sms = prop.multiProcessorCount;
     p->smem_optin = (int)prop.sharedMemPerBlockOptin;
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
+    // schedule overrides for experiments (the paper tunes its schedule offline, Section 3.4)
+    if (const char* v = getenv("MOE_B200_STAGES")) p->stages_cap = atoi(v);
+    if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) p->split_slack_kib = atoi(v);
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }

@@ -14,8 +14,8 @@
 //   reduce  : (token, 128-row block) tasks spread over all CTAs sum the per-slot
 //             results in slot order (deterministic, no float atomics)
 //
-// Warp roles (Section 3.3, warp specialisation): warp 0 = TMA producer, warp 1 =
-// tcgen05 MMA issuer, warps 4..7 = accumulator/epilogue warps (one TMEM lane
+// Warp roles (Section 3.3, warp specialisation): warps 0 and 2 = TMA producers (weight tiles,
+// activation tiles), warps 1 and 3 = tcgen05 MMA issuers (even and odd k-steps), warps 4..7 = accumulator/epilogue warps (one TMEM lane
 // quadrant each); all eight warps share phase R.  Weights are the MMA "A"
 // operand (M = 128 weight rows), the whole token tile is the "B" operand with
 // N = 16/32/64 (Eq. 9), K = 32 per instruction, four instructions per 128-wide
@@ -265,7 +265,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
     int o = stages * L.stage_bytes;
-    L.bar_off = o;  o += (2 * kMaxStages + 16) * 8;
+    L.bar_off = o;  o += (3 * kMaxStages + 16) * 8;
     L.misc_off = o; o += 64;
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
@@ -467,6 +467,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kTmemBufs);
     const uint32_t bar_drain = smem_u32(bars + 2 * kMaxStages + 2 * kTmemBufs);
+    const uint32_t bar_fullb = smem_u32(bars + 2 * kMaxStages + 16);   // activation tile landed (second producer)
     uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] routing published, [3] give-up flag of the accumulator warps
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
@@ -488,9 +489,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
-        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
         mbar_init(bar_drain, 1);
+        mbar_init(bar_drain + 16, 1);
         misc[3] = 0u;
         fence_barrier_init();
     }
@@ -590,106 +592,121 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int up_lo = range_lo(S_up, cta, G, q_up), up_hi = range_lo(S_up, cta + 1, G, q_up);
     const int dn_lo = range_lo(S_dn, cta, G, q_dn), dn_hi = range_lo(S_dn, cta + 1, G, q_dn);
 
-    // ------------------------------------------------------------------ role: TMA producer
+    // ------------------------------------------------------------------ role: TMA producers
+    // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.  A stage = one
+    // 128x128 weight tile (warp 0) + one Nx128 activation tile (warp 2), each on its own mbarrier; the up tile of a
+    // k-step reuses the activation tile of its gate stage.  Two issuing threads because one thread cannot issue
+    // two bulk-tensor copies per 16 KiB fast enough to saturate HBM3e; and because only the activation tiles of the
+    // down projection wait for the up projection's intermediate tile, the weight stream never stalls on it
+    // (Section 3.3: lookahead across the projection boundary).
     if (warp == 0) {
         if (lane == 0 && alive) {
-            // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.
-            // A stage = one 128x128 weight tile + one Nx128 activation tile on one mbarrier; the up tile of a
-            // k-step reuses the activation tile of its gate stage.  Weight tiles (cursor A) run ahead of
-            // activation tiles (cursor B): only the latter wait for the up projection's intermediate tile.
-            fence_proxy_async();                 // xq was written with ordinary stores by other CTAs
             const uint64_t stream_once = l2_policy_evict_first();
             const int n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
-            Walk aw, bw;
-            int a_cur = 0, a_st = 0, b_cur = 0, b_st = 0;
+            Walk aw;
+            int a_cur = 0, a_st = 0;
             uint32_t a_ph = 1u;                  // parity to wait for on the empty barrier
-            if (n_up_st > 0) { aw.init(up_lo, KBu, IB, s_act); bw = aw; }
-            else if (n_st > 0) { aw.init(dn_lo, KBd, HB, s_act); bw = aw; }
-            int ready_e = -1;                    // expert whose intermediate tile is known to be published
-            uint32_t idle = 0;
+            uint32_t dst = smem_u32(smem), full = bar_full, empty = bar_empty;
+            if (n_up_st > 0) aw.init(up_lo, KBu, IB, s_act);
+            else if (n_st > 0) aw.init(dn_lo, KBd, HB, s_act);
             bool stamped = false;
             MOE_STAMP(8);
-            while (b_cur < n_st && !wt.dead) {
-                bool progress = false;
-                while (a_cur < n_st && a_cur - b_cur < S) {
-                    if (!mbar_try_wait(bar_empty + 8 * a_st, a_ph)) break;
-                    const uint32_t dst = smem_u32(smem + (size_t)a_st * L.stage_bytes);
-                    const uint32_t full = bar_full + 8 * a_st;
-                    if (a_cur < n_up_st) {
-                        const int half = a_cur & 1;
-                        mbar_expect_tx(full, (uint32_t)kATileBytes + (half ? 0u : (uint32_t)(N * kBlock)));
-                        tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
-                        ++a_cur;
-                        if (half) { if (a_cur == n_up_st) { if (a_cur < n_st) aw.init(dn_lo, KBd, HB, s_act); } else aw.next(s_act); }
-                    } else {
-                        mbar_expect_tx(full, (uint32_t)(kATileBytes + N * kBlock));
-                        tma_load_2d_hint(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full, stream_once);
-                        ++a_cur;
-                        aw.next(s_act);
-                    }
-                    if (++a_st == S) { a_st = 0; a_ph ^= 1u; }
-                    progress = true;
-                }
-                while (b_cur < a_cur) {
-                    const uint32_t dst = smem_u32(smem + (size_t)b_st * L.stage_bytes + kATileBytes);
-                    const uint32_t full = bar_full + 8 * b_st;
-                    if (b_cur < n_up_st) {
-                        if ((b_cur & 1) == 0) {
-                            tma_load_2d(dst, &tmXq, bw.kb * kBlock, 0, full);
-                        } else {
-                            if (b_cur + 1 == n_up_st) { if (b_cur + 1 < n_st) bw.init(dn_lo, KBd, HB, s_act); } else bw.next(s_act);
-                        }
-                    } else {
-                        if (bw.e != ready_e) {                   // intermediate tile published? (Section 3.2)
-                            if (ld_acquire(e_cnt + bw.e) != (unsigned)IB) break;
-                            fence_proxy_async();
-                            ready_e = bw.e;
-                        }
-                        tma_load_2d(dst, &tmHq, bw.kb * kBlock, bw.e * N, full);
-                        bw.next(s_act);
-                    }
-                    ++b_cur;
-                    if (++b_st == S) b_st = 0;
-                    progress = true;
-                }
-                if (!stamped) { MOE_STAMP(9); stamped = true; }
-                if (progress) idle = 0;
-                else if ((++idle & 63u) == 0) { if (wt.expired(2)) break; __nanosleep(40); }
+            for (; a_cur < n_up_st; ++a_cur) {                       // gate/up weight tiles
+                if (!wt.mbar(empty, a_ph, 2)) break;
+                const int half = a_cur & 1;
+                mbar_expect_tx(full, (uint32_t)kATileBytes);
+                tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
+                if (half) aw.next(s_act);
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; if (!stamped) { MOE_STAMP(9); stamped = true; } }
             }
-            if (wt.dead) {
-                // give-up path: complete the byte count of half-armed stages, then wait for copies in flight
-                for (int it = b_cur; it < a_cur; ++it) {
-                    if (it < n_up_st && (it & 1)) continue;
-                    const int st = it % S;
-                    tma_load_2d(smem_u32(smem + (size_t)st * L.stage_bytes + kATileBytes), &tmXq, 0, 0, bar_full + 8 * st);
-                }
-                for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it) {
-                    const int st = it % S;
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * st, (uint32_t)((it / S) & 1)); ++i) {}
-                }
+            if (!wt.dead && n_st > n_up_st) aw.init(dn_lo, KBd, HB, s_act);
+            for (; a_cur < n_st && !wt.dead; ++a_cur) {              // down weight tiles
+                if (!wt.mbar(empty, a_ph, 2)) break;
+                mbar_expect_tx(full, (uint32_t)kATileBytes);
+                tma_load_2d_hint(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full, stream_once);
+                aw.next(s_act);
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; }
+            }
+            if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight
+                for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it)
+                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
             }
         }
         __syncwarp();
     }
-    // ------------------------------------------------------------------ role: MMA issuer
-    else if (warp == 1) {
+    else if (warp == 2) {
+        if (lane == 0 && alive) {
+            fence_proxy_async();                 // xq was written with ordinary stores by other CTAs
+            const int n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
+            Walk bw;
+            int b_cur = 0, b_st = 0;
+            uint32_t b_ph = 1u;
+            uint32_t dst = smem_u32(smem) + kATileBytes, full = bar_fullb, empty = bar_empty;
+            if (n_up_st > 0) bw.init(up_lo, KBu, IB, s_act);
+            else if (n_st > 0) bw.init(dn_lo, KBd, HB, s_act);
+            for (; b_cur < n_up_st; ++b_cur) {                       // input activation tiles (gate stages only)
+                if (!wt.mbar(empty, b_ph, 10)) break;
+                if ((b_cur & 1) == 0) {
+                    mbar_expect_tx(full, (uint32_t)(N * kBlock));
+                    tma_load_2d(dst, &tmXq, bw.kb * kBlock, 0, full);
+                } else {
+                    mbar_arrive(full);
+                    bw.next(s_act);
+                }
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
+            }
+            if (!wt.dead && n_st > n_up_st) bw.init(dn_lo, KBd, HB, s_act);
+            int ready_e = -1;                    // expert whose intermediate tile is known to be published
+            for (; b_cur < n_st && !wt.dead; ++b_cur) {              // intermediate activation tiles
+                if (!wt.mbar(empty, b_ph, 10)) break;
+                if (bw.e != ready_e) {                               // published? (Section 3.2, readiness hand-off)
+                    if (!wt.flag(e_cnt + bw.e, (unsigned)IB, 11)) break;
+                    fence_proxy_async();
+                    ready_e = bw.e;
+                }
+                mbar_expect_tx(full, (uint32_t)(N * kBlock));
+                tma_load_2d(dst, &tmHq, bw.kb * kBlock, bw.e * N, full);
+                bw.next(s_act);
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
+            }
+            if (wt.dead) {
+                for (int it = (b_cur > S ? b_cur - S : 0); it < b_cur; ++it)
+                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_fullb + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
+            }
+        }
+        __syncwarp();
+    }
+    // ------------------------------------------------------------------ role: MMA issuers
+    // Two issuing threads (warp 1: even k-steps, warp 3: odd k-steps), each with its own TMEM buffers (k-step mod 4)
+    // and its own commits: issuing four tcgen05.mma per 16 KiB tile from one thread alone costs more time than the
+    // tile takes to arrive from HBM.
+    else if (warp == 1 || warp == 3) {
         if (lane == 0 && alive) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
             const uint32_t ring = smem_u32(smem);
-            int st = 0, buf = 0;
-            uint32_t ph = 0, tph = 1u;           // full-barrier parity; tmem-empty parity
-            bool first = true;
+            const int who = warp >> 1;           // 0 or 1
             const int n_up = up_hi - up_lo, n_dn = dn_hi - dn_lo;
-            for (int s = 0; s < n_up + n_dn && !wt.dead; ++s) {
-                const bool up = s < n_up;
+            int st = 0;
+            uint32_t ph = 0;                     // full-barrier parity of stage `st`
+            auto advance = [&](int n) { st += n; while (st >= S) { st -= S; ph ^= 1u; } };
+            bool first = true;
+            if (who == 1) advance(n_up > 0 ? 2 : 1);               // skip k-step 0
+            for (int ks = who; ks < n_up + n_dn && !wt.dead; ks += 2) {
+                const bool up = ks < n_up;
+                const int buf = ks & (kTmemBufs - 1);
+                const uint32_t tph = (uint32_t)((ks >> 2) & 1) ^ 1u;
                 if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
                 const int st0 = st;
+                const uint32_t ph0 = ph;
                 const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)L.stage_bytes;
-                if (!wt.mbar(bar_full + 8 * st0, ph, 4)) break;
-                if (++st == S) { st = 0; ph ^= 1u; }
+                if (!wt.mbar(bar_full + 8 * st0, ph0, 4) || !wt.mbar(bar_fullb + 8 * st0, ph0, 4)) break;
                 const uint64_t b_desc = make_smem_desc(a0 + kATileBytes);
                 const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
-                if (first) { MOE_STAMP(10); first = false; }
+                if (first && who == 0) { MOE_STAMP(10); first = false; }
                 tc_fence_after();
                 {
                     const uint64_t a_desc = make_smem_desc(a0);
@@ -698,9 +715,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         umma_f8(d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, k > 0 ? 1u : 0u);
                 }
                 if (up) {                                      // up tile of the same K block, same activation tile
+                    advance(1);
                     const int st1 = st;
-                    if (!wt.mbar(bar_full + 8 * st1, ph, 4)) break;
-                    if (++st == S) { st = 0; ph ^= 1u; }
+                    if (!wt.mbar(bar_full + 8 * st1, ph, 4) || !wt.mbar(bar_fullb + 8 * st1, ph, 4)) break;
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc(ring + (uint32_t)st1 * (uint32_t)L.stage_bytes);
 #pragma unroll
@@ -712,11 +729,13 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     umma_commit(bar_empty + 8 * st0);
                 }
                 umma_commit(bar_tfull + 8 * buf);              // accumulator of this K block complete
-                if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
+                // move past the rest of this k-step and the other issuer's k-step
+                advance(1);
+                if (ks + 1 < n_up + n_dn) advance(ks + 1 < n_up ? 2 : 1);
             }
             if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
-                umma_commit(bar_drain);
-                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain, 0); ++i) {}
+                umma_commit(bar_drain + 8 * (uint32_t)who * 2);
+                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain + 8 * (uint32_t)who * 2, 0); ++i) {}
             }
         }
         __syncwarp();
