@@ -41,7 +41,7 @@ constexpr int kATileBytes = kBlock * kBlock;  // 16 KiB of FP8
 constexpr int kMaxTopK = 32;
 constexpr int kMaxExperts = 512;
 constexpr int kMaxTokens = 64;
-constexpr int kTmemBufs = 4;         // accumulator buffers in TMEM (one K block each)
+constexpr int kMaxTmemBufs = 8;      // accumulator buffers in TMEM (one K block each): 8 for N=16, 4 for N=32/64
 constexpr int kStampsPerCta = 16;
 
 // control words at the head of the workspace
@@ -265,7 +265,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
     int o = stages * L.stage_bytes;
-    L.bar_off = o;  o += (3 * kMaxStages + 16) * 8;
+    L.bar_off = o;  o += (3 * kMaxStages + 2 * kMaxTmemBufs + 8) * 8;
     L.misc_off = o; o += 64;
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
@@ -465,9 +465,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
-    const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kTmemBufs);
-    const uint32_t bar_drain = smem_u32(bars + 2 * kMaxStages + 2 * kTmemBufs);
-    const uint32_t bar_fullb = smem_u32(bars + 2 * kMaxStages + 16);   // activation tile landed (second producer)
+    constexpr int kTmemBufs = (N == 16) ? 8 : 4;                 // 8 x 32 = 256, 4 x 64 = 256, 4 x 128 = 512 columns
+    constexpr int kBufShift = (N == 16) ? 3 : 2;
+    const uint32_t bar_fullb = smem_u32(bars + 2 * kMaxStages);  // activation tile landed (second producer)
+    const uint32_t bar_tfull = smem_u32(bars + 3 * kMaxStages), bar_tempty = smem_u32(bars + 3 * kMaxStages + kMaxTmemBufs);
+    const uint32_t bar_drain = smem_u32(bars + 3 * kMaxStages + 2 * kMaxTmemBufs);
     uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] routing published, [3] give-up flag of the accumulator warps
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
@@ -698,7 +700,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             for (int ks = who; ks < n_up + n_dn && !wt.dead; ks += 2) {
                 const bool up = ks < n_up;
                 const int buf = ks & (kTmemBufs - 1);
-                const uint32_t tph = (uint32_t)((ks >> 2) & 1) ^ 1u;
+                const uint32_t tph = (uint32_t)((ks >> kBufShift) & 1) ^ 1u;
                 if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
                 const int st0 = st;
                 const uint32_t ph0 = ph;
