@@ -272,8 +272,9 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
     L.act_off = o;  o += (E + 1) * 4;
-    L.xs_off = o;   o += T * (H / kBlock) * 4;      // input activation scales [T][H/128]
-    L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]
+    o = (o + 15) & ~15;
+    L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;   // input activation scales [H/128][T rounded up to 4]
+    L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
     L.red_off = o;  o += kWarps * 64 * 4;           // cross-warp reduction scratch
     L.total = o;
     return L;
@@ -462,6 +463,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock, KBd = IB;
     const int S = P.stages;
     const SmemLayout L = smem_layout(N, T, K, E, H, I, S);
+    const int TS = (T + 3) & ~3;                              // token stride of the transposed input scales
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
@@ -567,7 +569,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     // ------------------------------------------------------------------ top-k + routing metadata (every CTA)
     if (alive) {
-        for (int i = tid; i < T * KBu; i += kThreads) s_xs[i] = __ldcg(P.xs + i);
+        for (int i = tid; i < T * KBu; i += kThreads) s_xs[(i % KBu) * TS + i / KBu] = __ldcg(P.xs + i);   // transposed: [K block][token]
         // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
         int chunk = (S * L.stage_bytes) / (4 * route_scratch_words(E, K));
         chunk = chunk < kWarps ? chunk : kWarps;
@@ -798,8 +800,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     hs_e = e;
                     epi_bar();
                 }
-                const float* as_p = up ? (s_xs + kb0) : (s_hs + kb0 * N);
-                const int as_tok = up ? KBu : 1, as_step = up ? 1 : N;
+                const float* as_p = up ? (s_xs + kb0 * TS) : (s_hs + kb0 * N);   // activation scales [K block][token]
+                const int as_step = up ? TS : N;
 #pragma unroll
                 for (int n = 0; n < TC; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
@@ -828,12 +830,22 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             __syncwarp();
                             if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
                         }
+                        float as[CH];
+                        if constexpr (CH >= 4) {
+#pragma unroll
+                            for (int jj = 0; jj < CH; jj += 4) {
+                                const float4 v = *reinterpret_cast<const float4*>(as_p + i * as_step + c + jj);
+                                as[jj] = v.x; as[jj + 1] = v.y; as[jj + 2] = v.z; as[jj + 3] = v.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < CH; ++jj) as[jj] = as_p[i * as_step + c + jj];
+                        }
 #pragma unroll
                         for (int jj = 0; jj < CH; ++jj) {
                             const int n = c + jj;
-                            const float as = as_p[n * as_tok + i * as_step];
-                            accg[n] = fmaf(dg[jj], wsg * as, accg[n]);
-                            if (up) accu[n] = fmaf(du[jj], wsu * as, accu[n]);
+                            accg[n] = fmaf(dg[jj], wsg * as[jj], accg[n]);
+                            if (up) accu[n] = fmaf(du[jj], wsu * as[jj], accu[n]);
                         }
                     }
                     if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
@@ -851,7 +863,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
                     for (int n = 0; n < TC; ++n)
-                        if (n < T) {
+                        if ((mask >> n) & 1ull) {                        // only tokens routed to this expert matter
                             __stcg(dst + n * kBlock + row, accg[n]);
                             if (up) __stcg(dst + (N + n) * kBlock + row, accu[n]);
                         }
@@ -879,7 +891,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TC; ++n)
-                            if (n < T) {
+                            if ((mask >> n) & 1ull) {
                                 accg[n] += __ldcg(src + n * kBlock + row);
                                 if (up) accu[n] += __ldcg(src + (N + n) * kBlock + row);
                             }
@@ -889,13 +901,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
                     for (int n = 0; n < TC; ++n) {
-                        float a = 0.f;
-                        if (n < T && ((mask >> n) & 1ull)) {
+                        if ((mask >> n) & 1ull) {                        // warp-uniform: other tokens cost nothing
                             const float g = accg[n];
-                            a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
-                        }
-                        accg[n] = a;
-                        if (n < T) {
+                            const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
+                            accg[n] = a;
                             float m = fabsf(a);
 #pragma unroll
                             for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -905,7 +914,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     epi_bar();
 #pragma unroll
                     for (int n = 0; n < TC; ++n) {
-                        if (n < T && ((mask >> n) & 1ull)) {
+                        if ((mask >> n) & 1ull) {
                             const float amax = fmaxf(fmaxf(s_red[n], s_red[N + n]), fmaxf(s_red[2 * N + n], s_red[3 * N + n]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
                             const float2 v = make_float2(__fdiv_rn(accg[n], sc), 0.f);
@@ -921,7 +930,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
                     for (int n = 0; n < TC; ++n) {
-                        if (n < T && ((mask >> n) & 1ull)) {
+                        if ((mask >> n) & 1ull) {
                             int sl = 0;
                             for (int jj = 0; jj < K; ++jj) if (s_ids[n * K + jj] == e) sl = jj;
                             __stcg(P.y + ((size_t)n * K + sl) * H + mb * kBlock + row, accg[n]);
