@@ -75,6 +75,7 @@ struct moe_plan {
     unsigned long long timeout_ns;
     int split_slack_kib = 100;
     int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
+    int use_pdl = 1;                // programmatic dependent launch
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
@@ -141,8 +142,18 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
             return fail(MOE_ERR_CUDA, "cudaFuncSetAttribute(max dynamic smem) failed: %s", cudaGetErrorString(cudaGetLastError()));
         configured_device = p->device;
     }
-    moe::moe_decode_kernel<N, TC><<<p->sms, moe::kThreads, smem_bytes, stream>>>(m13, m2, mx, mh, P);
-    cudaError_t err = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p->sms, 1, 1);
+    cfg.blockDim = dim3(moe::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap our launch latency with the previous
+    attr[0].val.programmaticStreamSerializationAllowed = 1;            // kernel's tail; the kernel itself waits for it
+    cfg.attrs = attr;
+    cfg.numAttrs = p->use_pdl ? 1 : 0;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_decode_kernel<N, TC>, m13, m2, mx, mh, P);
+    if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
     return MOE_OK;
 }
@@ -264,6 +275,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
     // schedule overrides for experiments (the paper tunes its schedule offline, Section 3.4)
     if (const char* v = getenv("MOE_B200_STAGES")) p->stages_cap = atoi(v);
+    if (const char* v = getenv("MOE_B200_PDL")) p->use_pdl = atoi(v) != 0;
     if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) p->split_slack_kib = atoi(v);
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);

@@ -481,6 +481,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
 
+    // Programmatic dependent launch: let the next launch in the stream start placing its CTAs as ours retire, and
+    // do not touch any global memory before the previous launch has completed and flushed (both are no-ops when the
+    // launch was not made with the programmatic-serialization attribute).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     Waiter wt;
     wt.init(P.ctrl, P.timeout_ns);
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
