@@ -144,7 +144,7 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p->sms, 1, 1);
-    cfg.blockDim = dim3(moe::kThreads, 1, 1);
+    cfg.blockDim = dim3(128 + 128 * (TC >= 32 ? 2 : 1), 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -162,7 +162,7 @@ template <int N, int TC>
 bool resident(int smem_optin, int smem_bytes) {
     int blocks = 0;
     if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return false;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, moe::moe_decode_kernel<N, TC>, moe::kThreads, smem_bytes) != cudaSuccess) return false;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, moe::moe_decode_kernel<N, TC>, 128 + 128 * (TC >= 32 ? 2 : 1), smem_bytes) != cudaSuccess) return false;
     return blocks >= 1;
 }
 

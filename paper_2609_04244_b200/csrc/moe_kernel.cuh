@@ -32,10 +32,10 @@
 namespace moe {
 
 constexpr int kBlock = 128;          // weight block edge = activation group = MMA M = K block
-constexpr int kThreads = 256;
-constexpr int kWarps = 8;
+constexpr int kRoleWarps = 4;         // warps 0..3: two TMA producers, two MMA issuers
+constexpr int kMaxWarps = 12;
 constexpr int kEpiWarp0 = 4;         // warps 4..7
-constexpr int kEpiThreads = 128;
+constexpr int kEpiGroupThreads = 128; // one accumulator group = 4 warps = the 4 TMEM lane quadrants
 constexpr int kMaxStages = 16;
 constexpr int kATileBytes = kBlock * kBlock;  // 16 KiB of FP8
 constexpr int kMaxTopK = 32;
@@ -199,16 +199,16 @@ __device__ __forceinline__ unsigned long long gtime() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// barrier over the 128 epilogue threads that also ANDs a predicate, so that give-up decisions are uniform
-__device__ __forceinline__ bool epi_all(bool ok) {
+__device__ __forceinline__ void epi_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
+// barrier over the accumulator threads that also ANDs a predicate, so that give-up decisions are uniform
+__device__ __forceinline__ bool epi_all(bool ok, int nthreads) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)ok) : "memory");
+        : "=r"(r) : "r"((uint32_t)ok), "r"(nthreads) : "memory");
     return r != 0;
 }
 
@@ -275,7 +275,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     o = (o + 15) & ~15;
     L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;   // input activation scales [H/128][T rounded up to 4]
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
-    L.red_off = o;  o += kWarps * 64 * 4;           // cross-warp reduction scratch
+    L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
     L.total = o;
     return L;
 }
@@ -333,6 +333,7 @@ __device__ __forceinline__ int route_scratch_words(int E, int K) { return 2 * E 
 __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int tid, uint32_t* scratch, int* s_ids,
                                              float* s_w, unsigned long long* s_mask, bool write_global) {
     const int E = P.E, K = P.K, warp = tid >> 5, lane = tid & 31;
+    const int kThreads = blockDim.x, kWarps = blockDim.x >> 5;
     const int nseg = (E + 31) / 32, Kc = K < 32 ? K : 32, C = nseg * Kc;
     uint32_t* s_key = scratch;
     float* s_val = reinterpret_cast<float*>(scratch + nt * E);
@@ -380,8 +381,8 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
         if (rank < K && me < E) { s_ids[(t0 + t) * K + rank] = me; s_w[(t0 + t) * K + rank] = s_val[t * E + me]; }
     }
     __syncthreads();
-    if (warp < nt) {                                       // weights of the selected experts, one warp per token
-        const int t = t0 + warp;
+    for (int tl = warp; tl < nt; tl += kWarps) {           // weights of the selected experts, one warp per token
+        const int t = t0 + tl;
         float v = (lane < K) ? s_w[t * K + lane] : 0.f;
         float total = 1.0f;
         if (softmax) {
@@ -389,7 +390,7 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
             v = (lane < K) ? expf(v - mx) : 0.f;
             if (!P.renorm) {
                 total = 0.f;
-                for (int e = lane; e < E; e += 32) total += expf(s_val[warp * E + e] - mx);
+                for (int e = lane; e < E; e += 32) total += expf(s_val[tl * E + e] - mx);
 #pragma unroll
                 for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
             }
@@ -418,13 +419,14 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
 }
 
 // dot products of two router rows (e0 and, if `two`, e1) with up to 8 tokens: this thread's share of H
-// (16-byte chunks strided by the block); both rows travel together so that all loads are in flight at once
-__device__ __forceinline__ void router_partial(const Params& P, int e0, int e1, bool two, int t0, int tid, float* acc0, float* acc1) {
+// (16-byte chunks strided by `nthreads`); both rows travel together so that all loads are in flight at once
+__device__ __forceinline__ void router_partial(const Params& P, int e0, int e1, bool two, int t0, int tid, int nthreads,
+                                               float* acc0, float* acc1) {
     const int H = P.H, T = P.T;
     const uint4* w0 = reinterpret_cast<const uint4*>(P.Wr + (size_t)e0 * H);
     const uint4* w1 = reinterpret_cast<const uint4*>(P.Wr + (size_t)(two ? e1 : e0) * H);
 #pragma unroll 4
-    for (int c = tid; c < H / 8; c += kThreads) {
+    for (int c = tid; c < H / 8; c += nthreads) {
         const uint4 a = __ldg(w0 + c), b = __ldg(w1 + c);
         const uint32_t ar[4] = {a.x, a.y, a.z, a.w}, br[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -449,14 +451,19 @@ __device__ __forceinline__ void router_partial(const Params& P, int e0, int e1, 
 // the kernel
 // N  = MMA N (token tile, 16/32/64); TC = token columns the accumulator warps actually read (power of two >= T).
 // ---------------------------------------------------------------------------------------------
+// Accumulator warps: one group of 4 warps for TC <= 16, two groups (each half of the token columns) for TC >= 32.
 template <int N, int TC>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(128 + 128 * (TC >= 32 ? 2 : 1), 1)
 moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                   const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmHq,
                   const __grid_constant__ Params P) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
+    constexpr int kEpiGroups = (TC >= 32) ? 2 : 1;
+    constexpr int kEpiThreads = kEpiGroupThreads * kEpiGroups;
+    constexpr int kThreads = 128 + kEpiThreads, kWarps = kThreads / 32;
+    constexpr int TCG = TC / kEpiGroups;                         // token columns per accumulator group
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
@@ -499,7 +506,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
         for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4 * kEpiGroups); }
         mbar_init(bar_drain, 1);
         mbar_init(bar_drain + 16, 1);
         misc[3] = 0u;
@@ -526,15 +533,16 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (lane == 0) P.xs[p] = s;
         }
         if (tid == 0) MOE_STAMP(1);
-        // router logits: CTA c owns experts c, c+G, ...; two experts at a time, all 256 threads split H  (Section 3.3)
-        for (int e0 = cta; e0 < E; e0 += 2 * G) {
-            const int e1 = e0 + G;
-            const bool two = e1 < E;
-            for (int t0 = 0; t0 < T; t0 += 8) {
+        if (T <= 8) {
+            // router logits, few tokens: CTA c owns experts c, c+G, ...; two experts at a time, all 256 threads split H
+            // (Section 3.3)
+            for (int e0 = cta; e0 < E; e0 += 2 * G) {
+                const int e1 = e0 + G;
+                const bool two = e1 < E;
                 float acc0[8], acc1[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
-                router_partial(P, e0, e1, two, t0, tid, acc0, acc1);
+                router_partial(P, e0, e1, two, 0, tid, kThreads, acc0, acc1);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
 #pragma unroll
@@ -545,13 +553,29 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (lane == 0) { s_red[warp * 16 + j] = acc0[j]; s_red[warp * 16 + 8 + j] = acc1[j]; }
                 }
                 __syncthreads();
-                if (tid < 16 && t0 + (tid & 7) < T && (tid < 8 || two)) {
+                if (tid < 16 && (tid & 7) < T && (tid < 8 || two)) {
                     float v = 0.f;
 #pragma unroll
                     for (int w = 0; w < kWarps; ++w) v += s_red[w * 16 + tid];
-                    P.logits[(size_t)(t0 + (tid & 7)) * E + (tid < 8 ? e0 : e1)] = v;
+                    P.logits[(size_t)(tid & 7) * E + (tid < 8 ? e0 : e1)] = v;
                 }
                 __syncthreads();
+            }
+        } else {
+            // router logits, many tokens: one warp per (expert, group of 8 tokens), lanes split H; no block barrier
+            const int groups8 = (T + 7) / 8;
+            for (int item = cta * kWarps + warp; item < E * groups8; item += G * kWarps) {
+                const int e = item / groups8, t0 = (item - e * groups8) * 8;
+                float acc0[8], acc1[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+                router_partial(P, e, e, false, t0, lane, 32, acc0, acc1);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                    for (int o = 16; o; o >>= 1) acc0[j] += __shfl_xor_sync(0xffffffffu, acc0[j], o);
+                    if (lane == 0 && t0 + j < T) P.logits[(size_t)(t0 + j) * E + e] = acc0[j];
+                }
             }
         }
     }
@@ -577,7 +601,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         for (int i = tid; i < T * KBu; i += kThreads) s_xs[(i % KBu) * TS + i / KBu] = __ldcg(P.xs + i);   // transposed: [K block][token]
         // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
         int chunk = (S * L.stage_bytes) / (4 * route_scratch_words(E, K));
-        chunk = chunk < kWarps ? chunk : kWarps;
+        chunk = chunk < kMaxTokens ? chunk : kMaxTokens;
         for (int t0 = 0; t0 < T; t0 += chunk)
             route_tokens(P, t0, min(chunk, T - t0), tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0);
         if (tid == 0) MOE_STAMP(6);
@@ -753,13 +777,14 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     else if (warp >= kEpiWarp0 && alive) {
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
+        const int cb = ((warp - kEpiWarp0) >> 2) * TCG;        // first token column of this accumulator group
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         volatile uint32_t* s_giveup = misc + 3;
         bool first_acc = true;
-        constexpr int CH = TC < 16 ? TC : 16;                  // columns per TMEM load
+        constexpr int CH = TCG < 16 ? TCG : 16;                // columns per TMEM load
         int buf = 0, hs_e = -1;
         uint32_t tph = 0;
-        float accg[TC], accu[TC];
+        float accg[TCG], accu[TCG];
 
         for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
             const bool up = (phase == 0);
@@ -800,15 +825,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (!up && e != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert)
                     const bool got = (etid == 0) ? wt.flag(e_cnt + e, (unsigned)IB, 8) : true;
-                    if (!epi_all(got)) { wt.dead = true; break; }
+                    if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
                     for (int i = etid; i < IB * N; i += kEpiThreads) s_hs[i] = __ldcg(P.hs + (size_t)e * IB * N + i);
                     hs_e = e;
-                    epi_bar();
+                    epi_bar(kEpiThreads);
                 }
                 const float* as_p = up ? (s_xs + kb0 * TS) : (s_hs + kb0 * N);   // activation scales [K block][token]
                 const int as_step = up ? TS : N;
 #pragma unroll
-                for (int n = 0; n < TC; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
+                for (int n = 0; n < TCG; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
                 for (int i = 0; i < pend - s; ++i) {
                     const int j = (s + i - lo) & 31;
@@ -825,12 +850,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
                     const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
 #pragma unroll
-                    for (int c = 0; c < TC; c += CH) {
+                    for (int c = 0; c < TCG; c += CH) {
                         float dg[CH], du[CH];
-                        tmem_ld<CH>(tcol + c, dg);
-                        if (up) tmem_ld<CH>(tcol + N + c, du);
+                        tmem_ld<CH>(tcol + cb + c, dg);
+                        if (up) tmem_ld<CH>(tcol + N + cb + c, du);
                         tmem_ld_wait();
-                        if (c + CH == TC) {                             // accumulator is in registers: free the buffer
+                        if (c + CH == TCG) {                             // accumulator is in registers: free the buffer
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
@@ -839,12 +864,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         if constexpr (CH >= 4) {
 #pragma unroll
                             for (int jj = 0; jj < CH; jj += 4) {
-                                const float4 v = *reinterpret_cast<const float4*>(as_p + i * as_step + c + jj);
+                                const float4 v = *reinterpret_cast<const float4*>(as_p + i * as_step + cb + c + jj);
                                 as[jj] = v.x; as[jj + 1] = v.y; as[jj + 2] = v.z; as[jj + 3] = v.w;
                             }
                         } else {
 #pragma unroll
-                            for (int jj = 0; jj < CH; ++jj) as[jj] = as_p[i * as_step + c + jj];
+                            for (int jj = 0; jj < CH; ++jj) as[jj] = as_p[i * as_step + cb + c + jj];
                         }
 #pragma unroll
                         for (int jj = 0; jj < CH; ++jj) {
@@ -858,7 +883,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const bool unit_done = (pend == uend);
                 s = pend;
                 if (s < hi && unit_done) w.init(s, KB, MB, s_act);
-                epi_bar();
+                epi_bar(kEpiThreads);
                 if (*s_giveup) { wt.dead = true; break; }
                 const unsigned long long mask = s_mask[e];
 
@@ -867,12 +892,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // not the owner: park the partial accumulator, [column][row] so rows are contiguous
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
-                    for (int n = 0; n < TC; ++n)
-                        if ((mask >> n) & 1ull) {                        // only tokens routed to this expert matter
-                            __stcg(dst + n * kBlock + row, accg[n]);
-                            if (up) __stcg(dst + (N + n) * kBlock + row, accu[n]);
+                    for (int n = 0; n < TCG; ++n)
+                        if ((mask >> (cb + n)) & 1ull) {                        // only tokens routed to this expert matter
+                            __stcg(dst + (cb + n) * kBlock + row, accg[n]);
+                            if (up) __stcg(dst + (N + cb + n) * kBlock + row, accu[n]);
                         }
-                    epi_bar();
+                    epi_bar(kEpiThreads);
                     if (etid == 0) st_release(pflag + cta, tag);
                     continue;
                 }
@@ -890,69 +915,73 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         if (range_lo(S_all, min(base + kEpiThreads, G), G, q_all) >= uend) break;
                     }
                     while (c_end < G && range_lo(S_all, c_end, G, q_all) < uend) ++c_end;
-                    if (!epi_all(got)) { wt.dead = true; break; }
+                    if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
                     for (int c = cta + 1; c < c_end; ++c) {
                         if (range_lo(S_all, c + 1, G, q_all) == range_lo(S_all, c, G, q_all)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
-                        for (int n = 0; n < TC; ++n)
-                            if ((mask >> n) & 1ull) {
-                                accg[n] += __ldcg(src + n * kBlock + row);
-                                if (up) accu[n] += __ldcg(src + (N + n) * kBlock + row);
+                        for (int n = 0; n < TCG; ++n)
+                            if ((mask >> (cb + n)) & 1ull) {
+                                accg[n] += __ldcg(src + (cb + n) * kBlock + row);
+                                if (up) accu[n] += __ldcg(src + (N + cb + n) * kBlock + row);
                             }
                     }
                 }
                 if (up) {
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
-                    for (int n = 0; n < TC; ++n) {
-                        if ((mask >> n) & 1ull) {                        // warp-uniform: other tokens cost nothing
+                    for (int n = 0; n < TCG; ++n) {
+                        if ((mask >> (cb + n)) & 1ull) {                        // warp-uniform: other tokens cost nothing
                             const float g = accg[n];
                             const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
                             accg[n] = a;
                             float m = fabsf(a);
 #pragma unroll
                             for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                            if (lane == 0) s_red[q * N + n] = m;
+                            if (lane == 0) s_red[q * N + cb + n] = m;
                         }
                     }
-                    epi_bar();
+                    epi_bar(kEpiThreads);
 #pragma unroll
-                    for (int n = 0; n < TC; ++n) {
-                        if ((mask >> n) & 1ull) {
-                            const float amax = fmaxf(fmaxf(s_red[n], s_red[N + n]), fmaxf(s_red[2 * N + n], s_red[3 * N + n]));
+                    for (int n = 0; n < TCG; ++n) {
+                        if ((mask >> (cb + n)) & 1ull) {
+                            const float amax = fmaxf(fmaxf(s_red[cb + n], s_red[N + cb + n]), fmaxf(s_red[2 * N + cb + n], s_red[3 * N + cb + n]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
                             const float2 v = make_float2(__fdiv_rn(accg[n], sc), 0.f);
                             const uint8_t code = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
-                            P.hq[((size_t)e * N + n) * I + mb * kBlock + row] = code;
-                            if (row == 0) P.hs[((size_t)e * IB + mb) * N + n] = sc;
+                            P.hq[((size_t)e * N + cb + n) * I + mb * kBlock + row] = code;
+                            if (row == 0) P.hs[((size_t)e * IB + mb) * N + cb + n] = sc;
                         }
                     }
                     fence_proxy_async();
-                    epi_bar();
+                    epi_bar(kEpiThreads);
                     if (etid == 0) red_release_add(e_cnt + e, 1u);   // the expert's tile is complete at count == I/128
                 } else {
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
-                    for (int n = 0; n < TC; ++n) {
-                        if ((mask >> n) & 1ull) {
+                    for (int n = 0; n < TCG; ++n) {
+                        if ((mask >> (cb + n)) & 1ull) {
                             int sl = 0;
-                            for (int jj = 0; jj < K; ++jj) if (s_ids[n * K + jj] == e) sl = jj;
-                            __stcg(P.y + ((size_t)n * K + sl) * H + mb * kBlock + row, accg[n]);
+                            for (int jj = 0; jj < K; ++jj) if (s_ids[(cb + n) * K + jj] == e) sl = jj;
+                            __stcg(P.y + ((size_t)(cb + n) * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
-                    epi_bar();
+                    epi_bar(kEpiThreads);
                     if (etid == 0) st_release(P.dn_done + e * HB + mb, tag);
                 }
             }
         }
         if (etid == 0) MOE_STAMP(13);
         // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block) over all CTAs
-        for (int task = cta; task < T * HB && !wt.dead; task += G) {
-            const int t = task / HB, hb = task - t * HB;
+        const int grp = (warp - kEpiWarp0) >> 2, gtid = etid & (kEpiGroupThreads - 1);
+        for (int task0 = cta * kEpiGroups; task0 < T * HB && !wt.dead; task0 += G * kEpiGroups) {
+            const int task = task0 + grp;
+            const bool mine = task < T * HB;
+            const int t = mine ? task / HB : 0, hb = mine ? task - t * HB : 0;
             bool got = true;
-            if (etid < K) got = wt.flag(P.dn_done + s_ids[t * K + etid] * HB + hb, tag, 7);
-            if (!epi_all(got)) { wt.dead = true; break; }
+            if (mine && gtid < K) got = wt.flag(P.dn_done + s_ids[t * K + gtid] * HB + hb, tag, 7);
+            if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
+            if (!mine) continue;
             float acc = 0.f;
             const float* yp = P.y + (size_t)t * K * H + hb * kBlock + row;
             for (int j0 = 0; j0 < K; j0 += 8) {
