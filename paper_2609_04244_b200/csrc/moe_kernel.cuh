@@ -340,6 +340,7 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
     // candidates are packed as (key << 32 | ~index): "a beats b" is then one 64-bit compare
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
     const bool softmax = (P.scoring == 0);
+#pragma unroll 4
     for (int p = tid; p < nt * E; p += kThreads) {
         const float l = __ldcg(P.logits + (size_t)t0 * E + p);
         if (softmax) {
@@ -562,20 +563,41 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 __syncthreads();
             }
         } else {
-            // router logits, many tokens: one warp per (expert, group of 8 tokens), lanes split H; no block barrier
-            const int groups8 = (T + 7) / 8;
-            for (int item = cta * kWarps + warp; item < E * groups8; item += G * kWarps) {
-                const int e = item / groups8, t0 = (item - e * groups8) * 8;
-                float acc0[8], acc1[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
-                router_partial(P, e, e, false, t0, lane, 32, acc0, acc1);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-#pragma unroll
-                    for (int o = 16; o; o >>= 1) acc0[j] += __shfl_xor_sync(0xffffffffu, acc0[j], o);
-                    if (lane == 0 && t0 + j < T) P.logits[(size_t)(t0 + j) * E + e] = acc0[j];
+            // router logits, many tokens: a CTA takes a (16 experts x 8 tokens) tile, its warps split H, each warp
+            // accumulates its share with warp-level bf16 MMAs (m16n8k16, fp32 accumulate) straight from global
+            // memory; the warps' partial tiles are summed in warp order (deterministic).  The router is ~0.01 % of
+            // the step's flops; this is about latency, not about the tensor pipe.
+            float* tile = reinterpret_cast<float*>(smem);               // [kWarps][32 lanes][4] partial tiles
+            const int nEB = (E + 15) / 16, nTB = (T + 7) / 8;
+            const int g = lane >> 2, tq = lane & 3;
+            const int kper = (H / 16 + kWarps - 1) / kWarps * 16;       // K range of one warp (multiple of 16)
+            for (int item = cta; item < nEB * nTB; item += G) {
+                const int eb = item / nTB, tb = item - eb * nTB;
+                const int r0 = eb * 16 + g, r1 = r0 + 8, tok = tb * 8 + g;
+                const uint32_t* a0p = reinterpret_cast<const uint32_t*>(P.Wr + (size_t)(r0 < E ? r0 : 0) * H);
+                const uint32_t* a1p = reinterpret_cast<const uint32_t*>(P.Wr + (size_t)(r1 < E ? r1 : 0) * H);
+                const uint32_t* bp = reinterpret_cast<const uint32_t*>(P.hidden + (size_t)(tok < T ? tok : 0) * H);
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
+                const int k_lo = warp * kper, k_hi = min(H, k_lo + kper);
+#pragma unroll 4
+                for (int k = k_lo; k < k_hi; k += 16) {
+                    const int o = (k >> 1) + tq;                          // 32-bit word holding elements k+2tq, k+2tq+1
+                    const uint32_t a0 = __ldg(a0p + o), a1 = __ldg(a1p + o), a2 = __ldg(a0p + o + 4), a3 = __ldg(a1p + o + 4);
+                    const uint32_t b0 = __ldg(bp + o), b1 = __ldg(bp + o + 4);
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
                 }
+                *reinterpret_cast<float4*>(tile + (warp * 32 + lane) * 4) = make_float4(c[0], c[1], c[2], c[3]);
+                __syncthreads();
+                if (tid < 128) {
+                    float v = 0.f;
+                    for (int w = 0; w < kWarps; ++w) v += tile[w * 128 + tid];
+                    const int ln = tid >> 2, i = tid & 3;
+                    const int row = eb * 16 + (ln >> 2) + (i >= 2 ? 8 : 0), col = tb * 8 + 2 * (ln & 3) + (i & 1);
+                    if (row < E && col < T) P.logits[(size_t)col * E + row] = v;
+                }
+                __syncthreads();
             }
         }
     }
