@@ -334,16 +334,16 @@ def main():
     # end to end: the step's input comes from pinned host memory, the result goes back to the host
     e2e = None
     if not args.no_e2e:
+        # through the public C-ABI call that takes HOST activations (moe_forward_host): per step one pinned
+        # host-to-device copy of the hidden state, the kernel, one device-to-host copy of the output, and a stream
+        # synchronisation because the caller consumes the result before the next step
         h_in = [layers[l]["hidden"].cpu().pin_memory() for l in range(L)]
         h_out = torch.empty((T, shape.H), dtype=torch.bfloat16).pin_memory()
-        d_in = torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev)
 
         def e2e_step(i):
             d = layers[i % L]
-            d_in.copy_(h_in[i % L], non_blocking=True)
-            plan.forward(d_in, d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], out=outs[i % L])
-            h_out.copy_(outs[i % L], non_blocking=True)
-            stream.synchronize()          # the caller consumes the result before the next step
+            plan.forward_host(h_in[i % L], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], h_out, stream)
+            stream.synchronize()
 
         Ke = min(K, 2000)
         for i in range(W):

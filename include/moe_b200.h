@@ -100,6 +100,19 @@ int moe_forward(moe_plan_t plan, int T,
                 void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream);
 
 /*
+ * moe_forward_host: moe_forward with the step's activations in HOST memory (Section 3: same operator).
+ *   hidden_host [T,H] bf16 and out_host [T,H] bf16 are host pointers (pinned memory makes the copies asynchronous);
+ *   every other tensor is a device pointer as in moe_forward.  Enqueues, on `stream`: a host-to-device copy of
+ *   `hidden_host` into a staging area of the workspace, the kernel, and a device-to-host copy of the result.  The
+ *   host buffers must stay valid, and `out_host` must not be read, until the stream has been synchronised.
+ */
+int moe_forward_host(moe_plan_t plan, int T,
+                     const void* hidden_host, const void* Wr_bf16, const float* sel_bias,
+                     const void* W13_fp8, const float* W13_scale,
+                     const void* W2_fp8, const float* W2_scale,
+                     void* out_host, void* workspace, size_t workspace_bytes, moe_stream_t stream);
+
+/*
  * moe_forward_noalloc: moe_forward for callers that cannot give the library device memory.  (The paper has no
  * counterpart: this entry point exists only for integration.)  Some hosts of this library may not call cudaMalloc
  * at the point where they run a decode step -- for instance code running inside a memory pool that owns the whole

@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_noalloc", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -56,6 +56,8 @@ def load_library():
     lib.moe_forward.argtypes = [vp, i] + [vp] * 9 + [sz, vp]
     lib.moe_forward_noalloc.restype = i
     lib.moe_forward_noalloc.argtypes = [vp, i] + [vp] * 8 + [vp]
+    lib.moe_forward_host.restype = i
+    lib.moe_forward_host.argtypes = [vp, i] + [vp] * 9 + [sz, vp]
     lib.moe_forward_debug.restype = i
     lib.moe_forward_debug.argtypes = [vp, i] + [vp] * 9 + [sz, vp] + [vp] * 5
     lib.moe_sync_status.restype = i
@@ -116,6 +118,15 @@ def moe_forward(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, worksp
                                       _stream(stream)))
 
 
+def moe_forward_host(plan, T, hidden_host, Wr, sel_bias, W13q, W13s, W2q, W2s, out_host, workspace, stream=None) -> None:
+    """One decode step with the activations in (pinned) host tensors; weights and workspace stay on the device."""
+    if hidden_host.is_cuda or out_host.is_cuda or not hidden_host.is_contiguous() or not out_host.is_contiguous():
+        raise MoEError(-1, "hidden_host and out_host must be contiguous host tensors")
+    _check(load_library().moe_forward_host(plan, T, ctypes.c_void_p(hidden_host.data_ptr()), _p(Wr), _p(sel_bias),
+                                           _p(W13q), _p(W13s), _p(W2q), _p(W2s), ctypes.c_void_p(out_host.data_ptr()),
+                                           _p(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def moe_forward_noalloc(plan, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, stream=None) -> None:
     """One decode step using the library's built-in scratch array instead of a caller workspace.
 
@@ -167,6 +178,11 @@ class MoEPlan:
             out = torch.empty((T, self.H), dtype=torch.bfloat16, device=hidden.device)
         moe_forward(self.handle, T, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out, self.workspace, stream)
         return out
+
+    def forward_host(self, hidden_host, Wr, sel_bias, W13q, W13s, W2q, W2s, out_host, stream=None):
+        moe_forward_host(self.handle, hidden_host.shape[0], hidden_host, Wr, sel_bias, W13q, W13s, W2q, W2s, out_host,
+                         self.workspace, stream)
+        return out_host
 
     def forward_debug(self, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, stream=None):
         T, dev = hidden.shape[0], hidden.device

@@ -56,7 +56,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
     size_t ctrl, e_cnt, dn_done, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
-    size_t stamps, logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, total;
+    size_t stamps, logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, total;
 };
 
 struct MapKey {
@@ -103,6 +103,8 @@ struct moe_plan {
         L.part_up = o;  o += align_up((size_t)G * 2 * N * 128 * 4, 256);
         L.part_dn = o;  o += align_up((size_t)G * N * 128 * 4, 256);
         L.y = o;        o += align_up((size_t)Tc * K * H * 4, 256);
+        L.stage_in = o;  o += align_up((size_t)Tc * H * 2, 256);    // device copies of host-resident input/output
+        L.stage_out = o; o += align_up((size_t)Tc * H * 2, 256);    // (moe_forward_host)
         L.total = o;
         return L;
     }
@@ -421,6 +423,35 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     if (T <= 16) return launch<16, 16>(plan, m13, m2, mx, mh, P, smem_bytes, s);
     if (T <= 32) return launch<32, 32>(plan, m13, m2, mx, mh, P, smem_bytes, s);
     return launch<64, 64>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+}
+
+int moe_forward_host(moe_plan_t plan, int T, const void* hidden_host, const void* Wr_bf16, const float* sel_bias,
+                     const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
+                     void* out_host, void* workspace, size_t workspace_bytes, moe_stream_t stream) {
+    if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (!hidden_host || !out_host) return fail(MOE_ERR_ARG, "a host buffer is NULL");
+    if (!workspace) return fail(MOE_ERR_WORKSPACE, "workspace is NULL");
+    if (T < 1) return fail(MOE_ERR_ARG, "T must be >= 1 (got %d)", T);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    for (int t0 = 0; t0 < T; t0 += moe::kMaxTokens) {
+        const int tc = (T - t0 < moe::kMaxTokens) ? T - t0 : moe::kMaxTokens;
+        const WsLayout L = plan->layout(tc);
+        if (workspace_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", workspace_bytes, L.total, tc);
+        const size_t bytes = (size_t)tc * plan->H * 2;
+        const uint8_t* src = static_cast<const uint8_t*>(hidden_host) + (size_t)t0 * plan->H * 2;
+        uint8_t* dst = static_cast<uint8_t*>(out_host) + (size_t)t0 * plan->H * 2;
+        if (cudaMemcpyAsync(w + L.stage_in, src, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return fail(MOE_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+        int rc = check_forward_args(plan, tc, w + L.stage_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, w + L.stage_out, workspace);
+        if (rc == MOE_OK)
+            rc = forward_chunk(plan, tc, w + L.stage_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, w + L.stage_out,
+                               workspace, workspace_bytes, s);
+        if (rc != MOE_OK) return rc;
+        if (cudaMemcpyAsync(dst, w + L.stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return fail(MOE_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    return MOE_OK;
 }
 
 int moe_forward_debug(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_bf16, const float* sel_bias,

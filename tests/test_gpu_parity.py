@@ -64,3 +64,19 @@ def test_more_than_64_tokens_is_chunked():
         r = check_against_oracle(shape, hi - lo, dd, dbg, max_oracle_tokens=12)
         assert r["rel_l2"] < 2e-3, r
     plan.close()
+
+
+def test_host_activation_entry_point_matches_device_entry_point():
+    """moe_forward_host stages pinned host activations through the workspace; same kernel, same bits."""
+    from paper_2609_04244_b200 import MoEPlan
+    shape, T = SMALL_SIG, 70                                   # > 64: two chunks through the staging area
+    d = wl.make_layer(shape, T, device="cuda")
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T)
+    args = (d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
+    ref = plan.forward(d["hidden"], *args)
+    h_in = d["hidden"].cpu().pin_memory()
+    h_out = torch.zeros((T, shape.H), dtype=torch.bfloat16).pin_memory()
+    plan.forward_host(h_in, *args, h_out)
+    plan.sync_status()
+    assert torch.equal(h_out, ref.cpu())
+    plan.close()
