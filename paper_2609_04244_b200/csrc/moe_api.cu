@@ -55,8 +55,8 @@ bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t ctrl, e_cnt, dn_done, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
-    size_t stamps, logits, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, total;
+    size_t ctrl, e_cnt, dn_flag, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
+    size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, total;
 };
 
 struct MapKey {
@@ -88,12 +88,13 @@ struct moe_plan {
         size_t o = 0;
         L.ctrl = o;     o += moe::kCtrlWords * 4;
         L.e_cnt = o;    o += align_up((size_t)2 * E * 4, 256);
-        L.dn_done = o;  o += align_up((size_t)E * (H / 128) * 4, 256);
+        L.dn_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
         L.flags_end = o;
         L.stamps = o;   o += align_up((size_t)G * 16 * 8, 256);
         L.logits = o;   o += align_up((size_t)Tc * E * 4, 256);
+        L.lpart = o;    o += align_up((size_t)16 * Tc * E * 4, 256);
         L.ids = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.wts = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.xs = o;       o += align_up((size_t)Tc * (H / 128) * 4, 256);
@@ -201,6 +202,7 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.out = static_cast<__nv_bfloat16*>(out);
     P.ctrl = reinterpret_cast<unsigned*>(w + L.ctrl);
     P.logits = reinterpret_cast<float*>(w + L.logits);
+    P.lpart = reinterpret_cast<float*>(w + L.lpart);
     P.ids = reinterpret_cast<int*>(w + L.ids);
     P.wts = reinterpret_cast<float*>(w + L.wts);
     P.xq = w + L.xq;
@@ -208,7 +210,7 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.hq = w + L.hq;
     P.hs = reinterpret_cast<float*>(w + L.hs);
     P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
-    P.dn_done = reinterpret_cast<unsigned*>(w + L.dn_done);
+    P.dn_flag = reinterpret_cast<unsigned*>(w + L.dn_flag);
     P.part_up = reinterpret_cast<float*>(w + L.part_up);
     P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
     P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
@@ -401,6 +403,7 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     P.out = static_cast<__nv_bfloat16*>(out_bf16);
     P.ctrl = reinterpret_cast<unsigned*>(w + L.ctrl);
     P.logits = reinterpret_cast<float*>(w + L.logits);
+    P.lpart = reinterpret_cast<float*>(w + L.lpart);
     P.ids = reinterpret_cast<int*>(w + L.ids);
     P.wts = reinterpret_cast<float*>(w + L.wts);
     P.xq = w + L.xq;
@@ -408,7 +411,7 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     P.hq = w + L.hq;
     P.hs = reinterpret_cast<float*>(w + L.hs);
     P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
-    P.dn_done = reinterpret_cast<unsigned*>(w + L.dn_done);
+    P.dn_flag = reinterpret_cast<unsigned*>(w + L.dn_flag);
     P.part_up = reinterpret_cast<float*>(w + L.part_up);
     P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
     P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);

@@ -63,7 +63,8 @@ struct Params {
     const float* W2s;
     __nv_bfloat16* out;
     unsigned* ctrl;
-    float* logits;      // [T,E]
+    float* logits;      // [T,E]   (diagnostics: summed router logits, written by CTA 0)
+    float* lpart;       // [<=16][T,E] router logits, one slice per K-split part
     int* ids;           // [T,K]
     float* wts;         // [T,K]
     uint8_t* xq;        // [64,H]
@@ -71,7 +72,7 @@ struct Params {
     uint8_t* hq;        // [E,N,I]
     float* hs;          // [E,I/128,N]
     unsigned* e_cnt;    // [2][E] published I-blocks of an expert's intermediate tile (one row per launch parity)
-    unsigned* dn_done;  // [E,H/128] == tag once the expert's down-projection rows of that block are stored
+    unsigned* dn_flag;  // [grid] == tag once the CTA has stored every down-projection result of its range
     float* part_up;     // [grid][2N][128]
     float* part_dn;     // [grid][N][128]
     unsigned* pu_flag;  // [grid]
@@ -258,7 +259,7 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, xs_off, hs_off, red_off, misc_off, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, red_off, misc_off, total;
 };
 __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages) {
     SmemLayout L;
@@ -272,6 +273,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
     L.act_off = o;  o += (E + 1) * 4;
+    L.uidx_off = o; o += E * 4;
     o = (o + 15) & ~15;
     L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;   // input activation scales [H/128][T rounded up to 4]
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
@@ -304,6 +306,11 @@ struct Walk {
         mb = unit - u * MB;
         e = act[u];
     }
+    __device__ __forceinline__ void next_unit(const int* act) {
+        kb = 0;
+        if (++mb == MB) { mb = 0; ++u; }
+        e = act[u];
+    }
     __device__ __forceinline__ void next(const int* act) {
         if (++kb == KB) {
             kb = 0;
@@ -330,8 +337,8 @@ __device__ __forceinline__ uint32_t orderable(float f) {
 // Shared-memory scratch per token: E keys, E scores, ceil(E/32) * min(K,32) 64-bit candidates.
 __device__ __forceinline__ int route_scratch_words(int E, int K) { return 2 * E + 2 * ((E + 31) / 32) * (K < 32 ? K : 32); }
 
-__device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int tid, uint32_t* scratch, int* s_ids,
-                                             float* s_w, unsigned long long* s_mask, bool write_global) {
+__device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int ksplit, int tid, uint32_t* scratch,
+                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global) {
     const int E = P.E, K = P.K, warp = tid >> 5, lane = tid & 31;
     const int kThreads = blockDim.x, kWarps = blockDim.x >> 5;
     const int nseg = (E + 31) / 32, Kc = K < 32 ? K : 32, C = nseg * Kc;
@@ -340,9 +347,14 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
     // candidates are packed as (key << 32 | ~index): "a beats b" is then one 64-bit compare
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
     const bool softmax = (P.scoring == 0);
-#pragma unroll 4
     for (int p = tid; p < nt * E; p += kThreads) {
-        const float l = __ldcg(P.logits + (size_t)t0 * E + p);
+        float part[16];                                      // router logit = sum of the K-split parts, fixed order
+#pragma unroll
+        for (int kp = 0; kp < 16; ++kp) part[kp] = (kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
+        float l = part[0];
+#pragma unroll
+        for (int kp = 1; kp < 16; ++kp) l += part[kp];
+        if (write_global) P.logits[(size_t)t0 * E + p] = l;
         if (softmax) {
             s_val[p] = l;
             s_key[p] = orderable(l);
@@ -419,35 +431,6 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
     return lo | (hi << 16);
 }
 
-// dot products of two router rows (e0 and, if `two`, e1) with up to 8 tokens: this thread's share of H
-// (16-byte chunks strided by `nthreads`); both rows travel together so that all loads are in flight at once
-__device__ __forceinline__ void router_partial(const Params& P, int e0, int e1, bool two, int t0, int tid, int nthreads,
-                                               float* acc0, float* acc1) {
-    const int H = P.H, T = P.T;
-    const uint4* w0 = reinterpret_cast<const uint4*>(P.Wr + (size_t)e0 * H);
-    const uint4* w1 = reinterpret_cast<const uint4*>(P.Wr + (size_t)(two ? e1 : e0) * H);
-#pragma unroll 4
-    for (int c = tid; c < H / 8; c += nthreads) {
-        const uint4 a = __ldg(w0 + c), b = __ldg(w1 + c);
-        const uint32_t ar[4] = {a.x, a.y, a.z, a.w}, br[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (t0 + j < T) {
-                const uint4 xv = __ldg(reinterpret_cast<const uint4*>(P.hidden + (size_t)(t0 + j) * H) + c);
-                const uint32_t xr[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float xl = __uint_as_float(xr[q] << 16), xh = __uint_as_float(xr[q] & 0xFFFF0000u);
-                    acc0[j] = fmaf(__uint_as_float(ar[q] << 16), xl, acc0[j]);
-                    acc0[j] = fmaf(__uint_as_float(ar[q] & 0xFFFF0000u), xh, acc0[j]);
-                    acc1[j] = fmaf(__uint_as_float(br[q] << 16), xl, acc1[j]);
-                    acc1[j] = fmaf(__uint_as_float(br[q] & 0xFFFF0000u), xh, acc1[j]);
-                }
-            }
-        }
-    }
-}
-
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // N  = MMA N (token tile, 16/32/64); TC = token columns the accumulator warps actually read (power of two >= T).
@@ -485,6 +468,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
     int* s_act = (int*)(smem + L.act_off);
+    int* s_uidx = (int*)(smem + L.uidx_off);               // expert -> position in the active list
     float* s_xs = (float*)(smem + L.xs_off);
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
@@ -518,6 +502,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
     // ------------------------------------------------------------------ phase R: quantise + logits
+    int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
+    {
+        const int items = ((E + 15) / 16) * ((T + 7) / 8);
+        while (ksplit < 16 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
+    }
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
         const int groups = T * KBu;
@@ -534,51 +523,26 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (lane == 0) P.xs[p] = s;
         }
         if (tid == 0) MOE_STAMP(1);
-        if (T <= 8) {
-            // router logits, few tokens: CTA c owns experts c, c+G, ...; two experts at a time, all 256 threads split H
-            // (Section 3.3)
-            for (int e0 = cta; e0 < E; e0 += 2 * G) {
-                const int e1 = e0 + G;
-                const bool two = e1 < E;
-                float acc0[8], acc1[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
-                router_partial(P, e0, e1, two, 0, tid, kThreads, acc0, acc1);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-#pragma unroll
-                    for (int o = 16; o; o >>= 1) {
-                        acc0[j] += __shfl_xor_sync(0xffffffffu, acc0[j], o);
-                        acc1[j] += __shfl_xor_sync(0xffffffffu, acc1[j], o);
-                    }
-                    if (lane == 0) { s_red[warp * 16 + j] = acc0[j]; s_red[warp * 16 + 8 + j] = acc1[j]; }
-                }
-                __syncthreads();
-                if (tid < 16 && (tid & 7) < T && (tid < 8 || two)) {
-                    float v = 0.f;
-#pragma unroll
-                    for (int w = 0; w < kWarps; ++w) v += s_red[w * 16 + tid];
-                    P.logits[(size_t)(tid & 7) * E + (tid < 8 ? e0 : e1)] = v;
-                }
-                __syncthreads();
-            }
-        } else {
-            // router logits, many tokens: a CTA takes a (16 experts x 8 tokens) tile, its warps split H, each warp
-            // accumulates its share with warp-level bf16 MMAs (m16n8k16, fp32 accumulate) straight from global
-            // memory; the warps' partial tiles are summed in warp order (deterministic).  The router is ~0.01 % of
-            // the step's flops; this is about latency, not about the tensor pipe.
+        // Router logits (Section 3.3): a (16 experts x 8 tokens) tile and one of `ksplit` parts of H per CTA turn; the
+        // CTA's warps split that part of H, each accumulates with warp-level bf16 MMAs (m16n8k16, fp32 accumulate)
+        // straight from global memory, the warps' partial tiles are summed in warp order, and the K-split parts are
+        // summed in part order by whoever reads the logits (deterministic).  The router is ~0.01 % of the step's
+        // flops: this is about latency and about spreading the reads of Wr over all SMs, not about the tensor pipe.
+        {
             float* tile = reinterpret_cast<float*>(smem);               // [kWarps][32 lanes][4] partial tiles
             const int nEB = (E + 15) / 16, nTB = (T + 7) / 8;
             const int g = lane >> 2, tq = lane & 3;
-            const int kper = (H / 16 + kWarps - 1) / kWarps * 16;       // K range of one warp (multiple of 16)
-            for (int item = cta; item < nEB * nTB; item += G) {
+            const int kpart_len = H / ksplit;
+            const int kper = (kpart_len / 16 + kWarps - 1) / kWarps * 16;   // K range of one warp (multiple of 16)
+            for (int wi = cta; wi < nEB * nTB * ksplit; wi += G) {
+                const int item = wi / ksplit, kp = wi - item * ksplit;
                 const int eb = item / nTB, tb = item - eb * nTB;
                 const int r0 = eb * 16 + g, r1 = r0 + 8, tok = tb * 8 + g;
                 const uint32_t* a0p = reinterpret_cast<const uint32_t*>(P.Wr + (size_t)(r0 < E ? r0 : 0) * H);
                 const uint32_t* a1p = reinterpret_cast<const uint32_t*>(P.Wr + (size_t)(r1 < E ? r1 : 0) * H);
                 const uint32_t* bp = reinterpret_cast<const uint32_t*>(P.hidden + (size_t)(tok < T ? tok : 0) * H);
                 float c[4] = {0.f, 0.f, 0.f, 0.f};
-                const int k_lo = warp * kper, k_hi = min(H, k_lo + kper);
+                const int k_lo = kp * kpart_len + warp * kper, k_hi = min((kp + 1) * kpart_len, k_lo + kper);
 #pragma unroll 4
                 for (int k = k_lo; k < k_hi; k += 16) {
                     const int o = (k >> 1) + tq;                          // 32-bit word holding elements k+2tq, k+2tq+1
@@ -595,7 +559,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     for (int w = 0; w < kWarps; ++w) v += tile[w * 128 + tid];
                     const int ln = tid >> 2, i = tid & 3;
                     const int row = eb * 16 + (ln >> 2) + (i >= 2 ? 8 : 0), col = tb * 8 + 2 * (ln & 3) + (i & 1);
-                    if (row < E && col < T) P.logits[(size_t)col * E + row] = v;
+                    if (row < E && col < T) P.lpart[((size_t)kp * T + col) * E + row] = v;
                 }
                 __syncthreads();
             }
@@ -625,7 +589,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         int chunk = (S * L.stage_bytes) / (4 * route_scratch_words(E, K));
         chunk = chunk < kMaxTokens ? chunk : kMaxTokens;
         for (int t0 = 0; t0 < T; t0 += chunk)
-            route_tokens(P, t0, min(chunk, T - t0), tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0);
+            route_tokens(P, t0, min(chunk, T - t0), ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0);
         if (tid == 0) MOE_STAMP(6);
         if (warp == 0) {                                   // active-expert list in ascending expert order
             int base = 0;
@@ -633,7 +597,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int e = e0 + lane;
                 const bool on = (e < E) && (s_mask[e] != 0ull);
                 const unsigned b = __ballot_sync(0xffffffffu, on);
-                if (on) s_act[base + __popc(b & ((1u << lane) - 1u))] = e;
+                if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
                 base += __popc(b);
             }
             if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
@@ -904,10 +868,23 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 }
                 const bool unit_done = (pend == uend);
                 s = pend;
-                if (s < hi && unit_done) w.init(s, KB, MB, s_act);
+                if (unit_done) w.next_unit(s_act);
+                const unsigned long long mask = s_mask[e];
+                if (!up && unit_done && ustart >= lo) {
+                    // whole down unit: every warp stores its rows and counts itself done -- no block-level barrier
+                    // (units of the down projection can be as short as two k-steps)
+#pragma unroll
+                    for (int n = 0; n < TCG; ++n) {
+                        if ((mask >> (cb + n)) & 1ull) {
+                            int sl = 0;
+                            for (int jj = 0; jj < K; ++jj) if (s_ids[(cb + n) * K + jj] == e) sl = jj;
+                            __stcg(P.y + ((size_t)(cb + n) * K + sl) * H + mb * kBlock + row, accg[n]);
+                        }
+                    }
+                    continue;                                   // published once per CTA, after the last down unit
+                }
                 epi_bar(kEpiThreads);
                 if (*s_giveup) { wt.dead = true; break; }
-                const unsigned long long mask = s_mask[e];
 
                 // ---- end of this CTA's piece of the unit: combine split-K partials, then the epilogue
                 if (ustart < lo) {
@@ -988,12 +965,14 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             __stcg(P.y + ((size_t)(cb + n) * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
-                    epi_bar(kEpiThreads);
-                    if (etid == 0) st_release(P.dn_done + e * HB + mb, tag);
+                    // (published once per CTA, after the last down unit)
                 }
             }
         }
-        if (etid == 0) MOE_STAMP(13);
+        // every down-projection result of this CTA's range is stored: one release for all of them (a release per
+        // unit would stall on the unit's own stores; units can be as short as two k-steps)
+        epi_bar(kEpiThreads);
+        if (etid == 0) { st_release(P.dn_flag + cta, tag); MOE_STAMP(13); }
         // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block) over all CTAs
         const int grp = (warp - kEpiWarp0) >> 2, gtid = etid & (kEpiGroupThreads - 1);
         for (int task0 = cta * kEpiGroups; task0 < T * HB && !wt.dead; task0 += G * kEpiGroups) {
@@ -1001,7 +980,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const bool mine = task < T * HB;
             const int t = mine ? task / HB : 0, hb = mine ? task - t * HB : 0;
             bool got = true;
-            if (mine && gtid < K) got = wt.flag(P.dn_done + s_ids[t * K + gtid] * HB + hb, tag, 7);
+            if (mine && gtid < K) {
+                // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
+                const unsigned x = (unsigned)((s_uidx[s_ids[t * K + gtid]] * HB + hb) * KBd / q_dn);
+                const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)(S_dn / q_dn);
+                got = wt.flag(P.dn_flag + owner, tag, 7);
+            }
             if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
             if (!mine) continue;
             float acc = 0.f;
