@@ -46,7 +46,7 @@ constexpr int kStampsPerCta = 16;
 
 // control words at the head of the workspace
 // (the two arrival counters are used by alternate launches: a launch counts in one and clears the other)
-enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kExitCnt = 5, kCtrlWords = 64 };
+enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kExitCnt = 5, kRouteCnt2 = 6, kCtrlWords = 64 };
 // device status codes
 enum DevStatus { kDevOk = 0, kDevTimeout = 1 };
 
@@ -64,7 +64,7 @@ struct Params {
     __nv_bfloat16* out;
     unsigned* ctrl;
     float* logits;      // [T,E]   (diagnostics: summed router logits, written by CTA 0)
-    float* lpart;       // [<=16][T,E] router logits, one slice per K-split part
+    float* lpart;       // [<=4][T,E] router logits, one slice per K-split part
     int* ids;           // [T,K]
     float* wts;         // [T,K]
     uint8_t* xq;        // [64,H]
@@ -338,7 +338,8 @@ __device__ __forceinline__ uint32_t orderable(float f) {
 __device__ __forceinline__ int route_scratch_words(int E, int K) { return 2 * E + 2 * ((E + 31) / 32) * (K < 32 ? K : 32); }
 
 __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int ksplit, int tid, uint32_t* scratch,
-                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global) {
+                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global,
+                                             bool build_mask) {
     const int E = P.E, K = P.K, warp = tid >> 5, lane = tid & 31;
     const int kThreads = blockDim.x, kWarps = blockDim.x >> 5;
     const int nseg = (E + 31) / 32, Kc = K < 32 ? K : 32, C = nseg * Kc;
@@ -347,25 +348,35 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
     // candidates are packed as (key << 32 | ~index): "a beats b" is then one 64-bit compare
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
     const bool softmax = (P.scoring == 0);
-    for (int p = tid; p < nt * E; p += kThreads) {
-        float part[16];                                      // router logit = sum of the K-split parts, fixed order
+    for (int p0 = tid; p0 < nt * E; p0 += 2 * kThreads) {      // two elements per turn: all their loads in flight at once
+        float part[2][4];                                        // router logit = sum of the K-split parts, fixed order
 #pragma unroll
-        for (int kp = 0; kp < 16; ++kp) part[kp] = (kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
-        float l = part[0];
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-        for (int kp = 1; kp < 16; ++kp) l += part[kp];
-        if (write_global) P.logits[(size_t)t0 * E + p] = l;
-        if (softmax) {
-            s_val[p] = l;
-            s_key[p] = orderable(l);
-        } else {
-            const int e = p % E;
-            const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
-            s_val[p] = sg;
-            s_key[p] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
+            for (int kp = 0; kp < 4; ++kp) {
+                const int p = p0 + j * kThreads;
+                part[j][kp] = (p < nt * E && kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
+            }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int p = p0 + j * kThreads;
+            if (p < nt * E) {
+                const float l = ((part[j][0] + part[j][1]) + part[j][2]) + part[j][3];
+                if (write_global) P.logits[(size_t)t0 * E + p] = l;
+                if (softmax) {
+                    s_val[p] = l;
+                    s_key[p] = orderable(l);
+                } else {
+                    const int e = p % E;
+                    const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
+                    s_val[p] = sg;
+                    s_key[p] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
+                }
+            }
         }
     }
     __syncthreads();
+#pragma unroll 2
     for (int seg = warp; seg < nt * nseg; seg += kWarps) {  // level 1: rank inside a 32-expert segment
         const int t = seg / nseg, sg = seg - t * nseg, e = sg * 32 + lane;
         const uint32_t my = (e < E) ? s_key[t * E + e] : 0u;
@@ -378,6 +389,7 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
         if (lr < Kc) cand[t * C + sg * Kc + lr] = ((unsigned long long)my << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)e);
     }
     __syncthreads();
+#pragma unroll 2
     for (int p = tid; p < nt * C; p += kThreads) {          // level 2: rank among the token's candidates
         const int t = p / C;
         const unsigned long long* ck = cand + t * C;
@@ -415,7 +427,7 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
             const int id = s_ids[t * K + lane];
             const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
             s_w[t * K + lane] = w;
-            atomicOr(&s_mask[id], 1ull << t);
+            if (build_mask) atomicOr(&s_mask[id], 1ull << t);
             if (write_global) { P.ids[t * K + lane] = id; P.wts[t * K + lane] = w; }
         }
     }
@@ -485,7 +497,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const unsigned par = tag & 1u;
     unsigned* e_cnt = P.e_cnt + par * E;                    // counters of this launch
     for (int e = cta * kThreads + tid; e < E; e += G * kThreads) P.e_cnt[(par ^ 1u) * E + e] = 0u;
-    if (cta == 0 && tid == 0) P.ctrl[kRouteCnt + (par ^ 1u)] = 0u;
+    if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
 
     constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
@@ -505,7 +517,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
     {
         const int items = ((E + 15) / 16) * ((T + 7) / 8);
-        while (ksplit < 16 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
+        while (ksplit < 4 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
     }
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
@@ -580,16 +592,38 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         MOE_STAMP(4);
     }
     __syncthreads();
-    const bool alive = (misc[2] != 0u);
+    bool alive = (misc[2] != 0u);
 
     // ------------------------------------------------------------------ top-k + routing metadata (every CTA)
     if (alive) {
         for (int i = tid; i < T * KBu; i += kThreads) s_xs[(i % KBu) * TS + i / KBu] = __ldcg(P.xs + i);   // transposed: [K block][token]
         // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
-        int chunk = (S * L.stage_bytes) / (4 * route_scratch_words(E, K));
-        chunk = chunk < kMaxTokens ? chunk : kMaxTokens;
-        for (int t0 = 0; t0 < T; t0 += chunk)
-            route_tokens(P, t0, min(chunk, T - t0), ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0);
+        if (T < 4) {
+            // few tokens: every CTA selects for all of them (no second grid-wide wait)
+            route_tokens(P, 0, T, ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0, true);
+        } else {
+            // many tokens: CTA t selects for token t and publishes ids and weights; everybody reads all of them
+            // after a second arrival counter (one more L2 round trip, but T times less selection work per CTA)
+            for (int t = cta; t < T; t += G)
+                route_tokens(P, t, 1, ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, true, false);
+            __syncthreads();
+            if (tid == 0) {
+                if (cta < T) red_release_add(P.ctrl + kRouteCnt2 + par, 1u);
+                const bool ok = wt.flag(P.ctrl + kRouteCnt2 + par, (unsigned)(T < G ? T : G), 12);
+                misc[2] = ok ? 1u : 0u;
+            }
+            __syncthreads();
+            alive = (misc[2] != 0u);
+            if (alive) {
+                for (int i = tid; i < T * K; i += kThreads) {
+                    const int id = __ldcg(P.ids + i);
+                    s_ids[i] = id;
+                    s_w[i] = __ldcg(P.wts + i);
+                    atomicOr(&s_mask[id], 1ull << (i / K));
+                }
+            }
+            __syncthreads();
+        }
         if (tid == 0) MOE_STAMP(6);
         if (warp == 0) {                                   // active-expert list in ascending expert order
             int base = 0;
