@@ -94,7 +94,7 @@ struct moe_plan {
         L.flags_end = o;
         L.stamps = o;   o += align_up((size_t)G * 16 * 8, 256);
         L.logits = o;   o += align_up((size_t)Tc * E * 4, 256);
-        L.lpart = o;    o += align_up((size_t)4 * Tc * E * 4, 256);
+        L.lpart = o;    o += align_up((size_t)8 * Tc * E * 4, 256);
         L.ids = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.wts = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.xs = o;       o += align_up((size_t)Tc * (H / 128) * 4, 256);

@@ -64,7 +64,7 @@ struct Params {
     __nv_bfloat16* out;
     unsigned* ctrl;
     float* logits;      // [T,E]   (diagnostics: summed router logits, written by CTA 0)
-    float* lpart;       // [<=4][T,E] router logits, one slice per K-split part
+    float* lpart;       // [<=8][T,E] router logits, one slice per K-split part
     int* ids;           // [T,K]
     float* wts;         // [T,K]
     uint8_t* xq;        // [64,H]
@@ -349,11 +349,11 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
     unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
     const bool softmax = (P.scoring == 0);
     for (int p0 = tid; p0 < nt * E; p0 += 2 * kThreads) {      // two elements per turn: all their loads in flight at once
-        float part[2][4];                                        // router logit = sum of the K-split parts, fixed order
+        float part[2][8];                                        // router logit = sum of the K-split parts, fixed order
 #pragma unroll
         for (int j = 0; j < 2; ++j)
 #pragma unroll
-            for (int kp = 0; kp < 4; ++kp) {
+            for (int kp = 0; kp < 8; ++kp) {
                 const int p = p0 + j * kThreads;
                 part[j][kp] = (p < nt * E && kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
             }
@@ -361,7 +361,7 @@ __device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, in
         for (int j = 0; j < 2; ++j) {
             const int p = p0 + j * kThreads;
             if (p < nt * E) {
-                const float l = ((part[j][0] + part[j][1]) + part[j][2]) + part[j][3];
+                const float l = (((part[j][0] + part[j][1]) + (part[j][2] + part[j][3])) + ((part[j][4] + part[j][5]) + (part[j][6] + part[j][7])));
                 if (write_global) P.logits[(size_t)t0 * E + p] = l;
                 if (softmax) {
                     s_val[p] = l;
@@ -517,7 +517,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
     {
         const int items = ((E + 15) / 16) * ((T + 7) / 8);
-        while (ksplit < 4 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
+        while (ksplit < 8 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
     }
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
