@@ -260,10 +260,14 @@ def main():
     uniq = []
     for l in range(L):
         d = layers[l]
-        dbg = plan.forward_debug(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
-        plan.sync_status()
-        uniq.append(int(torch.unique(dbg["ids"]).numel()))
-    ids0 = dbg["ids"].cpu().numpy() if L == 1 else None
+        ids_all = []
+        for lo in range(0, T, 64):               # the debug entry point takes at most 64 tokens per call
+            dbg = plan.forward_debug(d["hidden"][lo:lo + 64].contiguous(), d["Wr"], d["bias"], d["W13q"], d["W13s"],
+                                     d["W2q"], d["W2s"])
+            plan.sync_status()
+            ids_all.append(dbg["ids"])
+        ids_last = torch.cat(ids_all)
+        uniq.append(int(torch.unique(ids_last).numel()))
     bytes_per_step = float(np.mean([wl.algorithmic_bytes(shape, T, u) for u in uniq]))
     launches_per_step = -(-T // 64)
 
@@ -396,8 +400,7 @@ def main():
                            "d2h_bytes_per_step": 2 * T * shape.H, "steps": e2e["steps"]}
         if world == 1 and not args.no_cpu_baseline:
             d = layers[L - 1]
-            ids = dbg["ids"].cpu().numpy()
-            host = oracle_inputs(d, ids)
+            host = oracle_inputs(d, ids_last.cpu().numpy())
             us_cpu, reps, thr = time_oracle(shape, host)
             line["cpu_baseline"] = {"value": us_cpu, "unit": "us", "cores": thr, "kind": "oracle",
                                     "sample": f"{reps} full layer-steps of the same workload (T={T}), mean"}
