@@ -288,10 +288,11 @@ __device__ __forceinline__ int range_lo(int S, int c, int G, int q) { return (in
 
 // Split a projection's units across CTAs (split-K, partial sums exchanged through L2) or keep units whole?
 // Whole units cost no exchange but load the busiest CTA with ceil(units/G) units; take them when that surplus,
-// in KiB of weight tiles, stays below `slack_kib` (what an exchange costs in streaming time).
+// in KiB of weight tiles, stays below `slack_kib` (what an exchange costs in streaming time).  Measured: letting
+// the down projection of config 2 split at T=8 (surplus 26 KiB) is no faster than whole units.
 __device__ __forceinline__ int range_quantum(int units, int KB, int G, int kstep_kib, int slack_kib) {
     const int whole = ((units + G - 1) / G) * KB * kstep_kib;
-    const int split = (int)(((long long)units * KB * kstep_kib + G - 1) / G);
+    const int split = (units * KB * kstep_kib + G - 1) / G;
     return (whole - split <= slack_kib) ? KB : 1;
 }
 
@@ -968,10 +969,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             const float g = accg[n];
                             const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
                             accg[n] = a;
-                            float m = fabsf(a);
-#pragma unroll
-                            for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                            if (lane == 0) s_red[q * N + cb + n] = m;
+                            // |a| as an integer orders like the float: one warp-wide integer max instead of a shuffle tree
+                            const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a)));
+                            if (lane == 0) s_red[q * N + cb + n] = __uint_as_float(m);
                         }
                     }
                     epi_bar(kEpiThreads);
