@@ -870,17 +870,19 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     tc_fence_after();
                     if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
                     const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
+                    // all TMEM loads of this k-step first, one wait, free the buffer, then the arithmetic
+                    float dg[TCG], du[TCG];
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
-                        float dg[CH], du[CH];
-                        tmem_ld<CH>(tcol + cb + c, dg);
-                        if (up) tmem_ld<CH>(tcol + N + cb + c, du);
-                        tmem_ld_wait();
-                        if (c + CH == TCG) {                             // accumulator is in registers: free the buffer
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-                        }
+                        tmem_ld<CH>(tcol + cb + c, dg + c);
+                        if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
+                    }
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+#pragma unroll
+                    for (int c = 0; c < TCG; c += CH) {
                         float as[CH];
                         if constexpr (CH >= 4) {
 #pragma unroll
@@ -895,8 +897,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                         for (int jj = 0; jj < CH; ++jj) {
                             const int n = c + jj;
-                            accg[n] = fmaf(dg[jj], wsg * as[jj], accg[n]);
-                            if (up) accu[n] = fmaf(du[jj], wsu * as[jj], accu[n]);
+                            accg[n] = fmaf(dg[n], wsg * as[jj], accg[n]);
+                            if (up) accu[n] = fmaf(du[n], wsu * as[jj], accu[n]);
                         }
                     }
                     if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
