@@ -74,6 +74,7 @@ struct moe_plan {
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
     int split_slack_kib = 100;
+    int route_all_tokens = 16;
     int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
     int use_pdl = 1;                // programmatic dependent launch
     std::mutex mu;
@@ -194,6 +195,8 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.routed_scale = p->routed_scale;
     P.stages = stages;
     P.split_slack_kib = p->split_slack_kib;
+    P.route_all_tokens = p->route_all_tokens;
+    P.grid_magic = (1ull << 40) / (unsigned long long)p->sms + 1ull;
     P.timeout_ns = p->timeout_ns;
     P.hidden = static_cast<const __nv_bfloat16*>(hidden);
     P.Wr = static_cast<const __nv_bfloat16*>(Wr);
@@ -281,6 +284,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (const char* v = getenv("MOE_B200_STAGES")) p->stages_cap = atoi(v);
     if (const char* v = getenv("MOE_B200_PDL")) p->use_pdl = atoi(v) != 0;
     if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) p->split_slack_kib = atoi(v);
+    if (const char* v = getenv("MOE_B200_ROUTE_ALL")) p->route_all_tokens = atoi(v) < 0 ? 0 : (atoi(v) > 64 ? 64 : atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
@@ -395,6 +399,8 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     P.routed_scale = plan->routed_scale;
     P.stages = stages;
     P.split_slack_kib = plan->split_slack_kib;
+    P.route_all_tokens = plan->route_all_tokens;
+    P.grid_magic = (1ull << 40) / (unsigned long long)plan->sms + 1ull;
     P.timeout_ns = plan->timeout_ns;
     P.hidden = static_cast<const __nv_bfloat16*>(hidden_bf16);
     P.Wr = static_cast<const __nv_bfloat16*>(Wr_bf16);

@@ -55,6 +55,8 @@ struct Params {
     float routed_scale;
     int stages;
     int split_slack_kib;            // see range_quantum()
+    int route_all_tokens;           // up to this many tokens every CTA selects for all of them
+    unsigned long long grid_magic;  // floor(2^40 / grid) + 1: division by the grid size as a multiplication
     unsigned long long timeout_ns;
     const __nv_bfloat16* hidden;
     const __nv_bfloat16* Wr;
@@ -284,15 +286,26 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
 
 // per-phase split of a linear k-step list into contiguous per-CTA ranges
 // (q = 1: equal k-step counts, units may be split between neighbouring CTAs; q = K blocks per unit: whole units only)
-__device__ __forceinline__ int range_lo(int S, int c, int G, int q) { return (int)(((unsigned)(S / q) * (unsigned)c) / (unsigned)G) * q; }
+// (Sq = number of quanta in the list; the range of CTA c starts at quantum floor(Sq * c / G))
+// Integer divisions cost ~100 cycles each on one thread and the range arithmetic sits on the latency-critical path
+// between routing and the first weight request, so: division by the grid size is a multiplication by
+// magic = floor(2^40 / G) + 1 (exact while a * G < 2^40), small divisions go through a float reciprocal plus fix-up.
+__device__ __forceinline__ unsigned div_grid(unsigned a, unsigned long long magic) { return (unsigned)(((unsigned long long)a * magic) >> 40); }
+__device__ __forceinline__ int div_small(int a, int d) {          // 0 <= a < 2^22, d > 0
+    int q = (int)(__int2float_rz(a) * __frcp_rn(__int2float_rz(d)));
+    const int r = a - q * d;
+    q += (r >= d) - (r < 0);
+    return q;
+}
+__device__ __forceinline__ int range_lo(int Sq, int c, int q, unsigned long long magic) { return (int)div_grid((unsigned)Sq * (unsigned)c, magic) * q; }
 
 // Split a projection's units across CTAs (split-K, partial sums exchanged through L2) or keep units whole?
 // Whole units cost no exchange but load the busiest CTA with ceil(units/G) units; take them when that surplus,
 // in KiB of weight tiles, stays below `slack_kib` (what an exchange costs in streaming time).  Measured: letting
 // the down projection of config 2 split at T=8 (surplus 26 KiB) is no faster than whole units.
-__device__ __forceinline__ int range_quantum(int units, int KB, int G, int kstep_kib, int slack_kib) {
-    const int whole = ((units + G - 1) / G) * KB * kstep_kib;
-    const int split = (units * KB * kstep_kib + G - 1) / G;
+__device__ __forceinline__ int range_quantum(int units, int KB, int G, int kstep_kib, int slack_kib, unsigned long long magic) {
+    const int whole = (int)div_grid((unsigned)(units + G - 1), magic) * KB * kstep_kib;
+    const int split = (int)div_grid((unsigned)(units * KB * kstep_kib + G - 1), magic);
     return (whole - split <= slack_kib) ? KB : 1;
 }
 
@@ -301,9 +314,9 @@ struct Walk {
     int kb, mb, u, e, KB, MB;
     __device__ __forceinline__ void init(int s, int KB_, int MB_, const int* act) {
         KB = KB_; MB = MB_;
-        const int unit = s / KB;
+        const int unit = div_small(s, KB);
         kb = s - unit * KB;
-        u = unit / MB;
+        u = div_small(unit, MB);
         mb = unit - u * MB;
         e = act[u];
     }
@@ -327,112 +340,96 @@ __device__ __forceinline__ uint32_t orderable(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Scores and top-k for a few tokens at a time by the whole CTA (Section 4.1 routing policies): softmax over all
-// experts or sigmoid plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots
-// are in (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
-// Selection is by rank in two levels: a warp ranks the 32 experts of one segment against each other by shuffles
-// and keeps the best min(K,32) as candidates; then every candidate counts the candidates of its token that beat
-// it (larger key, or equal key and lower index) and takes that slot if the count is below K.
+// Scores and top-k of one token by one warp (Section 4.1 routing policies): softmax over all experts or sigmoid
+// plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots are in (key
+// descending, index ascending) order; weights are optionally renormalised over the selected experts.
+// Lane l holds experts l, l+32, ... (NPER of them) in registers.  Selection is K rounds of: warp-wide maximum of
+// the orderable keys (one redux), warp-wide minimum of the indices holding it (one redux), removal of the winner;
+// lane j keeps slot j.  No shared memory and no CTA barrier until the result is written.
 // The softmax key is the logit itself; its normaliser is only summed when the weights are not renormalised
 // (it cancels otherwise), with the largest logit -- slot 0 -- as the shift.
-// Shared-memory scratch per token: E keys, E scores, ceil(E/32) * min(K,32) 64-bit candidates.
-__device__ __forceinline__ int route_scratch_words(int E, int K) { return 2 * E + 2 * ((E + 31) / 32) * (K < 32 ? K : 32); }
-
-__device__ __forceinline__ void route_tokens(const Params& P, int t0, int nt, int ksplit, int tid, uint32_t* scratch,
-                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global,
-                                             bool build_mask) {
-    const int E = P.E, K = P.K, warp = tid >> 5, lane = tid & 31;
-    const int kThreads = blockDim.x, kWarps = blockDim.x >> 5;
-    const int nseg = (E + 31) / 32, Kc = K < 32 ? K : 32, C = nseg * Kc;
-    uint32_t* s_key = scratch;
-    float* s_val = reinterpret_cast<float*>(scratch + nt * E);
-    // candidates are packed as (key << 32 | ~index): "a beats b" is then one 64-bit compare
-    unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch + 2 * nt * E);
+template <int NPER>
+__device__ __forceinline__ void route_token_warp(const Params& P, int t, int ksplit, int lane, int* s_ids, float* s_w,
+                                                 unsigned long long* s_mask, bool write_global, bool build_mask) {
+    const int E = P.E, K = P.K;
     const bool softmax = (P.scoring == 0);
-    for (int p0 = tid; p0 < nt * E; p0 += 2 * kThreads) {      // two elements per turn: all their loads in flight at once
-        float part[2][8];                                        // router logit = sum of the K-split parts, fixed order
+    constexpr int UNR = 32 / NPER;                             // K-split parts loaded per turn: 32 loads in flight
+    float val[NPER];
+    uint32_t key[NPER];
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
+    for (int i = 0; i < NPER; ++i) val[i] = 0.f;
+    for (int kp0 = 0; kp0 < ksplit; kp0 += UNR) {              // router logit = sum of the K-split parts in part order
+        float part[UNR][NPER];
 #pragma unroll
-            for (int kp = 0; kp < 8; ++kp) {
-                const int p = p0 + j * kThreads;
-                part[j][kp] = (p < nt * E && kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
+        for (int j = 0; j < UNR; ++j)
+#pragma unroll
+            for (int i = 0; i < NPER; ++i) {
+                const int e = i * 32 + lane;
+                part[j][i] = (kp0 + j < ksplit && e < E) ? __ldcg(P.lpart + ((size_t)(kp0 + j) * P.T + t) * E + e) : 0.f;
             }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int p = p0 + j * kThreads;
-            if (p < nt * E) {
-                const float l = (((part[j][0] + part[j][1]) + (part[j][2] + part[j][3])) + ((part[j][4] + part[j][5]) + (part[j][6] + part[j][7])));
-                if (write_global) P.logits[(size_t)t0 * E + p] = l;
-                if (softmax) {
-                    s_val[p] = l;
-                    s_key[p] = orderable(l);
-                } else {
-                    const int e = p % E;
-                    const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
-                    s_val[p] = sg;
-                    s_key[p] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
-                }
+        for (int j = 0; j < UNR; ++j)
+#pragma unroll
+            for (int i = 0; i < NPER; ++i) val[i] += part[j][i];
+    }
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) {
+        const int e = i * 32 + lane;
+        key[i] = 0u;                                           // below every real key
+        if (e < E) {
+            const float l = val[i];
+            if (write_global) P.logits[(size_t)t * E + e] = l;
+            if (softmax) {
+                key[i] = orderable(l);
+            } else {
+                const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
+                val[i] = sg;
+                key[i] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
             }
         }
     }
-    __syncthreads();
-#pragma unroll 2
-    for (int seg = warp; seg < nt * nseg; seg += kWarps) {  // level 1: rank inside a 32-expert segment
-        const int t = seg / nseg, sg = seg - t * nseg, e = sg * 32 + lane;
-        const uint32_t my = (e < E) ? s_key[t * E + e] : 0u;
-        int lr = 0;
+    int my_id = 0;
+    float v = 0.f;
+    for (int j = 0; j < K; ++j) {
+        uint32_t m = key[0];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const uint32_t ko = __shfl_sync(0xffffffffu, my, i);
-            lr += (int)(ko > my) | ((int)(ko == my) & (int)(i < lane));
+        for (int i = 1; i < NPER; ++i) m = max(m, key[i]);
+        const uint32_t wm = __reduce_max_sync(0xffffffffu, m);
+        int cand = 0x7fffffff;
+#pragma unroll
+        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 + lane : cand;
+        const int we = __reduce_min_sync(0xffffffffu, cand);
+        float wv = 0.f;
+#pragma unroll
+        for (int i = 0; i < NPER; ++i) {
+            if (i == (we >> 5)) wv = val[i];
+            if (i * 32 + lane == we) key[i] = 0u;
         }
-        if (lr < Kc) cand[t * C + sg * Kc + lr] = ((unsigned long long)my << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)e);
+        wv = __shfl_sync(0xffffffffu, wv, we & 31);
+        if (lane == j) { my_id = we; v = wv; }
     }
-    __syncthreads();
-#pragma unroll 2
-    for (int p = tid; p < nt * C; p += kThreads) {          // level 2: rank among the token's candidates
-        const int t = p / C;
-        const unsigned long long* ck = cand + t * C;
-        const unsigned long long my = cand[p];
-        const int me = (int)(0xFFFFFFFFu - (uint32_t)my);
-        int rank = 0;
-        for (int o0 = 0; o0 < C; o0 += 8) {
-            unsigned long long v[8];
+    float total = 1.0f;
+    if (softmax) {
+        const float mx = __shfl_sync(0xffffffffu, v, 0);        // slot 0 holds the largest logit
+        v = (lane < K) ? expf(v - mx) : 0.f;
+        if (!P.renorm) {
+            total = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = (o0 + j < C) ? ck[o0 + j] : 0ull;
+            for (int i = 0; i < NPER; ++i) if (i * 32 + lane < E) total += expf(val[i] - mx);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) rank += (int)(v[j] > my);
-        }
-        if (rank < K && me < E) { s_ids[(t0 + t) * K + rank] = me; s_w[(t0 + t) * K + rank] = s_val[t * E + me]; }
-    }
-    __syncthreads();
-    for (int tl = warp; tl < nt; tl += kWarps) {           // weights of the selected experts, one warp per token
-        const int t = t0 + tl;
-        float v = (lane < K) ? s_w[t * K + lane] : 0.f;
-        float total = 1.0f;
-        if (softmax) {
-            const float mx = __shfl_sync(0xffffffffu, v, 0);          // slot 0 holds the largest logit
-            v = (lane < K) ? expf(v - mx) : 0.f;
-            if (!P.renorm) {
-                total = 0.f;
-                for (int e = lane; e < E; e += 32) total += expf(s_val[tl * E + e] - mx);
-#pragma unroll
-                for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-            }
-        }
-        float vsum = v;
-#pragma unroll
-        for (int o = 16; o; o >>= 1) vsum += __shfl_xor_sync(0xffffffffu, vsum, o);
-        if (lane < K) {
-            const int id = s_ids[t * K + lane];
-            const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
-            s_w[t * K + lane] = w;
-            if (build_mask) atomicOr(&s_mask[id], 1ull << t);
-            if (write_global) { P.ids[t * K + lane] = id; P.wts[t * K + lane] = w; }
+            for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
         }
     }
-    __syncthreads();
+    float vsum = v;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) vsum += __shfl_xor_sync(0xffffffffu, vsum, o);
+    if (lane < K) {
+        const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
+        s_ids[t * K + lane] = my_id;
+        s_w[t * K + lane] = w;
+        if (build_mask) atomicOr(&s_mask[my_id], 1ull << t);
+        if (write_global) { P.ids[t * K + lane] = my_id; P.wts[t * K + lane] = w; }
+    }
 }
 
 // quantise 4 floats with scale s into 4 E4M3 bytes (memory order x0..x3)
@@ -490,16 +487,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     // do not touch any global memory before the previous launch has completed and flushed (both are no-ops when the
     // launch was not made with the programmatic-serialization attribute).
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    Waiter wt;
-    wt.init(P.ctrl, P.timeout_ns);
-    const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
-    if (tid == 0) MOE_STAMP(0);
-    const unsigned par = tag & 1u;
-    unsigned* e_cnt = P.e_cnt + par * E;                    // counters of this launch
-    for (int e = cta * kThreads + tid; e < E; e += G * kThreads) P.e_cnt[(par ^ 1u) * E + e] = 0u;
-    if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
-
+    // Set-up that touches only this CTA's shared and tensor memory runs before the wait on the previous launch.
     constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
@@ -512,6 +500,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
     for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    Waiter wt;
+    wt.init(P.ctrl, P.timeout_ns);
+    const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
+    if (tid == 0) MOE_STAMP(0);
+    const unsigned par = tag & 1u;
+    unsigned* e_cnt = P.e_cnt + par * E;                    // counters of this launch
+    for (int e = cta * kThreads + tid; e < E; e += G * kThreads) P.e_cnt[(par ^ 1u) * E + e] = 0u;
+    if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
     // ------------------------------------------------------------------ phase R: quantise + logits
@@ -599,18 +596,22 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (alive) {
         for (int i = tid; i < T * KBu; i += kThreads) s_xs[(i % KBu) * TS + i / KBu] = __ldcg(P.xs + i);   // transposed: [K block][token]
         // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
-        if (T < 4) {
-            // few tokens: every CTA selects for all of them (no second grid-wide wait)
-            route_tokens(P, 0, T, ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, cta == 0, true);
-        } else {
-            // many tokens: CTA t selects for token t and publishes ids and weights; everybody reads all of them
-            // after a second arrival counter (one more L2 round trip, but T times less selection work per CTA)
-            for (int t = cta; t < T; t += G)
-                route_tokens(P, t, 1, ksplit, tid, reinterpret_cast<uint32_t*>(smem), s_ids, s_w, s_mask, true, false);
-            __syncthreads();
+        // few tokens: every CTA selects for all of them, one warp per token (no second grid-wide wait);
+        // many tokens: the grid's warps share the tokens, publish ids and weights, and everybody reads all of them
+        // after a second arrival counter (two more L2 round trips, but one selection per warp)
+        const bool route_all = (T <= P.route_all_tokens);
+        const int n_route_ctas = min(G, (T + kWarps - 1) / kWarps);
+        for (int t = route_all ? warp : cta * kWarps + warp; t < T; t += route_all ? kWarps : G * kWarps) {
+            const bool wg = route_all ? (cta == 0) : true;
+            if (E <= 128) route_token_warp<4>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
+            else if (E <= 256) route_token_warp<8>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
+            else route_token_warp<16>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
+        }
+        __syncthreads();
+        if (!route_all) {
             if (tid == 0) {
-                if (cta < T) red_release_add(P.ctrl + kRouteCnt2 + par, 1u);
-                const bool ok = wt.flag(P.ctrl + kRouteCnt2 + par, (unsigned)(T < G ? T : G), 12);
+                if (cta < n_route_ctas) red_release_add(P.ctrl + kRouteCnt2 + par, 1u);
+                const bool ok = wt.flag(P.ctrl + kRouteCnt2 + par, (unsigned)n_route_ctas, 12);
                 misc[2] = ok ? 1u : 0u;
             }
             __syncthreads();
@@ -620,7 +621,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     const int id = __ldcg(P.ids + i);
                     s_ids[i] = id;
                     s_w[i] = __ldcg(P.wts + i);
-                    atomicOr(&s_mask[id], 1ull << (i / K));
+                    atomicOr(&s_mask[id], 1ull << div_small(i, K));
                 }
             }
             __syncthreads();
@@ -642,9 +643,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int U = alive ? (int)misc[1] : 0;
     if (tid == 0) MOE_STAMP(7);
     const int S_up = U * IB * KBu, S_dn = U * HB * KBd;     // k-steps of the two projections (host checks the range)
-    const int q_up = range_quantum(U * IB, KBu, G, 32, P.split_slack_kib), q_dn = range_quantum(U * HB, KBd, G, 16, P.split_slack_kib);
-    const int up_lo = range_lo(S_up, cta, G, q_up), up_hi = range_lo(S_up, cta + 1, G, q_up);
-    const int dn_lo = range_lo(S_dn, cta, G, q_dn), dn_hi = range_lo(S_dn, cta + 1, G, q_dn);
+    const unsigned long long gm = P.grid_magic;
+    const int q_up = range_quantum(U * IB, KBu, G, 32, P.split_slack_kib, gm), q_dn = range_quantum(U * HB, KBd, G, 16, P.split_slack_kib, gm);
+    const int Sq_up = (q_up == 1) ? S_up : U * IB, Sq_dn = (q_dn == 1) ? S_dn : U * HB;      // quanta per list
+    const int up_lo = range_lo(Sq_up, cta, q_up, gm), up_hi = range_lo(Sq_up, cta + 1, q_up, gm);
+    const int dn_lo = range_lo(Sq_dn, cta, q_dn, gm), dn_hi = range_lo(Sq_dn, cta + 1, q_dn, gm);
 
     // ------------------------------------------------------------------ role: TMA producers
     // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.  A stage = one
@@ -811,7 +814,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const bool up = (phase == 0);
             const int lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
             const int KB = up ? KBu : KBd, MB = up ? IB : HB;  // K blocks per unit, row blocks per expert
-            const int S_all = up ? S_up : S_dn, q_all = up ? q_up : q_dn;
+            const int Sq_all = up ? Sq_up : Sq_dn, q_all = up ? q_up : q_dn;
             float* part = up ? P.part_up : P.part_dn;
             unsigned* pflag = up ? P.pu_flag : P.pd_flag;
             const int pcols = up ? 2 * N : N;
@@ -825,7 +828,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             auto fetch_scales = [&](int sidx, float& g, float& u2) {
                 g = 0.f; u2 = 0.f;
                 if (sidx < hi) {
-                    const int unit = sidx / KB, kb = sidx - unit * KB, uu = unit / MB, mb = unit - uu * MB, e = s_act[uu];
+                    const int unit = div_small(sidx, KB), kb = sidx - unit * KB, uu = div_small(unit, MB), mb = unit - uu * MB, e = s_act[uu];
                     if (up) {
                         g = __ldg(P.W13s + ((size_t)e * 2 * IB + mb) * KBu + kb);
                         u2 = __ldg(P.W13s + ((size_t)e * 2 * IB + IB + mb) * KBu + kb);
@@ -945,15 +948,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     for (int base = cta + 1; base < G; base += kEpiThreads) {
                         const int c = base + etid;
                         if (c < G) {
-                            const int clo = range_lo(S_all, c, G, q_all), chi = range_lo(S_all, c + 1, G, q_all);
+                            const int clo = range_lo(Sq_all, c, q_all, gm), chi = range_lo(Sq_all, c + 1, q_all, gm);
                             if (clo < uend && chi > clo) got = wt.flag(pflag + c, tag, 6) && got;
                         }
-                        if (range_lo(S_all, min(base + kEpiThreads, G), G, q_all) >= uend) break;
+                        if (range_lo(Sq_all, min(base + kEpiThreads, G), q_all, gm) >= uend) break;
                     }
-                    while (c_end < G && range_lo(S_all, c_end, G, q_all) < uend) ++c_end;
+                    while (c_end < G && range_lo(Sq_all, c_end, q_all, gm) < uend) ++c_end;
                     if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
                     for (int c = cta + 1; c < c_end; ++c) {
-                        if (range_lo(S_all, c + 1, G, q_all) == range_lo(S_all, c, G, q_all)) continue;
+                        if (range_lo(Sq_all, c + 1, q_all, gm) == range_lo(Sq_all, c, q_all, gm)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TCG; ++n)
@@ -1018,8 +1021,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             bool got = true;
             if (mine && gtid < K) {
                 // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
-                const unsigned x = (unsigned)((s_uidx[s_ids[t * K + gtid]] * HB + hb) * KBd / q_dn);
-                const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)(S_dn / q_dn);
+                const unsigned unit = (unsigned)(s_uidx[s_ids[t * K + gtid]] * HB + hb);
+                const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
+                const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
                 got = wt.flag(P.dn_flag + owner, tag, 7);
             }
             if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
