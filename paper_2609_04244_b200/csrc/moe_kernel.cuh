@@ -340,56 +340,58 @@ __device__ __forceinline__ uint32_t orderable(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Scores and top-k of one token by one warp (Section 4.1 routing policies): softmax over all experts or sigmoid
-// plus selection bias; the K largest keys win, equal keys go to the lowest expert index; slots are in (key
-// descending, index ascending) order; weights are optionally renormalised over the selected experts.
-// Lane l holds experts l, l+32, ... (NPER of them) in registers.  Selection is K rounds of: warp-wide maximum of
-// the orderable keys (one redux), warp-wide minimum of the indices holding it (one redux), removal of the winner;
-// lane j keeps slot j.  No shared memory and no CTA barrier until the result is written.
-// The softmax key is the logit itself; its normaliser is only summed when the weights are not renormalised
-// (it cancels otherwise), with the largest logit -- slot 0 -- as the shift.
-template <int NPER>
-__device__ __forceinline__ void route_token_warp(const Params& P, int t, int ksplit, int lane, int* s_ids, float* s_w,
-                                                 unsigned long long* s_mask, bool write_global, bool build_mask) {
-    const int E = P.E, K = P.K;
+// Routing (Section 4.1 policies) in two steps.
+// (1) route_scores: the whole CTA turns the router logits of a few tokens into selection keys and score values in
+//     shared memory: softmax over all experts (key = the logit itself) or sigmoid plus selection bias.
+// (2) route_select: one warp per token picks the K largest keys; equal keys go to the lowest expert index; slots
+//     are in (key descending, index ascending) order; weights are optionally renormalised over the selected experts.
+//     Lane l holds experts l, l+32, ... (NPER of them) in registers.  Selection is K rounds of: warp-wide maximum of
+//     the orderable keys (one redux), warp-wide minimum of the indices holding it (one redux), removal of the winner;
+//     lane j keeps slot j.  The softmax normaliser is only summed when the weights are not renormalised (it cancels
+//     otherwise), with the largest logit -- slot 0 -- as the shift.
+__device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, int ksplit, int tid, int nthreads,
+                                             uint32_t* s_key, float* s_val, bool write_global) {
+    const int E = P.E;
     const bool softmax = (P.scoring == 0);
-    constexpr int UNR = 32 / NPER;                             // K-split parts loaded per turn: 32 loads in flight
-    float val[NPER];
-    uint32_t key[NPER];
+    for (int p0 = tid; p0 < nt * E; p0 += 2 * nthreads) {      // two elements per turn: all their loads in flight at once
+        float part[2][8];                                        // router logit = sum of the K-split parts, fixed order
+        float bias[2];
 #pragma unroll
-    for (int i = 0; i < NPER; ++i) val[i] = 0.f;
-    for (int kp0 = 0; kp0 < ksplit; kp0 += UNR) {              // router logit = sum of the K-split parts in part order
-        float part[UNR][NPER];
+        for (int j = 0; j < 2; ++j) {
+            const int p = p0 + j * nthreads;
 #pragma unroll
-        for (int j = 0; j < UNR; ++j)
+            for (int kp = 0; kp < 8; ++kp)
+                part[j][kp] = (p < nt * E && kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
+            bias[j] = (!softmax && P.bias && p < nt * E) ? __ldg(P.bias + (p - div_small(p, E) * E)) : 0.f;
+        }
 #pragma unroll
-            for (int i = 0; i < NPER; ++i) {
-                const int e = i * 32 + lane;
-                part[j][i] = (kp0 + j < ksplit && e < E) ? __ldcg(P.lpart + ((size_t)(kp0 + j) * P.T + t) * E + e) : 0.f;
-            }
-#pragma unroll
-        for (int j = 0; j < UNR; ++j)
-#pragma unroll
-            for (int i = 0; i < NPER; ++i) val[i] += part[j][i];
-    }
-#pragma unroll
-    for (int i = 0; i < NPER; ++i) {
-        const int e = i * 32 + lane;
-        key[i] = 0u;                                           // below every real key
-        if (e < E) {
-            const float l = val[i];
-            if (write_global) P.logits[(size_t)t * E + e] = l;
-            if (softmax) {
-                key[i] = orderable(l);
-            } else {
-                const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
-                val[i] = sg;
-                key[i] = orderable(sg + (P.bias ? __ldg(P.bias + e) : 0.f));
+        for (int j = 0; j < 2; ++j) {
+            const int p = p0 + j * nthreads;
+            if (p < nt * E) {
+                const float l = (((part[j][0] + part[j][1]) + (part[j][2] + part[j][3])) + ((part[j][4] + part[j][5]) + (part[j][6] + part[j][7])));
+                if (write_global) P.logits[(size_t)t0 * E + p] = l;
+                if (softmax) {
+                    s_val[p] = l;
+                    s_key[p] = orderable(l);
+                } else {
+                    const float sg = __fdiv_rn(1.0f, 1.0f + expf(-l));
+                    s_val[p] = sg;
+                    s_key[p] = orderable(sg + bias[j]);
+                }
             }
         }
     }
+}
+
+template <int NPER>
+__device__ __forceinline__ void route_select(const Params& P, int t, int lane, const uint32_t* s_key, const float* s_val,
+                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global, bool build_mask) {
+    const int E = P.E, K = P.K;
+    const bool softmax = (P.scoring == 0);
+    uint32_t key[NPER];
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) key[i] = (i * 32 + lane < E) ? s_key[i * 32 + lane] : 0u;    // 0 is below every real key
     int my_id = 0;
-    float v = 0.f;
     for (int j = 0; j < K; ++j) {
         uint32_t m = key[0];
 #pragma unroll
@@ -397,25 +399,21 @@ __device__ __forceinline__ void route_token_warp(const Params& P, int t, int ksp
         const uint32_t wm = __reduce_max_sync(0xffffffffu, m);
         int cand = 0x7fffffff;
 #pragma unroll
-        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 + lane : cand;
-        const int we = __reduce_min_sync(0xffffffffu, cand);
-        float wv = 0.f;
+        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 : cand;
+        const int we = __reduce_min_sync(0xffffffffu, cand == 0x7fffffff ? cand : cand + lane);
+        const int mine = we - lane;                            // i * 32 if this lane holds the winner
 #pragma unroll
-        for (int i = 0; i < NPER; ++i) {
-            if (i == (we >> 5)) wv = val[i];
-            if (i * 32 + lane == we) key[i] = 0u;
-        }
-        wv = __shfl_sync(0xffffffffu, wv, we & 31);
-        if (lane == j) { my_id = we; v = wv; }
+        for (int i = 0; i < NPER; ++i) key[i] = (mine == i * 32) ? 0u : key[i];
+        if (lane == j) my_id = we;
     }
+    float v = (lane < K) ? s_val[my_id] : 0.f;
     float total = 1.0f;
     if (softmax) {
         const float mx = __shfl_sync(0xffffffffu, v, 0);        // slot 0 holds the largest logit
         v = (lane < K) ? expf(v - mx) : 0.f;
         if (!P.renorm) {
             total = 0.f;
-#pragma unroll
-            for (int i = 0; i < NPER; ++i) if (i * 32 + lane < E) total += expf(val[i] - mx);
+            for (int e = lane; e < E; e += 32) total += expf(s_val[e] - mx);
 #pragma unroll
             for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
         }
@@ -500,6 +498,25 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
     for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
+    int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
+    {
+        const int items = ((E + 15) / 16) * ((T + 7) / 8);
+        while (ksplit < 8 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
+        // Router weights of this CTA's first tile: ask L2 for them now (a prefetch reads nothing into the SM, and L2
+        // is the point of coherence, so this is safe ahead of the wait whatever the previous launch wrote).
+        const int nTB = (T + 7) / 8;
+        if (cta < ((E + 15) / 16) * nTB * ksplit) {
+            const int item = cta / ksplit, kp = cta - item * ksplit, eb = item / nTB;
+            const int kpart_len = H / ksplit;
+            const int kper = (kpart_len / 16 + kWarps - 1) / kWarps * 16;
+            const int k_lo = kp * kpart_len + warp * kper, k_hi = min((kp + 1) * kpart_len, k_lo + kper);
+            const int lines = (k_hi - k_lo + 63) / 64;                        // 128-byte lines per row
+            for (int idx = lane; idx < 16 * lines; idx += 32) {
+                const int r = eb * 16 + (idx & 15);
+                if (r < E) prefetch_l2(P.Wr + (size_t)r * H + k_lo + (idx >> 4) * 64);
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     Waiter wt;
     wt.init(P.ctrl, P.timeout_ns);
@@ -512,11 +529,6 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
     // ------------------------------------------------------------------ phase R: quantise + logits
-    int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
-    {
-        const int items = ((E + 15) / 16) * ((T + 7) / 8);
-        while (ksplit < 8 && items * ksplit * 2 <= G && H % (32 * ksplit) == 0 && H / (2 * ksplit) >= 128) ksplit *= 2;
-    }
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
         const int groups = T * KBu;
@@ -594,18 +606,26 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     // ------------------------------------------------------------------ top-k + routing metadata (every CTA)
     if (alive) {
-        for (int i = tid; i < T * KBu; i += kThreads) s_xs[(i % KBu) * TS + i / KBu] = __ldcg(P.xs + i);   // transposed: [K block][token]
-        // the weight ring is idle until the roles start: its first bytes serve as scratch for the routing
-        // few tokens: every CTA selects for all of them, one warp per token (no second grid-wide wait);
-        // many tokens: the grid's warps share the tokens, publish ids and weights, and everybody reads all of them
-        // after a second arrival counter (two more L2 round trips, but one selection per warp)
-        const bool route_all = (T <= P.route_all_tokens);
+        // input scales, transposed to [K block][token]: the first load is issued here and consumed after the routing loads
+        const float xs0 = (tid < T * KBu) ? __ldcg(P.xs + tid) : 0.f;
+        // few tokens: every CTA selects for all of them (no second grid-wide wait); many tokens: CTAs share the
+        // tokens (one warp's worth each), publish ids and weights, and everybody reads all of them after a second
+        // arrival counter (two more L2 round trips).  The idle weight ring holds the keys and score values.
+        const bool route_all = (T <= P.route_all_tokens) && (T * E <= 8192);
         const int n_route_ctas = min(G, (T + kWarps - 1) / kWarps);
-        for (int t = route_all ? warp : cta * kWarps + warp; t < T; t += route_all ? kWarps : G * kWarps) {
-            const bool wg = route_all ? (cta == 0) : true;
-            if (E <= 128) route_token_warp<4>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
-            else if (E <= 256) route_token_warp<8>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
-            else route_token_warp<16>(P, t, ksplit, lane, s_ids, s_w, s_mask, wg, route_all);
+        const int rt0 = route_all ? 0 : min(T, cta * kWarps), rnt = route_all ? T : min(T - rt0, kWarps);
+        uint32_t* s_key = reinterpret_cast<uint32_t*>(smem);
+        float* s_val = reinterpret_cast<float*>(smem) + rnt * E;
+        const bool wg = route_all ? (cta == 0) : true;
+        route_scores(P, rt0, rnt, ksplit, tid, kThreads, s_key, s_val, wg);
+        if (tid < T * KBu) { const int tt = div_small(tid, KBu); s_xs[(tid - tt * KBu) * TS + tt] = xs0; }
+        for (int i = tid + kThreads; i < T * KBu; i += kThreads) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
+        __syncthreads();
+        for (int tl = warp; tl < rnt; tl += kWarps) {
+            const int t = rt0 + tl;
+            if (E <= 128) route_select<4>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
+            else if (E <= 256) route_select<8>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
+            else route_select<16>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
         }
         __syncthreads();
         if (!route_all) {
