@@ -532,7 +532,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
         const int groups = T * KBu;
-        for (int p = cta * kWarps + warp; p < groups; p += G * kWarps) {
+        for (int p = (G - 1 - cta) * kWarps + warp; p < groups; p += G * kWarps) {   // from the last CTA down: the first ones have router tiles
             const int t = p / KBu, g = p % KBu;
             const uint2 raw = *reinterpret_cast<const uint2*>(P.hidden + (size_t)t * H + g * kBlock + lane * 4);
             const float x0 = __uint_as_float(raw.x << 16), x1 = __uint_as_float(raw.x & 0xFFFF0000u);
