@@ -80,15 +80,19 @@ struct moe_plan {
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
-    int n_hw(int T) const { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
+    // More than 8 tokens under sparse routing (on average at most 8 tokens per expert): the kernel compacts the tokens
+    // of each expert into the 16 MMA columns; denser routing takes all tokens as columns (N = 32 or 64).
+    bool compact(int T) const { return T > 8 && (long long)T * K <= 8ll * E; }
+    int n_hw(int T) const { return (T <= 8 || compact(T)) ? 16 : (T <= 32 ? 32 : 64); }
+    int nr(int T) const { return compact(T) ? ((T + 15) & ~15) : n_hw(T); }     // token rows per expert in hq / hs
     int cap(int T) const { return T < moe::kMaxTokens ? T : moe::kMaxTokens; }
 
     WsLayout layout(int T_max) const {
-        const int Tc = cap(T_max), N = n_hw(Tc), G = sms;
+        const int Tc = cap(T_max), N = n_hw(Tc), NR = nr(Tc), G = sms;
         WsLayout L;
         size_t o = 0;
         L.ctrl = o;     o += moe::kCtrlWords * 4;
-        L.e_cnt = o;    o += align_up((size_t)2 * E * 4, 256);
+        L.e_cnt = o;    o += align_up((size_t)2 * 4 * E * 4, 256);
         L.dn_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
@@ -100,8 +104,8 @@ struct moe_plan {
         L.wts = o;      o += align_up((size_t)Tc * K * 4, 256);
         L.xs = o;       o += align_up((size_t)Tc * (H / 128) * 4, 256);
         L.xq = o;       o += align_up((size_t)moe::kMaxTokens * H, 1024);
-        L.hq = o;       o += align_up((size_t)E * N * I, 1024);
-        L.hs = o;       o += align_up((size_t)E * N * (I / 128) * 4, 256);
+        L.hq = o;       o += align_up((size_t)E * NR * I, 1024);
+        L.hs = o;       o += align_up((size_t)E * NR * (I / 128) * 4, 256);
         L.part_up = o;  o += align_up((size_t)G * 2 * N * 128 * 4, 256);
         L.part_dn = o;  o += align_up((size_t)G * N * 128 * 4, 256);
         L.y = o;        o += align_up((size_t)Tc * K * H * 4, 256);
@@ -113,7 +117,7 @@ struct moe_plan {
 
     int stages_for(int N, int T) const {
         for (int s = (stages_cap > 0 && stages_cap < moe::kMaxStages) ? stages_cap : moe::kMaxStages; s >= 2; --s) {
-            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s);
+            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s, compact(T));
             if (L.total + 1024 <= smem_optin) return s;
         }
         return 0;
@@ -172,30 +176,16 @@ bool resident(int smem_optin, int smem_bytes) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
-                  const float* W13s, const void* W2, const float* W2s, void* out, void* ws, size_t ws_bytes,
-                  cudaStream_t stream) {
-    const int N = p->n_hw(T);
-    const WsLayout L = p->layout(T);
-    if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
-    const int stages = p->stages_for(N, T);
-    if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages);
-    uint8_t* w = static_cast<uint8_t*>(ws);
-
-    CUtensorMap m13, m2, mx, mh;
-    if (!p->get_map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) ||
-        !p->get_map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
-        !p->get_map(&mx, w + L.xq, moe::kMaxTokens, p->H, N) ||
-        !p->get_map(&mh, w + L.hq, (uint64_t)p->E * N, p->I, N))
-        return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-
+// Kernel parameters for a step of T tokens on workspace `w` laid out as L.
+moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uint8_t* w, const void* hidden, const void* Wr,
+                        const float* bias, const float* W13s, const float* W2s, void* out) {
     moe::Params P;
     P.T = T; P.H = p->H; P.E = p->E; P.I = p->I; P.K = p->K; P.scoring = p->scoring; P.renorm = p->renorm;
     P.routed_scale = p->routed_scale;
     P.stages = stages;
     P.split_slack_kib = p->split_slack_kib;
     P.route_all_tokens = p->route_all_tokens;
+    P.nr = p->nr(T);
     P.grid_magic = (1ull << 40) / (unsigned long long)p->sms + 1ull;
     P.timeout_ns = p->timeout_ns;
     P.hidden = static_cast<const __nv_bfloat16*>(hidden);
@@ -220,15 +210,40 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
     P.y = reinterpret_cast<float*>(w + L.y);
     P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
+    return P;
+}
 
-    const int smem_bytes = SL.total + 1024;
+// Pick the kernel variant for T tokens: (MMA N, token columns read by the accumulator warps).
+int dispatch(Plan* p, int T, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx,
+             const CUtensorMap& mh, const moe::Params& P, int smem_bytes, cudaStream_t stream) {
     if (T == 1) return launch<16, 1>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T == 2) return launch<16, 2>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (T <= 16) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (p->compact(T)) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T <= 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+}
+
+int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
+                  const float* W13s, const void* W2, const float* W2s, void* out, void* ws, size_t ws_bytes,
+                  cudaStream_t stream) {
+    const int N = p->n_hw(T);
+    const WsLayout L = p->layout(T);
+    if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
+    const int stages = p->stages_for(N, T);
+    if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
+    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages, p->compact(T));
+    uint8_t* w = static_cast<uint8_t*>(ws);
+
+    CUtensorMap m13, m2, mx, mh;
+    if (!p->get_map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) ||
+        !p->get_map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
+        !p->get_map(&mx, w + L.xq, moe::kMaxTokens, p->H, N) ||
+        !p->get_map(&mh, w + L.hq, (uint64_t)p->E * p->nr(T), p->I, N))
+        return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    const moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
+    return dispatch(p, T, m13, m2, mx, mh, P, SL.total + 1024, stream);
 }
 
 int check_forward_args(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
@@ -288,7 +303,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);
     if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
-    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, I, st).total + 1024;
+    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, I, st, false).total + 1024;
     const int optin = p->smem_optin;
     if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) ||
         !resident<16, 8>(optin, smem) || !resident<16, 4>(optin, smem) || !resident<16, 2>(optin, smem) ||
@@ -309,7 +324,9 @@ void moe_plan_destroy(moe_plan_t plan) { delete plan; }
 
 size_t moe_workspace_bytes(moe_plan_t plan, int T_max) {
     if (!plan || T_max < 1) return 0;
-    return plan->layout(T_max).total;
+    size_t need = 0;                      // the layout depends on the kernel variant: cover every T up to T_max
+    for (int T = 1; T <= plan->cap(T_max); ++T) { const size_t b = plan->layout(T).total; if (b > need) need = b; }
+    return need;
 }
 
 int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes, moe_stream_t stream) {
@@ -386,52 +403,16 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     const int N = plan->n_hw(T);
     const int stages = plan->stages_for(N, T);
     if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages);
+    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages, plan->compact(T));
     uint8_t* w = static_cast<uint8_t*>(ws);
     CUtensorMap m13, m2, mx, mh;       // encoded on the stack: no descriptor cache, nothing allocated
     if (!encode_2d(&m13, W13_fp8, (uint64_t)plan->E * 2 * plan->I, plan->H, 128) ||
         !encode_2d(&m2, W2_fp8, (uint64_t)plan->E * plan->H, plan->I, 128) ||
         !encode_2d(&mx, w + L.xq, moe::kMaxTokens, plan->H, N) ||
-        !encode_2d(&mh, w + L.hq, (uint64_t)plan->E * N, plan->I, N))
+        !encode_2d(&mh, w + L.hq, (uint64_t)plan->E * plan->nr(T), plan->I, N))
         return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-    moe::Params P;
-    P.T = T; P.H = plan->H; P.E = plan->E; P.I = plan->I; P.K = plan->K; P.scoring = plan->scoring; P.renorm = plan->renorm;
-    P.routed_scale = plan->routed_scale;
-    P.stages = stages;
-    P.split_slack_kib = plan->split_slack_kib;
-    P.route_all_tokens = plan->route_all_tokens;
-    P.grid_magic = (1ull << 40) / (unsigned long long)plan->sms + 1ull;
-    P.timeout_ns = plan->timeout_ns;
-    P.hidden = static_cast<const __nv_bfloat16*>(hidden_bf16);
-    P.Wr = static_cast<const __nv_bfloat16*>(Wr_bf16);
-    P.bias = (plan->scoring == MOE_SCORE_SIGMOID_BIAS) ? sel_bias : nullptr;
-    P.W13s = W13_scale; P.W2s = W2_scale;
-    P.out = static_cast<__nv_bfloat16*>(out_bf16);
-    P.ctrl = reinterpret_cast<unsigned*>(w + L.ctrl);
-    P.logits = reinterpret_cast<float*>(w + L.logits);
-    P.lpart = reinterpret_cast<float*>(w + L.lpart);
-    P.ids = reinterpret_cast<int*>(w + L.ids);
-    P.wts = reinterpret_cast<float*>(w + L.wts);
-    P.xq = w + L.xq;
-    P.xs = reinterpret_cast<float*>(w + L.xs);
-    P.hq = w + L.hq;
-    P.hs = reinterpret_cast<float*>(w + L.hs);
-    P.e_cnt = reinterpret_cast<unsigned*>(w + L.e_cnt);
-    P.dn_flag = reinterpret_cast<unsigned*>(w + L.dn_flag);
-    P.part_up = reinterpret_cast<float*>(w + L.part_up);
-    P.part_dn = reinterpret_cast<float*>(w + L.part_dn);
-    P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
-    P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
-    P.y = reinterpret_cast<float*>(w + L.y);
-    P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
-    const int smem_bytes = SL.total + 1024;
-    if (T == 1) return launch<16, 1>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    if (T == 2) return launch<16, 2>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    if (T <= 4) return launch<16, 4>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    if (T <= 8) return launch<16, 8>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    if (T <= 16) return launch<16, 16>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    if (T <= 32) return launch<32, 32>(plan, m13, m2, mx, mh, P, smem_bytes, s);
-    return launch<64, 64>(plan, m13, m2, mx, mh, P, smem_bytes, s);
+    const moe::Params P = make_params(plan, T, stages, L, w, hidden_bf16, Wr_bf16, sel_bias, W13_scale, W2_scale, out_bf16);
+    return dispatch(plan, T, m13, m2, mx, mh, P, SL.total + 1024, s);
 }
 
 int moe_forward_host(moe_plan_t plan, int T, const void* hidden_host, const void* Wr_bf16, const float* sel_bias,
@@ -513,7 +494,7 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
     if (grid) *grid = plan->sms;
     if (stages) *stages = st;
     if (n_hw) *n_hw = N;
-    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st).total + 1024;
+    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st, plan->compact(Tc)).total + 1024;
     return MOE_OK;
 }
 

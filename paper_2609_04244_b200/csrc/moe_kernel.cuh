@@ -56,6 +56,7 @@ struct Params {
     int stages;
     int split_slack_kib;            // see range_quantum()
     int route_all_tokens;           // up to this many tokens every CTA selects for all of them
+    int nr;                         // token rows per expert in hq / hs: the MMA N, or T rounded up to 16 when tokens are compacted per expert
     unsigned long long grid_magic;  // floor(2^40 / grid) + 1: division by the grid size as a multiplication
     unsigned long long timeout_ns;
     const __nv_bfloat16* hidden;
@@ -71,9 +72,9 @@ struct Params {
     float* wts;         // [T,K]
     uint8_t* xq;        // [64,H]
     float* xs;          // [T,H/128]
-    uint8_t* hq;        // [E,N,I]
-    float* hs;          // [E,I/128,N]
-    unsigned* e_cnt;    // [2][E] published I-blocks of an expert's intermediate tile (one row per launch parity)
+    uint8_t* hq;        // [E,nr,I]
+    float* hs;          // [E,I/128,nr]
+    unsigned* e_cnt;    // [2][4][E] published I-blocks of an expert's intermediate tile (per launch parity and 16-token pass)
     unsigned* dn_flag;  // [grid] == tag once the CTA has stored every down-projection result of its range
     float* part_up;     // [grid][2N][128]
     float* part_dn;     // [grid][N][128]
@@ -109,6 +110,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// 16-byte asynchronous copy global -> shared (L2 only), and "arrive on the mbarrier once my copies so far have landed"
+// (the arrival is one of the barrier's expected count)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_mbar_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -261,9 +271,9 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, red_off, misc_off, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, misc_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages) {
+__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages, bool compact) {
     SmemLayout L;
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
@@ -274,11 +284,12 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.w_off = o;    o += T * K * 4;
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
-    L.act_off = o;  o += (E + 1) * 4;
+    L.act_off = o;  o += (E + 1 + (compact ? (T * K) / 16 + 1 : 0)) * 4;   // + extra 16-token passes of crowded experts
     L.uidx_off = o; o += E * 4;
     o = (o + 15) & ~15;
     L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;   // input activation scales [H/128][T rounded up to 4]
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
+    L.as_off = o;   o += compact ? (16 + 16 * (H / kBlock)) * 4 : 0;   // compacted: tokens of the unit's 16 columns, their input scales [H/128][16]
     L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
     L.total = o;
     return L;
@@ -333,6 +344,17 @@ struct Walk {
         }
     }
 };
+
+// position of the n-th (0-based) set bit of a 64-bit mask that has more than n bits set
+__device__ __forceinline__ int nth_set_bit(unsigned long long m, int n) {
+    int pos = 0;
+#pragma unroll
+    for (int w = 32; w; w >>= 1) {
+        const int c = __popcll((m >> pos) & ((1ull << w) - 1ull));
+        if (n >= c) { pos += w; n -= c; }
+    }
+    return pos;
+}
 
 // monotone map float -> uint32 (larger float <=> larger integer); +0 and -0 are merged first
 __device__ __forceinline__ uint32_t orderable(float f) {
@@ -452,6 +474,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
+    // Tokens compacted per expert (N = TC = 16, used for more than 8 tokens under sparse routing): the 16 MMA columns
+    // of a unit are the tokens routed to its expert, not all tokens of the step, so the accumulator work follows the
+    // routed pairs; an expert with more than 16 tokens is walked in passes of 16 (its weights stream once per pass).
+    constexpr bool kCompact = (N == 16 && TC == 16);
     constexpr int kEpiGroups = (TC >= 32) ? 2 : 1;
     constexpr int kEpiThreads = kEpiGroupThreads * kEpiGroups;
     constexpr int kThreads = 128 + kEpiThreads, kWarps = kThreads / 32;
@@ -461,7 +487,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock, KBd = IB;
     const int S = P.stages;
-    const SmemLayout L = smem_layout(N, T, K, E, H, I, S);
+    const SmemLayout L = smem_layout(N, T, K, E, H, I, S, kCompact);
     const int TS = (T + 3) & ~3;                              // token stride of the transposed input scales
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
@@ -480,6 +506,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_xs = (float*)(smem + L.xs_off);
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
+    int* s_utok = (int*)(smem + L.as_off);                  // compacted only
+    float* s_as = (float*)(smem + L.as_off) + 16;
 
     // Programmatic dependent launch: let the next launch in the stream start placing its CTAs as ours retire, and
     // do not touch any global memory before the previous launch has completed and flushed (both are no-ops when the
@@ -489,7 +517,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
-        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, kCompact ? 32 : 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4 * kEpiGroups); }
         mbar_init(bar_drain, 1);
         mbar_init(bar_drain + 16, 1);
@@ -523,8 +551,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
     if (tid == 0) MOE_STAMP(0);
     const unsigned par = tag & 1u;
-    unsigned* e_cnt = P.e_cnt + par * E;                    // counters of this launch
-    for (int e = cta * kThreads + tid; e < E; e += G * kThreads) P.e_cnt[(par ^ 1u) * E + e] = 0u;
+    unsigned* e_cnt = P.e_cnt + par * 4 * E;                // counters of this launch: [pass][expert]
+    for (int e = cta * kThreads + tid; e < 4 * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * 4 * E + e] = 0u;
     if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
@@ -647,14 +675,26 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             __syncthreads();
         }
         if (tid == 0) MOE_STAMP(6);
-        if (warp == 0) {                                   // active-expert list in ascending expert order
+        if (warp == 0) {                                   // active list in ascending expert order: entry = expert | pass << 16
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
                 const int e = e0 + lane;
-                const bool on = (e < E) && (s_mask[e] != 0ull);
-                const unsigned b = __ballot_sync(0xffffffffu, on);
-                if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
-                base += __popc(b);
+                const unsigned long long m = (e < E) ? s_mask[e] : 0ull;
+                if constexpr (kCompact) {
+                    const int np = (__popcll(m) + 15) >> 4;        // passes of 16 tokens
+                    int incl = np;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                    const int u0 = base + incl - np;
+                    for (int ps = 0; ps < np; ++ps) s_act[u0 + ps] = e | (ps << 16);
+                    if (np) s_uidx[e] = u0;
+                    base += __shfl_sync(0xffffffffu, incl, 31);
+                } else {
+                    const bool on = (m != 0ull);
+                    const unsigned b = __ballot_sync(0xffffffffu, on);
+                    if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
+                    base += __popc(b);
+                }
             }
             if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
         }
@@ -692,7 +732,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (!wt.mbar(empty, a_ph, 2)) break;
                 const int half = a_cur & 1;
                 mbar_expect_tx(full, (uint32_t)kATileBytes);
-                tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, aw.e * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
+                tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, (aw.e & 0xFFFF) * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
                 if (half) aw.next(s_act);
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; if (!stamped) { MOE_STAMP(9); stamped = true; } }
@@ -701,7 +741,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             for (; a_cur < n_st && !wt.dead; ++a_cur) {              // down weight tiles
                 if (!wt.mbar(empty, a_ph, 2)) break;
                 mbar_expect_tx(full, (uint32_t)kATileBytes);
-                tma_load_2d_hint(dst, &tmW2, aw.kb * kBlock, aw.e * H + aw.mb * kBlock, full, stream_once);
+                tma_load_2d_hint(dst, &tmW2, aw.kb * kBlock, (aw.e & 0xFFFF) * H + aw.mb * kBlock, full, stream_once);
                 aw.next(s_act);
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; }
@@ -709,6 +749,81 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight
                 for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it)
                     for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
+            }
+        }
+        __syncwarp();
+    }
+    else if (warp == 2 && kCompact) {
+        // Compacted tokens: the activation tile of an up k-step is gathered -- row r = the quantised input of the
+        // unit's r-th token -- by the whole warp with 16-byte asynchronous copies into the 128-byte-swizzled layout
+        // the MMA expects (chunk c of row r sits at chunk c ^ (r & 7)); every lane arrives on the stage's barrier
+        // once its copies have landed.  The down projection's tile is one bulk-tensor copy (rows are already compact).
+        if (alive) {
+            const int n_up_st = 2 * (up_hi - up_lo), n_st = n_up_st + (dn_hi - dn_lo);
+            Walk bw;
+            int b_cur = 0, b_st = 0;
+            uint32_t b_ph = 1u;
+            uint32_t dst = smem_u32(smem) + kATileBytes, full = bar_fullb, empty = bar_empty;
+            if (n_up_st > 0) bw.init(up_lo, KBu, IB, s_act);
+            else if (n_st > 0) bw.init(dn_lo, KBd, HB, s_act);
+            const int chunk = lane & 7, r0 = lane >> 3;          // this lane copies chunk `chunk` of rows r0, r0+4, r0+8, r0+12
+            int b_entry = -1;
+            int tokr[4] = {-1, -1, -1, -1};
+            bool ok = true;
+            for (; b_cur < n_up_st; ++b_cur) {
+                if (lane == 0) ok = wt.mbar(empty, b_ph, 10);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if ((b_cur & 1) == 0) {
+                    if (bw.e != b_entry) {
+                        b_entry = bw.e;
+                        const unsigned long long m = s_mask[b_entry & 0xFFFF];
+                        const int colbase = (b_entry >> 16) * 16, cnt = min(16, __popcll(m) - colbase);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) tokr[i] = (r0 + 4 * i < cnt) ? nth_set_bit(m, colbase + r0 + 4 * i) : -1;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = r0 + 4 * i;
+                        if (tokr[i] >= 0)
+                            cp_async16(dst + (uint32_t)(r * kBlock + ((chunk ^ (r & 7)) << 4)),
+                                       P.xq + (size_t)tokr[i] * H + bw.kb * kBlock + chunk * 16);
+                    }
+                    cp_async_mbar_arrive(full);
+                } else {
+                    mbar_arrive(full);
+                    bw.next(s_act);
+                }
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
+            }
+            if (ok && n_st > n_up_st) bw.init(dn_lo, KBd, HB, s_act);
+            int ready_e = -1;                    // unit whose intermediate tile is known to be published
+            for (; b_cur < n_st && ok; ++b_cur) {
+                if (lane == 0) ok = wt.mbar(empty, b_ph, 10);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                const int be = bw.e & 0xFFFF, bpass = bw.e >> 16;
+                if (bw.e != ready_e) {                               // published? (Section 3.2, readiness hand-off)
+                    if (lane == 0) { ok = wt.flag(e_cnt + bpass * E + be, (unsigned)IB, 11); fence_proxy_async(); }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    ready_e = bw.e;
+                }
+                if (lane == 0) {
+                    mbar_expect_tx(full, (uint32_t)(N * kBlock));
+                    tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * 16, full);
+                } else {
+                    mbar_arrive(full);
+                }
+                bw.next(s_act);
+                dst += L.stage_bytes; full += 8; empty += 8;
+                if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
+            }
+            cp_async_wait_all();                 // nothing of this warp is in flight past this point ...
+            if (!ok && lane == 0) {              // ... except bulk copies: give-up path waits (bounded) for them
+                for (int it = (b_cur > S ? b_cur - S : 0); it < b_cur; ++it)
+                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_fullb + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
             }
         }
         __syncwarp();
@@ -739,13 +854,14 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             int ready_e = -1;                    // expert whose intermediate tile is known to be published
             for (; b_cur < n_st && !wt.dead; ++b_cur) {              // intermediate activation tiles
                 if (!wt.mbar(empty, b_ph, 10)) break;
+                const int be = bw.e & 0xFFFF, bpass = bw.e >> 16;
                 if (bw.e != ready_e) {                               // published? (Section 3.2, readiness hand-off)
-                    if (!wt.flag(e_cnt + bw.e, (unsigned)IB, 11)) break;
+                    if (!wt.flag(e_cnt + bpass * E + be, (unsigned)IB, 11)) break;
                     fence_proxy_async();
                     ready_e = bw.e;
                 }
                 mbar_expect_tx(full, (uint32_t)(N * kBlock));
-                tma_load_2d(dst, &tmHq, bw.kb * kBlock, bw.e * N, full);
+                tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * 16, full);
                 bw.next(s_act);
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
@@ -781,6 +897,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const uint32_t ph0 = ph;
                 const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)L.stage_bytes;
                 if (!wt.mbar(bar_full + 8 * st0, ph0, 4) || !wt.mbar(bar_fullb + 8 * st0, ph0, 4)) break;
+                if (kCompact && up) fence_proxy_async();       // the gathered tile was written through the generic proxy
                 const uint64_t b_desc = make_smem_desc(a0 + kATileBytes);
                 const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
                 if (first && who == 0) { MOE_STAMP(10); first = false; }
@@ -825,7 +942,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         volatile uint32_t* s_giveup = misc + 3;
         bool first_acc = true;
-        constexpr int CH = TCG < 16 ? TCG : 16;                // columns per TMEM load
+        constexpr int CH = kCompact ? 4 : (TCG < 16 ? TCG : 16);   // columns per TMEM load
         int buf = 0, hs_e = -1;
         uint32_t tph = 0;
         float accg[TCG], accu[TCG];
@@ -848,7 +965,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             auto fetch_scales = [&](int sidx, float& g, float& u2) {
                 g = 0.f; u2 = 0.f;
                 if (sidx < hi) {
-                    const int unit = div_small(sidx, KB), kb = sidx - unit * KB, uu = div_small(unit, MB), mb = unit - uu * MB, e = s_act[uu];
+                    const int unit = div_small(sidx, KB), kb = sidx - unit * KB, uu = div_small(unit, MB), mb = unit - uu * MB, e = s_act[uu] & 0xFFFF;
                     if (up) {
                         g = __ldg(P.W13s + ((size_t)e * 2 * IB + mb) * KBu + kb);
                         u2 = __ldg(P.W13s + ((size_t)e * 2 * IB + IB + mb) * KBu + kb);
@@ -863,19 +980,39 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
             for (int s = lo; s < hi && !wt.dead;) {
                 // ---- one piece: the k-steps [s, pend) of unit (e, mb), first K block kb0
-                const int e = w.e, mb = w.mb, kb0 = w.kb;
+                const int entry = w.e, e = entry & 0xFFFF, colbase = (entry >> 16) * 16, mb = w.mb, kb0 = w.kb;
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
-                if (!up && e != hs_e) {
-                    // activation scales of this expert's intermediate tile -> shared memory (once per expert)
-                    const bool got = (etid == 0) ? wt.flag(e_cnt + e, (unsigned)IB, 8) : true;
+                const unsigned long long mask = s_mask[e];
+                // compacted: column c of the unit = the (colbase + c)-th token routed to the expert; lane c knows it
+                int cnt = TCG, tok_lane = lane;
+                if constexpr (kCompact) {
+                    cnt = min(16, __popcll(mask) - colbase);
+                    tok_lane = (lane < cnt) ? nth_set_bit(mask, colbase + lane) : 0;
+                }
+                auto col_on = [&](int n) -> bool { return kCompact ? (n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
+                if (!up && entry != hs_e) {
+                    // activation scales of this expert's intermediate tile -> shared memory (once per expert and pass)
+                    const bool got = (etid == 0) ? wt.flag(e_cnt + (entry >> 16) * E + e, (unsigned)IB, 8) : true;
                     if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
-                    for (int i = etid; i < IB * N; i += kEpiThreads) s_hs[i] = __ldcg(P.hs + (size_t)e * IB * N + i);
-                    hs_e = e;
+                    for (int i = etid; i < IB * N; i += kEpiThreads) s_hs[i] = __ldcg(P.hs + ((size_t)e * IB + i / N) * P.nr + colbase + i % N);
+                    hs_e = entry;
                     epi_bar(kEpiThreads);
                 }
-                const float* as_p = up ? (s_xs + kb0 * TS) : (s_hs + kb0 * N);   // activation scales [K block][token]
-                const int as_step = up ? TS : N;
+                if constexpr (kCompact) {
+                    if (up) {
+                        // input scales of this piece's K blocks, gathered for the unit's tokens: [K block][column]
+                        if (etid < 16) s_utok[etid] = tok_lane;
+                        epi_bar(kEpiThreads);
+                        for (int idx = etid; idx < (pend - s) * 16; idx += kEpiThreads) {
+                            const int c = idx & 15;
+                            s_as[idx] = (c < cnt) ? s_xs[(kb0 + (idx >> 4)) * TS + s_utok[c]] : 0.f;
+                        }
+                        epi_bar(kEpiThreads);
+                    }
+                }
+                const float* as_p = up ? (kCompact ? s_as : s_xs + kb0 * TS) : (s_hs + kb0 * N);   // activation scales [K block][column]
+                const int as_step = up ? (kCompact ? 16 : TS) : N;
 #pragma unroll
                 for (int n = 0; n < TCG; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
@@ -897,6 +1034,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     float dg[TCG], du[TCG];
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
+                        if (kCompact && c >= cnt) break;            // warp-uniform: only the routed columns are read
                         tmem_ld<CH>(tcol + cb + c, dg + c);
                         if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
                     }
@@ -906,6 +1044,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
+                        if (kCompact && c >= cnt) break;
                         float as[CH];
                         if constexpr (CH >= 4) {
 #pragma unroll
@@ -929,16 +1068,16 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const bool unit_done = (pend == uend);
                 s = pend;
                 if (unit_done) w.next_unit(s_act);
-                const unsigned long long mask = s_mask[e];
                 if (!up && unit_done && ustart >= lo) {
                     // whole down unit: every warp stores its rows and counts itself done -- no block-level barrier
                     // (units of the down projection can be as short as two k-steps)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if ((mask >> (cb + n)) & 1ull) {
+                        if (col_on(n)) {
+                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, n) : cb + n;
                             int sl = 0;
-                            for (int jj = 0; jj < K; ++jj) if (s_ids[(cb + n) * K + jj] == e) sl = jj;
-                            __stcg(P.y + ((size_t)(cb + n) * K + sl) * H + mb * kBlock + row, accg[n]);
+                            for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
+                            __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
                     continue;                                   // published once per CTA, after the last down unit
@@ -952,7 +1091,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
                     for (int n = 0; n < TCG; ++n)
-                        if ((mask >> (cb + n)) & 1ull) {                        // only tokens routed to this expert matter
+                        if (col_on(n)) {                        // only tokens routed to this expert matter
                             __stcg(dst + (cb + n) * kBlock + row, accg[n]);
                             if (up) __stcg(dst + (N + cb + n) * kBlock + row, accu[n]);
                         }
@@ -980,7 +1119,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TCG; ++n)
-                            if ((mask >> (cb + n)) & 1ull) {
+                            if (col_on(n)) {
                                 accg[n] += __ldcg(src + (cb + n) * kBlock + row);
                                 if (up) accu[n] += __ldcg(src + (N + cb + n) * kBlock + row);
                             }
@@ -990,7 +1129,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if ((mask >> (cb + n)) & 1ull) {                        // warp-uniform: other tokens cost nothing
+                        if (col_on(n)) {                        // warp-uniform: other tokens cost nothing
                             const float g = accg[n];
                             const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
                             accg[n] = a;
@@ -1002,26 +1141,27 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     epi_bar(kEpiThreads);
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if ((mask >> (cb + n)) & 1ull) {
+                        if (col_on(n)) {
                             const float amax = fmaxf(fmaxf(s_red[cb + n], s_red[N + cb + n]), fmaxf(s_red[2 * N + cb + n], s_red[3 * N + cb + n]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
                             const float2 v = make_float2(__fdiv_rn(accg[n], sc), 0.f);
                             const uint8_t code = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
-                            P.hq[((size_t)e * N + cb + n) * I + mb * kBlock + row] = code;
-                            if (row == 0) P.hs[((size_t)e * IB + mb) * N + cb + n] = sc;
+                            P.hq[((size_t)e * P.nr + colbase + cb + n) * I + mb * kBlock + row] = code;
+                            if (row == 0) P.hs[((size_t)e * IB + mb) * P.nr + colbase + cb + n] = sc;
                         }
                     }
                     fence_proxy_async();
                     epi_bar(kEpiThreads);
-                    if (etid == 0) red_release_add(e_cnt + e, 1u);   // the expert's tile is complete at count == I/128
+                    if (etid == 0) red_release_add(e_cnt + (entry >> 16) * E + e, 1u);   // the expert's tile (of this pass) is complete at count == I/128
                 } else {
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if ((mask >> (cb + n)) & 1ull) {
+                        if (col_on(n)) {
+                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, n) : cb + n;
                             int sl = 0;
-                            for (int jj = 0; jj < K; ++jj) if (s_ids[(cb + n) * K + jj] == e) sl = jj;
-                            __stcg(P.y + ((size_t)(cb + n) * K + sl) * H + mb * kBlock + row, accg[n]);
+                            for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
+                            __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
                         }
                     }
                     // (published once per CTA, after the last down unit)
@@ -1041,7 +1181,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             bool got = true;
             if (mine && gtid < K) {
                 // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
-                const unsigned unit = (unsigned)(s_uidx[s_ids[t * K + gtid]] * HB + hb);
+                const int ex = s_ids[t * K + gtid];
+                const int ps = kCompact ? (__popcll(s_mask[ex] & ((1ull << t) - 1ull)) >> 4) : 0;   // the pass that holds token t
+                const unsigned unit = (unsigned)((s_uidx[ex] + ps) * HB + hb);
                 const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
                 const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
                 got = wt.flag(P.dn_flag + owner, tag, 7);

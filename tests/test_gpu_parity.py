@@ -13,8 +13,9 @@ SMALL_SIG = wl.MoEShape("small_sig", 5, H=512, E=32, I=256, top_k=4, scoring=wl.
 RAGGED = wl.MoEShape("ragged", 2, H=384, E=20, I=640, top_k=3, scoring=wl.SCORE_SOFTMAX)
 
 
-@pytest.mark.parametrize("T", [1, 2, 5, 16, 17, 33, 64])
+@pytest.mark.parametrize("T", [1, 2, 5, 9, 16, 17, 32, 33, 64])
 def test_tiny_all_token_tiles(T):
+    """Every kernel variant: token columns 1..8, tokens compacted per expert (9..32 here), all tokens as columns (33, 64)."""
     r = run_case(TINY, T, repeat=2)
     assert r["rel_l2"] < 2e-3, r
 
@@ -36,8 +37,10 @@ def test_config2_qwen3_like(T):
     assert r["rel_l2"] < 2e-3, r
 
 
-@pytest.mark.parametrize("regime,T", [("same", 4), ("disjoint", 4), ("disjoint", 32), ("natural", 64)])
+@pytest.mark.parametrize("regime,T", [("same", 4), ("disjoint", 4), ("disjoint", 32), ("natural", 64), ("same", 40), ("same", 64)])
 def test_config3_routing_regimes(regime, T):
+    """Natural, maximum-reuse and maximum-bytes routing; 40 and 64 tokens on the same 8 experts walk each expert in
+    three and four passes of 16 compacted tokens."""
     r = run_case(wl.SHAPES["c2_qwen3_30b_a3b"], T, regime=regime, max_oracle_tokens=8)
     if regime == "same":
         assert r["unique_experts"] == 8
