@@ -80,11 +80,15 @@ struct moe_plan {
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
-    // More than 8 tokens under sparse routing (on average at most 8 tokens per expert): the kernel compacts the tokens
-    // of each expert into the 16 MMA columns; denser routing takes all tokens as columns (N = 32 or 64).
-    bool compact(int T) const { return T > 8 && (long long)T * K <= 8ll * E; }
-    int n_hw(int T) const { return (T <= 8 || compact(T)) ? 16 : (T <= 32 ? 32 : 64); }
-    int nr(int T) const { return compact(T) ? ((T + 15) & ~15) : n_hw(T); }     // token rows per expert in hq / hs
+    // More than 8 tokens: the kernel compacts the tokens of each expert into the MMA columns -- 16 columns while an
+    // expert sees at most 8 tokens on average, 32 columns up to 20 on average (or whenever T <= 32); denser routing
+    // of more than 32 tokens takes all tokens as columns (N = 64).
+    int n_hw(int T) const {
+        if (T <= 8 || (long long)T * K <= 8ll * E) return 16;
+        return (T <= 32 || (long long)T * K <= 20ll * E) ? 32 : 64;
+    }
+    bool compact(int T) const { return T > 8 && n_hw(T) <= 32; }
+    int nr(int T) const { const int N = n_hw(T); return compact(T) ? (T + N - 1) / N * N : N; }   // token rows per expert in hq / hs
     int cap(int T) const { return T < moe::kMaxTokens ? T : moe::kMaxTokens; }
 
     WsLayout layout(int T_max) const {
@@ -220,8 +224,8 @@ int dispatch(Plan* p, int T, const CUtensorMap& m13, const CUtensorMap& m2, cons
     if (T == 2) return launch<16, 2>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (p->compact(T)) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (T <= 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (p->n_hw(T) == 16) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (p->n_hw(T) == 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
 }
 

@@ -284,12 +284,12 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.w_off = o;    o += T * K * 4;
     o = (o + 7) & ~7;
     L.mask_off = o; o += E * 8;
-    L.act_off = o;  o += (E + 1 + (compact ? (T * K) / 16 + 1 : 0)) * 4;   // + extra 16-token passes of crowded experts
+    L.act_off = o;  o += (E + 1 + (compact ? (T * K) / N + 1 : 0)) * 4;   // + extra N-token passes of crowded experts
     L.uidx_off = o; o += E * 4;
     o = (o + 15) & ~15;
     L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;   // input activation scales [H/128][T rounded up to 4]
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
-    L.as_off = o;   o += compact ? (16 + 16 * (H / kBlock)) * 4 : 0;   // compacted: tokens of the unit's 16 columns, their input scales [H/128][16]
+    L.as_off = o;   o += compact ? (N + N * (H / kBlock)) * 4 : 0;   // compacted: tokens of the unit's N columns, their input scales [H/128][N]
     L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
     L.total = o;
     return L;
@@ -474,10 +474,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
-    // Tokens compacted per expert (N = TC = 16, used for more than 8 tokens under sparse routing): the 16 MMA columns
-    // of a unit are the tokens routed to its expert, not all tokens of the step, so the accumulator work follows the
-    // routed pairs; an expert with more than 16 tokens is walked in passes of 16 (its weights stream once per pass).
-    constexpr bool kCompact = (N == 16 && TC == 16);
+    // Tokens compacted per expert (N = TC = 16 or 32, used for more than 8 tokens): the N MMA columns of a unit are
+    // the tokens routed to its expert, not all tokens of the step, so the accumulator work follows the routed pairs;
+    // an expert with more than N tokens is walked in passes of N (its weights stream once per pass).
+    constexpr bool kCompact = (TC >= 16 && TC == N && N <= 32);
     constexpr int kEpiGroups = (TC >= 32) ? 2 : 1;
     constexpr int kEpiThreads = kEpiGroupThreads * kEpiGroups;
     constexpr int kThreads = 128 + kEpiThreads, kWarps = kThreads / 32;
@@ -507,7 +507,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
     int* s_utok = (int*)(smem + L.as_off);                  // compacted only
-    float* s_as = (float*)(smem + L.as_off) + 16;
+    float* s_as = (float*)(smem + L.as_off) + N;
 
     // Programmatic dependent launch: let the next launch in the stream start placing its CTAs as ours retire, and
     // do not touch any global memory before the previous launch has completed and flushed (both are no-ops when the
@@ -681,7 +681,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int e = e0 + lane;
                 const unsigned long long m = (e < E) ? s_mask[e] : 0ull;
                 if constexpr (kCompact) {
-                    const int np = (__popcll(m) + 15) >> 4;        // passes of 16 tokens
+                    const int np = (__popcll(m) + N - 1) / N;      // passes of N tokens
                     int incl = np;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
@@ -766,9 +766,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             uint32_t dst = smem_u32(smem) + kATileBytes, full = bar_fullb, empty = bar_empty;
             if (n_up_st > 0) bw.init(up_lo, KBu, IB, s_act);
             else if (n_st > 0) bw.init(dn_lo, KBd, HB, s_act);
-            const int chunk = lane & 7, r0 = lane >> 3;          // this lane copies chunk `chunk` of rows r0, r0+4, r0+8, r0+12
+            const int chunk = lane & 7, r0 = lane >> 3;          // this lane copies chunk `chunk` of rows r0, r0+4, r0+8, ...
             int b_entry = -1;
-            int tokr[4] = {-1, -1, -1, -1};
+            int tokr[N / 4];
+#pragma unroll
+            for (int i = 0; i < N / 4; ++i) tokr[i] = -1;
             bool ok = true;
             for (; b_cur < n_up_st; ++b_cur) {
                 if (lane == 0) ok = wt.mbar(empty, b_ph, 10);
@@ -778,12 +780,12 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (bw.e != b_entry) {
                         b_entry = bw.e;
                         const unsigned long long m = s_mask[b_entry & 0xFFFF];
-                        const int colbase = (b_entry >> 16) * 16, cnt = min(16, __popcll(m) - colbase);
+                        const int colbase = (b_entry >> 16) * N, cnt = min(N, __popcll(m) - colbase);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) tokr[i] = (r0 + 4 * i < cnt) ? nth_set_bit(m, colbase + r0 + 4 * i) : -1;
+                        for (int i = 0; i < N / 4; ++i) tokr[i] = (r0 + 4 * i < cnt) ? nth_set_bit(m, colbase + r0 + 4 * i) : -1;
                     }
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                    for (int i = 0; i < N / 4; ++i) {
                         const int r = r0 + 4 * i;
                         if (tokr[i] >= 0)
                             cp_async16(dst + (uint32_t)(r * kBlock + ((chunk ^ (r & 7)) << 4)),
@@ -812,7 +814,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 }
                 if (lane == 0) {
                     mbar_expect_tx(full, (uint32_t)(N * kBlock));
-                    tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * 16, full);
+                    tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * N, full);
                 } else {
                     mbar_arrive(full);
                 }
@@ -861,7 +863,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     ready_e = bw.e;
                 }
                 mbar_expect_tx(full, (uint32_t)(N * kBlock));
-                tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * 16, full);
+                tma_load_2d(dst, &tmHq, bw.kb * kBlock, be * P.nr + bpass * N, full);
                 bw.next(s_act);
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
@@ -980,17 +982,17 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
             for (int s = lo; s < hi && !wt.dead;) {
                 // ---- one piece: the k-steps [s, pend) of unit (e, mb), first K block kb0
-                const int entry = w.e, e = entry & 0xFFFF, colbase = (entry >> 16) * 16, mb = w.mb, kb0 = w.kb;
+                const int entry = w.e, e = entry & 0xFFFF, colbase = (entry >> 16) * N, mb = w.mb, kb0 = w.kb;
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
                 const unsigned long long mask = s_mask[e];
                 // compacted: column c of the unit = the (colbase + c)-th token routed to the expert; lane c knows it
                 int cnt = TCG, tok_lane = lane;
                 if constexpr (kCompact) {
-                    cnt = min(16, __popcll(mask) - colbase);
+                    cnt = min(N, __popcll(mask) - colbase);
                     tok_lane = (lane < cnt) ? nth_set_bit(mask, colbase + lane) : 0;
                 }
-                auto col_on = [&](int n) -> bool { return kCompact ? (n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
+                auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
                 if (!up && entry != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert and pass)
                     const bool got = (etid == 0) ? wt.flag(e_cnt + (entry >> 16) * E + e, (unsigned)IB, 8) : true;
@@ -1002,17 +1004,17 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if constexpr (kCompact) {
                     if (up) {
                         // input scales of this piece's K blocks, gathered for the unit's tokens: [K block][column]
-                        if (etid < 16) s_utok[etid] = tok_lane;
+                        if (etid < N) s_utok[etid] = tok_lane;
                         epi_bar(kEpiThreads);
-                        for (int idx = etid; idx < (pend - s) * 16; idx += kEpiThreads) {
-                            const int c = idx & 15;
-                            s_as[idx] = (c < cnt) ? s_xs[(kb0 + (idx >> 4)) * TS + s_utok[c]] : 0.f;
+                        for (int idx = etid; idx < (pend - s) * N; idx += kEpiThreads) {
+                            const int c = idx & (N - 1);
+                            s_as[idx] = (c < cnt) ? s_xs[(kb0 + idx / N) * TS + s_utok[c]] : 0.f;
                         }
                         epi_bar(kEpiThreads);
                     }
                 }
                 const float* as_p = up ? (kCompact ? s_as : s_xs + kb0 * TS) : (s_hs + kb0 * N);   // activation scales [K block][column]
-                const int as_step = up ? (kCompact ? 16 : TS) : N;
+                const int as_step = up ? (kCompact ? N : TS) : N;
 #pragma unroll
                 for (int n = 0; n < TCG; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
@@ -1034,7 +1036,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     float dg[TCG], du[TCG];
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
-                        if (kCompact && c >= cnt) break;            // warp-uniform: only the routed columns are read
+                        if (kCompact && cb + c >= cnt) break;       // warp-uniform: only the routed columns are read
                         tmem_ld<CH>(tcol + cb + c, dg + c);
                         if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
                     }
@@ -1044,7 +1046,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
-                        if (kCompact && c >= cnt) break;
+                        if (kCompact && cb + c >= cnt) break;
                         float as[CH];
                         if constexpr (CH >= 4) {
 #pragma unroll
@@ -1074,7 +1076,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
                         if (col_on(n)) {
-                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, n) : cb + n;
+                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, cb + n) : cb + n;
                             int sl = 0;
                             for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
                             __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
@@ -1158,7 +1160,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
                         if (col_on(n)) {
-                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, n) : cb + n;
+                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, cb + n) : cb + n;
                             int sl = 0;
                             for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
                             __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
@@ -1182,7 +1184,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (mine && gtid < K) {
                 // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
                 const int ex = s_ids[t * K + gtid];
-                const int ps = kCompact ? (__popcll(s_mask[ex] & ((1ull << t) - 1ull)) >> 4) : 0;   // the pass that holds token t
+                const int ps = kCompact ? (__popcll(s_mask[ex] & ((1ull << t) - 1ull)) / N) : 0;   // the pass that holds token t
                 const unsigned unit = (unsigned)((s_uidx[ex] + ps) * HB + hb);
                 const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
                 const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
