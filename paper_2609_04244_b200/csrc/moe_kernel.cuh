@@ -1018,32 +1018,28 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                 for (int n = 0; n < TCG; ++n) { accg[n] = 0.f; accu[n] = 0.f; }
 
-                for (int i = 0; i < pend - s; ++i) {
-                    const int j = (s + i - lo) & 31;
-                    if (j == 0 && s + i != lo) {
+                // Two k-steps per turn when the second accumulator is already complete (one warp per scheduler: nothing
+                // else hides the TMEM-load latency); one k-step otherwise, so a just-in-time MMA stream is never waited on.
+                constexpr bool kDual = (TCG <= 16) && !kCompact;
+                auto next_scales = [&](int sidx, float& g, float& u2) {
+                    const int j = (sidx - lo) & 31;
+                    if (j == 0 && sidx != lo) {
                         sg_cur = sg_nxt; su_cur = su_nxt;
-                        fetch_scales(s + i + 32 + lane, sg_nxt, su_nxt);
+                        fetch_scales(sidx + 32 + lane, sg_nxt, su_nxt);
                     }
-                    const float wsg = __shfl_sync(0xffffffffu, sg_cur, j);
-                    const float wsu = __shfl_sync(0xffffffffu, su_cur, j);
-                    // A wait that runs out is recorded and the warp keeps walking in lockstep with the others;
-                    // the piece end below turns the record into a uniform decision to stop.
-                    if (!wt.mbar(bar_tfull + 8 * buf, tph, 5)) *s_giveup = 1u;
-                    tc_fence_after();
-                    if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
-                    const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
-                    // all TMEM loads of this k-step first, one wait, free the buffer, then the arithmetic
-                    float dg[TCG], du[TCG];
+                    g = __shfl_sync(0xffffffffu, sg_cur, j);
+                    u2 = __shfl_sync(0xffffffffu, su_cur, j);
+                };
+                auto load_acc = [&](int b, float* dg, float* du) {
+                    const uint32_t tcol = t_lane + (uint32_t)(b * 2 * N);
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
                         if (kCompact && cb + c >= cnt) break;       // warp-uniform: only the routed columns are read
                         tmem_ld<CH>(tcol + cb + c, dg + c);
                         if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
                     }
-                    tmem_ld_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                };
+                auto add_scaled = [&](const float* dg, const float* du, float wsg, float wsu, int i) {
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
                         if (kCompact && cb + c >= cnt) break;
@@ -1065,6 +1061,34 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                             if (up) accu[n] = fmaf(du[n], wsu * as[jj], accu[n]);
                         }
                     }
+                };
+                for (int i = 0; i < pend - s;) {
+                    float wsg0, wsu0, wsg1 = 0.f, wsu1 = 0.f;
+                    next_scales(s + i, wsg0, wsu0);
+                    // A wait that runs out is recorded and the warp keeps walking in lockstep with the others;
+                    // the piece end below turns the record into a uniform decision to stop.
+                    if (!wt.mbar(bar_tfull + 8 * buf, tph, 5)) *s_giveup = 1u;
+                    int buf1 = buf + 1;
+                    uint32_t tph1 = tph;
+                    if (buf1 == kTmemBufs) { buf1 = 0; tph1 ^= 1u; }
+                    bool two = false;
+                    if constexpr (kDual)
+                        two = (i + 1 < pend - s) && __all_sync(0xffffffffu, mbar_try_wait(bar_tfull + 8 * buf1, tph1));
+                    if (two) next_scales(s + i + 1, wsg1, wsu1);
+                    tc_fence_after();
+                    if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
+                    // all TMEM loads first, one wait, free the buffers, then the arithmetic
+                    float dg0[TCG], du0[TCG], dg1[kDual ? TCG : 1], du1[kDual ? TCG : 1];
+                    load_acc(buf, dg0, du0);
+                    if constexpr (kDual) { if (two) load_acc(buf1, dg1, du1); }
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(bar_tempty + 8 * buf); if (two) mbar_arrive(bar_tempty + 8 * buf1); }
+                    add_scaled(dg0, du0, wsg0, wsu0, i);
+                    if constexpr (kDual) { if (two) add_scaled(dg1, du1, wsg1, wsu1, i + 1); }
+                    if (two) { buf = buf1; tph = tph1; ++i; }
+                    ++i;
                     if (++buf == kTmemBufs) { buf = 0; tph ^= 1u; }
                 }
                 const bool unit_done = (pend == uend);
