@@ -271,7 +271,7 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, misc_off, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, wtok_off, misc_off, total;
 };
 __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages, bool compact) {
     SmemLayout L;
@@ -291,6 +291,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
     L.as_off = o;   o += compact ? (N + N * (H / kBlock)) * 4 : 0;   // compacted: tokens of the unit's N columns, their input scales [H/128][N]
     L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
+    L.wtok_off = o; o += kMaxWarps * 32 * 4;        // per accumulator warp: column -> token of the current unit
     L.total = o;
     return L;
 }
@@ -507,6 +508,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
     int* s_utok = (int*)(smem + L.as_off);                  // compacted only
+    int* s_wtok = (int*)(smem + L.wtok_off);
     float* s_as = (float*)(smem + L.as_off) + N;
 
     // Programmatic dependent launch: let the next launch in the stream start placing its CTAs as ours retire, and
@@ -987,12 +989,29 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int pend = uend < hi ? uend : hi;
                 const unsigned long long mask = s_mask[e];
                 // compacted: column c of the unit = the (colbase + c)-th token routed to the expert; lane c knows it
-                int cnt = TCG, tok_lane = lane;
+                // lane l of every warp looks after column cb + l: its token, and (down projection) where its result goes
+                int cnt = TCG, tok_lane = cb + lane;
                 if constexpr (kCompact) {
                     cnt = min(N, __popcll(mask) - colbase);
-                    tok_lane = (lane < cnt) ? nth_set_bit(mask, colbase + lane) : 0;
+                    // invert "rank of a token among the expert's tokens": every lane places tokens lane and lane + 32
+                    int* wtok = s_wtok + (warp - kEpiWarp0) * 32;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = lane + 32 * h;
+                        const int r = __popcll(mask & ((1ull << t) - 1ull)) - colbase;
+                        if (((mask >> t) & 1ull) && r >= 0 && r < N) wtok[r] = t;
+                    }
+                    __syncwarp();
+                    tok_lane = (cb + lane < cnt) ? wtok[cb + lane] : 0;
+                    __syncwarp();
                 }
                 auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
+                int yoff_lane = 0;                             // first element of the (token, slot) row of y for column cb + lane
+                if (!up && lane < TCG && col_on(lane)) {
+                    int sl = 0;
+                    for (int jj = 0; jj < K; ++jj) if (s_ids[tok_lane * K + jj] == e) sl = jj;
+                    yoff_lane = (tok_lane * K + sl) * H;
+                }
                 if (!up && entry != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert and pass)
                     const bool got = (etid == 0) ? wt.flag(e_cnt + (entry >> 16) * E + e, (unsigned)IB, 8) : true;
@@ -1032,11 +1051,26 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 };
                 auto load_acc = [&](int b, float* dg, float* du) {
                     const uint32_t tcol = t_lane + (uint32_t)(b * 2 * N);
+                    if constexpr (kCompact) {
+                        // one load as wide as the routed columns need (warp-uniform): a TMEM load costs about the
+                        // same whatever its width
+                        const int need = cnt - cb;
+                        if (need <= 4) {
+                            tmem_ld<4>(tcol + cb, dg);
+                            if (up) tmem_ld<4>(tcol + N + cb, du);
+                        } else if (need <= 8) {
+                            tmem_ld<8>(tcol + cb, dg);
+                            if (up) tmem_ld<8>(tcol + N + cb, du);
+                        } else {
+                            tmem_ld<16>(tcol + cb, dg);
+                            if (up) tmem_ld<16>(tcol + N + cb, du);
+                        }
+                    } else {
 #pragma unroll
-                    for (int c = 0; c < TCG; c += CH) {
-                        if (kCompact && cb + c >= cnt) break;       // warp-uniform: only the routed columns are read
-                        tmem_ld<CH>(tcol + cb + c, dg + c);
-                        if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
+                        for (int c = 0; c < TCG; c += CH) {
+                            tmem_ld<CH>(tcol + cb + c, dg + c);
+                            if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
+                        }
                     }
                 };
                 auto add_scaled = [&](const float* dg, const float* du, float wsg, float wsu, int i) {
@@ -1100,10 +1134,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
                         if (col_on(n)) {
-                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, cb + n) : cb + n;
-                            int sl = 0;
-                            for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
-                            __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
+                            const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
+                            __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
                         }
                     }
                     continue;                                   // published once per CTA, after the last down unit
@@ -1184,10 +1216,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
                         if (col_on(n)) {
-                            const int tok = kCompact ? __shfl_sync(0xffffffffu, tok_lane, cb + n) : cb + n;
-                            int sl = 0;
-                            for (int jj = 0; jj < K; ++jj) if (s_ids[tok * K + jj] == e) sl = jj;
-                            __stcg(P.y + ((size_t)tok * K + sl) * H + mb * kBlock + row, accg[n]);
+                            const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
+                            __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
                         }
                     }
                     // (published once per CTA, after the last down unit)
