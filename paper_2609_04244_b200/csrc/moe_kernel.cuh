@@ -271,7 +271,7 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, wtok_off, misc_off, total;
+    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, poff_off, pair_off, misc_off, total;
 };
 __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages, bool compact) {
     SmemLayout L;
@@ -291,7 +291,8 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.hs_off = o;   o += N * (I / kBlock) * 4;      // intermediate activation scales of the current expert [I/128][N]  (16-byte aligned rows)
     L.as_off = o;   o += compact ? (N + N * (H / kBlock)) * 4 : 0;   // compacted: tokens of the unit's N columns, their input scales [H/128][N]
     L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
-    L.wtok_off = o; o += kMaxWarps * 32 * 4;        // per accumulator warp: column -> token of the current unit
+    L.poff_off = o; o += E * 4;                     // expert -> first entry of its (token, slot) pairs
+    L.pair_off = o; o += ((T * K * 2 + 15) & ~15);  // (token | slot << 8) of every routed pair, grouped by expert, tokens ascending
     L.total = o;
     return L;
 }
@@ -508,7 +509,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     float* s_hs = (float*)(smem + L.hs_off);
     float* s_red = (float*)(smem + L.red_off);
     int* s_utok = (int*)(smem + L.as_off);                  // compacted only
-    int* s_wtok = (int*)(smem + L.wtok_off);
+    int* s_poff = (int*)(smem + L.poff_off);
+    unsigned short* s_pair = (unsigned short*)(smem + L.pair_off);
     float* s_as = (float*)(smem + L.as_off) + N;
 
     // Programmatic dependent launch: let the next launch in the stream start placing its CTAs as ours retire, and
@@ -951,6 +953,26 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         uint32_t tph = 0;
         float accg[TCG], accu[TCG];
 
+        // While the first weight tiles are in flight: the routed (token, slot) pairs grouped by expert, tokens
+        // ascending -- entry r of expert e is the r-th token routed to e and the top-k slot e holds for it.
+        if (warp == kEpiWarp0) {
+            int base = 0;
+            for (int e0 = 0; e0 < E; e0 += 32) {
+                const int c = (e0 + lane < E) ? __popcll(s_mask[e0 + lane]) : 0;
+                int incl = c;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                if (e0 + lane < E) s_poff[e0 + lane] = base + incl - c;
+                base += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        }
+        epi_bar(kEpiThreads);
+        for (int pi = etid; pi < T * K; pi += kEpiThreads) {
+            const int t = div_small(pi, K), ex = s_ids[pi];
+            s_pair[s_poff[ex] + __popcll(s_mask[ex] & ((1ull << t) - 1ull))] = (unsigned short)(t | ((pi - t * K) << 8));
+        }
+        epi_bar(kEpiThreads);
+
         for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
             const bool up = (phase == 0);
             const int lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
@@ -988,29 +1010,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
                 const unsigned long long mask = s_mask[e];
-                // compacted: column c of the unit = the (colbase + c)-th token routed to the expert; lane c knows it
-                // lane l of every warp looks after column cb + l: its token, and (down projection) where its result goes
-                int cnt = TCG, tok_lane = cb + lane;
-                if constexpr (kCompact) {
-                    cnt = min(N, __popcll(mask) - colbase);
-                    // invert "rank of a token among the expert's tokens": every lane places tokens lane and lane + 32
-                    int* wtok = s_wtok + (warp - kEpiWarp0) * 32;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int t = lane + 32 * h;
-                        const int r = __popcll(mask & ((1ull << t) - 1ull)) - colbase;
-                        if (((mask >> t) & 1ull) && r >= 0 && r < N) wtok[r] = t;
-                    }
-                    __syncwarp();
-                    tok_lane = (cb + lane < cnt) ? wtok[cb + lane] : 0;
-                    __syncwarp();
-                }
+                // lane l of every warp looks after column cb + l: its token and (down projection) where its result goes
+                int cnt = TCG, tok_lane = cb + lane, yoff_lane = 0;
+                if constexpr (kCompact) cnt = min(N, __popcll(mask) - colbase);
                 auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
-                int yoff_lane = 0;                             // first element of the (token, slot) row of y for column cb + lane
-                if (!up && lane < TCG && col_on(lane)) {
-                    int sl = 0;
-                    for (int jj = 0; jj < K; ++jj) if (s_ids[tok_lane * K + jj] == e) sl = jj;
-                    yoff_lane = (tok_lane * K + sl) * H;
+                if (lane < TCG && col_on(lane)) {
+                    const int r = kCompact ? colbase + cb + lane : __popcll(mask & ((1ull << (cb + lane)) - 1ull));
+                    const unsigned pr = s_pair[s_poff[e] + r];
+                    tok_lane = (int)(pr & 0xFFu);
+                    yoff_lane = (tok_lane * K + (int)(pr >> 8)) * H;   // first element of the (token, slot) row of y
                 }
                 if (!up && entry != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert and pass)
@@ -1023,7 +1031,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if constexpr (kCompact) {
                     if (up) {
                         // input scales of this piece's K blocks, gathered for the unit's tokens: [K block][column]
-                        if (etid < N) s_utok[etid] = tok_lane;
+                        if (q == 0 && lane < TCG) s_utok[cb + lane] = tok_lane;   // each group's first warp: its columns
                         epi_bar(kEpiThreads);
                         for (int idx = etid; idx < (pend - s) * N; idx += kEpiThreads) {
                             const int c = idx & (N - 1);
