@@ -1141,6 +1141,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // (units of the down projection can be as short as two k-steps)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
+                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
                             const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
                             __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
@@ -1156,11 +1157,13 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // not the owner: park the partial accumulator, [column][row] so rows are contiguous
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
-                    for (int n = 0; n < TCG; ++n)
+                    for (int n = 0; n < TCG; ++n) {
+                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {                        // only tokens routed to this expert matter
                             __stcg(dst + (cb + n) * kBlock + row, accg[n]);
                             if (up) __stcg(dst + (N + cb + n) * kBlock + row, accu[n]);
                         }
+                    }
                     epi_bar(kEpiThreads);
                     if (etid == 0) st_release(pflag + cta, tag);
                     continue;
@@ -1184,17 +1187,20 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         if (range_lo(Sq_all, c + 1, q_all, gm) == range_lo(Sq_all, c, q_all, gm)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
-                        for (int n = 0; n < TCG; ++n)
+                        for (int n = 0; n < TCG; ++n) {
+                            if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                             if (col_on(n)) {
                                 accg[n] += __ldcg(src + (cb + n) * kBlock + row);
                                 if (up) accu[n] += __ldcg(src + (N + cb + n) * kBlock + row);
                             }
+                        }
                     }
                 }
                 if (up) {
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
+                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {                        // warp-uniform: other tokens cost nothing
                             const float g = accg[n];
                             const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
@@ -1207,6 +1213,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     epi_bar(kEpiThreads);
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
+                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
                             const float amax = fmaxf(fmaxf(s_red[cb + n], s_red[N + cb + n]), fmaxf(s_red[2 * N + cb + n], s_red[3 * N + cb + n]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
@@ -1223,6 +1230,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
+                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
                             const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
                             __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
