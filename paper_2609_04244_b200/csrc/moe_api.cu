@@ -75,6 +75,7 @@ struct moe_plan {
     unsigned long long timeout_ns;
     int split_slack_kib = 100;
     int route_all_tokens = 16;
+    int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
     int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
     int use_pdl = 1;                // programmatic dependent launch
     std::mutex mu;
@@ -84,10 +85,10 @@ struct moe_plan {
     // expert sees at most 8 tokens on average, 32 columns up to 20 on average (or whenever T <= 32); denser routing
     // of more than 32 tokens takes all tokens as columns (N = 64).
     int n_hw(int T) const {
-        if (T <= 8 || (long long)T * K <= 8ll * E) return 16;
+        if (T < compact_min || (long long)T * K <= 8ll * E) return 16;
         return (T <= 32 || (long long)T * K <= 20ll * E) ? 32 : 64;
     }
-    bool compact(int T) const { return T > 8 && n_hw(T) <= 32; }
+    bool compact(int T) const { return T >= compact_min && n_hw(T) <= 32; }
     int nr(int T) const { const int N = n_hw(T); return compact(T) ? (T + N - 1) / N * N : N; }   // token rows per expert in hq / hs
     int cap(int T) const { return T < moe::kMaxTokens ? T : moe::kMaxTokens; }
 
@@ -220,10 +221,12 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
 // Pick the kernel variant for T tokens: (MMA N, token columns read by the accumulator warps).
 int dispatch(Plan* p, int T, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx,
              const CUtensorMap& mh, const moe::Params& P, int smem_bytes, cudaStream_t stream) {
-    if (T == 1) return launch<16, 1>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (T == 2) return launch<16, 2>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
-    if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    if (!p->compact(T)) {
+        if (T == 1) return launch<16, 1>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        if (T == 2) return launch<16, 2>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    }
     if (p->n_hw(T) == 16) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (p->n_hw(T) == 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
@@ -303,6 +306,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (const char* v = getenv("MOE_B200_STAGES")) p->stages_cap = atoi(v);
     if (const char* v = getenv("MOE_B200_PDL")) p->use_pdl = atoi(v) != 0;
     if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) p->split_slack_kib = atoi(v);
+    if (const char* v = getenv("MOE_B200_COMPACT_MIN")) p->compact_min = atoi(v) < 2 ? 2 : (atoi(v) > 9 ? 9 : atoi(v));
     if (const char* v = getenv("MOE_B200_ROUTE_ALL")) p->route_all_tokens = atoi(v) < 0 ? 0 : (atoi(v) > 64 ? 64 : atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, moe::kMaxTokens);
