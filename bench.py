@@ -258,18 +258,19 @@ def main():
 
     # unique experts per layer copy (from the kernel's own routing) -> algorithmic bytes per step
     uniq = []
+    tpl = plan.tokens_per_launch()
     for l in range(L):
         d = layers[l]
         ids_all = []
-        for lo in range(0, T, 64):               # the debug entry point takes at most 64 tokens per call
-            dbg = plan.forward_debug(d["hidden"][lo:lo + 64].contiguous(), d["Wr"], d["bias"], d["W13q"], d["W13s"],
+        for lo in range(0, T, tpl):              # the debug entry point takes one launch's worth of tokens
+            dbg = plan.forward_debug(d["hidden"][lo:lo + tpl].contiguous(), d["Wr"], d["bias"], d["W13q"], d["W13s"],
                                      d["W2q"], d["W2s"])
             plan.sync_status()
             ids_all.append(dbg["ids"])
         ids_last = torch.cat(ids_all)
         uniq.append(int(torch.unique(ids_last).numel()))
     bytes_per_step = float(np.mean([wl.algorithmic_bytes(shape, T, u) for u in uniq]))
-    launches_per_step = -(-T // 64)
+    launches_per_step = -(-T // tpl)
 
     # The timed steps are replayed from CUDA graphs (Section 4.1 of the paper times graph replays): a graph holds
     # up to 1000 consecutive steps, so the host's per-call cost (Python, ctypes, launch) is not what is measured.

@@ -54,8 +54,8 @@ enum {
 
 enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID_BIAS = 1 };
 
-/* Largest number of tokens one kernel launch handles; larger T is split into launches of this size. */
-#define MOE_MAX_TOKENS_PER_LAUNCH 64
+/* Largest number of tokens one kernel launch can handle; a plan's own limit is moe_tokens_per_launch(). */
+#define MOE_MAX_TOKENS_PER_LAUNCH 128
 
 /*
  * moe_plan: fix the layer shape and routing policy (Section 3.4: shape and
@@ -88,9 +88,10 @@ int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes,
  *   hidden_bf16 [T,H] bf16          Wr_bf16 [E,H] bf16         sel_bias [E] fp32 or NULL (sigmoid policy only)
  *   W13_fp8 [E,2I,H] E4M3 bytes     W13_scale [E,2I/128,H/128] fp32
  *   W2_fp8  [E,H,I]  E4M3 bytes     W2_scale  [E,H/128,I/128] fp32
- *   out_bf16 [T,H] bf16 (written)   workspace: see moe_workspace_init; sized for >= min(T,64) tokens
+ *   out_bf16 [T,H] bf16 (written)   workspace: see moe_workspace_init; sized for >= min(T, moe_tokens_per_launch()) tokens
  * All launches that share one workspace must be ordered on the device (same stream, or events): two calls
- * that overlap on the GPU race on the scratch.  T > 64 is processed as consecutive launches of <= 64 tokens.
+ * that overlap on the GPU race on the scratch.  More tokens than moe_tokens_per_launch() are processed as
+ * consecutive launches of at most that many tokens.
  * Returns MOE_OK once the work is enqueued.
  */
 int moe_forward(moe_plan_t plan, int T,
@@ -138,7 +139,8 @@ int moe_forward_noalloc(moe_plan_t plan, int T,
 
 /*
  * moe_forward_debug: moe_forward, then copies (device to device, on `stream`) the routing and input
- * quantisation results of the step into caller buffers; any of them may be NULL.  Requires T <= 64.
+ * quantisation results of the step into caller buffers; any of them may be NULL.  Requires
+ * T <= moe_tokens_per_launch().
  *   topk_ids [T,top_k] int32 (slot order: key descending, index ascending)   topk_w [T,top_k] fp32
  *   xq [T,H] E4M3 bytes   xs [T,H/128] fp32   logits [T,E] fp32
  */
@@ -152,6 +154,10 @@ int moe_forward_debug(moe_plan_t plan, int T,
 /* Synchronise `stream`, read the workspace's device status word and return MOE_OK, MOE_ERR_TIMEOUT or
  * MOE_ERR_CUDA.  After MOE_ERR_TIMEOUT the workspace must be re-initialised. */
 int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream);
+
+/* Tokens one launch of this plan handles: 128 when the routing is sparse enough (128 * top_k <= 20 * E) for the
+ * kernel to compact each expert's tokens into its MMA columns (Eq. 9 puts tokens on the N dimension), otherwise 64. */
+int moe_tokens_per_launch(moe_plan_t plan);
 
 /* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);

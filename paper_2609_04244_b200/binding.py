@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_tokens_per_launch", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -66,6 +66,8 @@ def load_library():
     lib.moe_debug_stamps.argtypes = [vp, vp, vp, vp]
     lib.moe_plan_info.restype = i
     lib.moe_plan_info.argtypes = [vp, i] + [ctypes.POINTER(i)] * 4
+    lib.moe_tokens_per_launch.restype = i
+    lib.moe_tokens_per_launch.argtypes = [vp]
     lib.moe_plan_set_timeout_ms.restype = i
     lib.moe_plan_set_timeout_ms.argtypes = [vp, i]
     lib.moe_last_error.restype = ctypes.c_char_p
@@ -157,6 +159,10 @@ def moe_debug_stamps(plan, workspace, grid: int, stream=None):
     return buf
 
 
+def moe_tokens_per_launch(plan) -> int:
+    return int(load_library().moe_tokens_per_launch(plan))
+
+
 def moe_plan_info(plan, T: int) -> dict:
     g, s, n, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     _check(load_library().moe_plan_info(plan, T, ctypes.byref(g), ctypes.byref(s), ctypes.byref(n), ctypes.byref(b)))
@@ -205,6 +211,9 @@ class MoEPlan:
 
     def info(self, T):
         return moe_plan_info(self.handle, T)
+
+    def tokens_per_launch(self):
+        return moe_tokens_per_launch(self.handle)
 
     def close(self):
         if self.handle is not None:

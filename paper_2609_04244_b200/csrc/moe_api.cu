@@ -90,14 +90,16 @@ struct moe_plan {
     }
     bool compact(int T) const { return T >= compact_min && n_hw(T) <= 32; }
     int nr(int T) const { const int N = n_hw(T); return compact(T) ? (T + N - 1) / N * N : N; }   // token rows per expert in hq / hs
-    int cap(int T) const { return T < moe::kMaxTokens ? T : moe::kMaxTokens; }
+    // tokens per launch: 128 while 128 tokens can still be compacted (sparse routing), otherwise 64
+    int chunk() const { return compact(moe::kMaxTokens) ? moe::kMaxTokens : 64; }
+    int cap(int T) const { return T < chunk() ? T : chunk(); }
 
     WsLayout layout(int T_max) const {
         const int Tc = cap(T_max), N = n_hw(Tc), NR = nr(Tc), G = sms;
         WsLayout L;
         size_t o = 0;
         L.ctrl = o;     o += moe::kCtrlWords * 4;
-        L.e_cnt = o;    o += align_up((size_t)2 * 4 * E * 4, 256);
+        L.e_cnt = o;    o += align_up((size_t)2 * moe::kMaxPasses * E * 4, 256);
         L.dn_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
@@ -309,9 +311,9 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (const char* v = getenv("MOE_B200_COMPACT_MIN")) p->compact_min = atoi(v) < 2 ? 2 : (atoi(v) > 9 ? 9 : atoi(v));
     if (const char* v = getenv("MOE_B200_ROUTE_ALL")) p->route_all_tokens = atoi(v) < 0 ? 0 : (atoi(v) > 64 ? 64 : atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
-    const int st = p->stages_for(64, moe::kMaxTokens);
-    if (st < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
-    const int smem = moe::smem_layout(64, moe::kMaxTokens, top_k, E, H, I, st, false).total + 1024;
+    const int st = p->stages_for(64, 64);
+    if (st < 2 || p->stages_for(p->n_hw(p->chunk()), p->chunk()) < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
+    const int smem = moe::smem_layout(64, 64, top_k, E, H, I, st, false).total + 1024;
     const int optin = p->smem_optin;
     if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) ||
         !resident<16, 8>(optin, smem) || !resident<16, 4>(optin, smem) || !resident<16, 2>(optin, smem) ||
@@ -353,8 +355,8 @@ int moe_forward(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_
                 void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream) {
     int rc = check_forward_args(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, workspace);
     if (rc != MOE_OK) return rc;
-    for (int t0 = 0; t0 < T; t0 += moe::kMaxTokens) {
-        const int tc = (T - t0 < moe::kMaxTokens) ? T - t0 : moe::kMaxTokens;
+    for (int t0 = 0; t0 < T; t0 += plan->chunk()) {
+        const int tc = plan->cap(T - t0);
         rc = forward_chunk(plan, tc, static_cast<const uint16_t*>(hidden_bf16) + (size_t)t0 * plan->H, Wr_bf16, sel_bias,
                            W13_fp8, W13_scale, W2_fp8, W2_scale, static_cast<uint16_t*>(out_bf16) + (size_t)t0 * plan->H,
                            workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
@@ -378,8 +380,8 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
                         const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
                         void* out_bf16, moe_stream_t stream) {
     if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
-    if (T < 1 || T > moe::kMaxTokens)
-        return fail(MOE_ERR_ARG, "moe_forward_noalloc handles 1..%d tokens per call (got %d)", moe::kMaxTokens, T);
+    if (T < 1 || T > 64)
+        return fail(MOE_ERR_ARG, "moe_forward_noalloc handles 1..64 tokens per call (got %d)", T);
     const WsLayout L = plan->layout(T);
     if (L.total > MOE_NOALLOC_SCRATCH_BYTES)
         return fail(MOE_ERR_WORKSPACE, "this shape with T=%d needs %zu bytes of scratch; the built-in array holds %u",
@@ -432,8 +434,8 @@ int moe_forward_host(moe_plan_t plan, int T, const void* hidden_host, const void
     if (T < 1) return fail(MOE_ERR_ARG, "T must be >= 1 (got %d)", T);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* w = static_cast<uint8_t*>(workspace);
-    for (int t0 = 0; t0 < T; t0 += moe::kMaxTokens) {
-        const int tc = (T - t0 < moe::kMaxTokens) ? T - t0 : moe::kMaxTokens;
+    for (int t0 = 0; t0 < T; t0 += plan->chunk()) {
+        const int tc = plan->cap(T - t0);
         const WsLayout L = plan->layout(tc);
         if (workspace_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", workspace_bytes, L.total, tc);
         const size_t bytes = (size_t)tc * plan->H * 2;
@@ -456,7 +458,7 @@ int moe_forward_debug(moe_plan_t plan, int T, const void* hidden_bf16, const voi
                       const void* W13_fp8, const float* W13_scale, const void* W2_fp8, const float* W2_scale,
                       void* out_bf16, void* workspace, size_t workspace_bytes, moe_stream_t stream,
                       int32_t* topk_ids, float* topk_w, uint8_t* xq, float* xs, float* logits) {
-    if (plan && T > moe::kMaxTokens) return fail(MOE_ERR_ARG, "moe_forward_debug needs T <= %d", moe::kMaxTokens);
+    if (plan && T > plan->chunk()) return fail(MOE_ERR_ARG, "moe_forward_debug needs T <= %d (one launch)", plan->chunk());
     int rc = moe_forward(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, workspace,
                          workspace_bytes, stream);
     if (rc != MOE_OK) return rc;
@@ -495,6 +497,8 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
     if (e != cudaSuccess) return fail(MOE_ERR_CUDA, "CUDA error while reading stamps: %s", cudaGetErrorString(e));
     return MOE_OK;
 }
+
+int moe_tokens_per_launch(moe_plan_t plan) { return plan ? plan->chunk() : 0; }
 
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes) {
     if (!plan || T < 1) return fail(MOE_ERR_ARG, "bad arguments");

@@ -40,7 +40,8 @@ constexpr int kMaxStages = 16;
 constexpr int kATileBytes = kBlock * kBlock;  // 16 KiB of FP8
 constexpr int kMaxTopK = 32;
 constexpr int kMaxExperts = 512;
-constexpr int kMaxTokens = 64;
+constexpr int kMaxTokens = 128;       // per launch when tokens are compacted per expert; 64 when all tokens are MMA columns
+constexpr int kMaxPasses = 8;         // kMaxTokens / 16
 constexpr int kMaxTmemBufs = 8;      // accumulator buffers in TMEM (one K block each): 8 for N=16, 4 for N=32/64
 constexpr int kStampsPerCta = 16;
 
@@ -74,7 +75,7 @@ struct Params {
     float* xs;          // [T,H/128]
     uint8_t* hq;        // [E,nr,I]
     float* hs;          // [E,I/128,nr]
-    unsigned* e_cnt;    // [2][4][E] published I-blocks of an expert's intermediate tile (per launch parity and 16-token pass)
+    unsigned* e_cnt;    // [2][kMaxPasses][E] published I-blocks of an expert's intermediate tile (per launch parity and 16-token pass)
     unsigned* dn_flag;  // [grid] == tag once the CTA has stored every down-projection result of its range
     float* part_up;     // [grid][2N][128]
     float* part_dn;     // [grid][N][128]
@@ -283,7 +284,7 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
     o = (o + 7) & ~7;
-    L.mask_off = o; o += E * 8;
+    L.mask_off = o; o += E * 16;
     L.act_off = o;  o += (E + 1 + (compact ? (T * K) / N + 1 : 0)) * 4;   // + extra N-token passes of crowded experts
     L.uidx_off = o; o += E * 4;
     o = (o + 15) & ~15;
@@ -357,6 +358,19 @@ __device__ __forceinline__ int nth_set_bit(unsigned long long m, int n) {
     }
     return pos;
 }
+
+// Token sets of up to 128 tokens: two 64-bit words per expert (word 0 = tokens 0..63).
+struct TokMask { unsigned long long lo, hi; };
+__device__ __forceinline__ TokMask load_mask(const unsigned long long* s_mask, int e) { TokMask m; m.lo = s_mask[2 * e]; m.hi = s_mask[2 * e + 1]; return m; }
+__device__ __forceinline__ int mask_count(const TokMask& m) { return __popcll(m.lo) + __popcll(m.hi); }
+__device__ __forceinline__ int mask_rank(const TokMask& m, int t) {      // members below token t
+    return t < 64 ? __popcll(m.lo & ((1ull << t) - 1ull)) : __popcll(m.lo) + __popcll(m.hi & ((1ull << (t - 64)) - 1ull));
+}
+__device__ __forceinline__ int mask_nth(const TokMask& m, int n) {       // the n-th (0-based) member; needs n < count
+    const int c = __popcll(m.lo);
+    return n < c ? nth_set_bit(m.lo, n) : 64 + nth_set_bit(m.hi, n - c);
+}
+__device__ __forceinline__ void mask_add(unsigned long long* s_mask, int e, int t) { atomicOr(&s_mask[2 * e + (t >> 6)], 1ull << (t & 63)); }
 
 // monotone map float -> uint32 (larger float <=> larger integer); +0 and -0 are merged first
 __device__ __forceinline__ uint32_t orderable(float f) {
@@ -449,7 +463,7 @@ __device__ __forceinline__ void route_select(const Params& P, int t, int lane, c
         const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
         s_ids[t * K + lane] = my_id;
         s_w[t * K + lane] = w;
-        if (build_mask) atomicOr(&s_mask[my_id], 1ull << t);
+        if (build_mask) mask_add(s_mask, my_id, t);
         if (write_global) { P.ids[t * K + lane] = my_id; P.wts[t * K + lane] = w; }
     }
 }
@@ -529,7 +543,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
-    for (int e = tid; e < E; e += kThreads) s_mask[e] = 0ull;
+    for (int e = tid; e < 2 * E; e += kThreads) s_mask[e] = 0ull;
     int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
     {
         const int items = ((E + 15) / 16) * ((T + 7) / 8);
@@ -555,8 +569,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
     if (tid == 0) MOE_STAMP(0);
     const unsigned par = tag & 1u;
-    unsigned* e_cnt = P.e_cnt + par * 4 * E;                // counters of this launch: [pass][expert]
-    for (int e = cta * kThreads + tid; e < 4 * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * 4 * E + e] = 0u;
+    unsigned* e_cnt = P.e_cnt + par * kMaxPasses * E;       // counters of this launch: [pass][expert]
+    for (int e = cta * kThreads + tid; e < kMaxPasses * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * kMaxPasses * E + e] = 0u;
     if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
@@ -673,7 +687,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     const int id = __ldcg(P.ids + i);
                     s_ids[i] = id;
                     s_w[i] = __ldcg(P.wts + i);
-                    atomicOr(&s_mask[id], 1ull << div_small(i, K));
+                    mask_add(s_mask, id, div_small(i, K));
                 }
             }
             __syncthreads();
@@ -683,9 +697,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
                 const int e = e0 + lane;
-                const unsigned long long m = (e < E) ? s_mask[e] : 0ull;
+                const int mc = (e < E) ? mask_count(load_mask(s_mask, e)) : 0;
                 if constexpr (kCompact) {
-                    const int np = (__popcll(m) + N - 1) / N;      // passes of N tokens
+                    const int np = (mc + N - 1) / N;               // passes of N tokens
                     int incl = np;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
@@ -694,7 +708,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if (np) s_uidx[e] = u0;
                     base += __shfl_sync(0xffffffffu, incl, 31);
                 } else {
-                    const bool on = (m != 0ull);
+                    const bool on = (mc != 0);
                     const unsigned b = __ballot_sync(0xffffffffu, on);
                     if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
                     base += __popc(b);
@@ -783,10 +797,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if ((b_cur & 1) == 0) {
                     if (bw.e != b_entry) {
                         b_entry = bw.e;
-                        const unsigned long long m = s_mask[b_entry & 0xFFFF];
-                        const int colbase = (b_entry >> 16) * N, cnt = min(N, __popcll(m) - colbase);
+                        const TokMask m = load_mask(s_mask, b_entry & 0xFFFF);
+                        const int colbase = (b_entry >> 16) * N, cnt = min(N, mask_count(m) - colbase);
 #pragma unroll
-                        for (int i = 0; i < N / 4; ++i) tokr[i] = (r0 + 4 * i < cnt) ? nth_set_bit(m, colbase + r0 + 4 * i) : -1;
+                        for (int i = 0; i < N / 4; ++i) tokr[i] = (r0 + 4 * i < cnt) ? mask_nth(m, colbase + r0 + 4 * i) : -1;
                     }
 #pragma unroll
                     for (int i = 0; i < N / 4; ++i) {
@@ -958,7 +972,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         if (warp == kEpiWarp0) {
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
-                const int c = (e0 + lane < E) ? __popcll(s_mask[e0 + lane]) : 0;
+                const int c = (e0 + lane < E) ? mask_count(load_mask(s_mask, e0 + lane)) : 0;
                 int incl = c;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
@@ -969,7 +983,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         epi_bar(kEpiThreads);
         for (int pi = etid; pi < T * K; pi += kEpiThreads) {
             const int t = div_small(pi, K), ex = s_ids[pi];
-            s_pair[s_poff[ex] + __popcll(s_mask[ex] & ((1ull << t) - 1ull))] = (unsigned short)(t | ((pi - t * K) << 8));
+            s_pair[s_poff[ex] + mask_rank(load_mask(s_mask, ex), t)] = (unsigned short)(t | ((pi - t * K) << 8));
         }
         epi_bar(kEpiThreads);
 
@@ -1009,10 +1023,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int entry = w.e, e = entry & 0xFFFF, colbase = (entry >> 16) * N, mb = w.mb, kb0 = w.kb;
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
-                const unsigned long long mask = s_mask[e];
+                const unsigned long long mask = s_mask[2 * e];  // tokens 0..63 (all there are unless compacted)
                 // lane l of every warp looks after column cb + l: its token and (down projection) where its result goes
                 int cnt = TCG, tok_lane = cb + lane, yoff_lane = 0;
-                if constexpr (kCompact) cnt = min(N, __popcll(mask) - colbase);
+                if constexpr (kCompact) cnt = min(N, __popcll(mask) + __popcll(s_mask[2 * e + 1]) - colbase);
                 auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
                 if (lane < TCG && col_on(lane)) {
                     const int r = kCompact ? colbase + cb + lane : __popcll(mask & ((1ull << (cb + lane)) - 1ull));
@@ -1254,7 +1268,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (mine && gtid < K) {
                 // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
                 const int ex = s_ids[t * K + gtid];
-                const int ps = kCompact ? (__popcll(s_mask[ex] & ((1ull << t) - 1ull)) / N) : 0;   // the pass that holds token t
+                const int ps = kCompact ? mask_rank(load_mask(s_mask, ex), t) / N : 0;   // the pass that holds token t
                 const unsigned unit = (unsigned)((s_uidx[ex] + ps) * HB + hb);
                 const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
                 const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;

@@ -51,7 +51,9 @@ def check_against_oracle(shape, T, d, dbg, routed_scale=1.0, max_oracle_tokens=N
     exact = [t for t in range(T) if t not in ambiguous]
     np.testing.assert_allclose(g_w[exact], rt["w"][exact], rtol=2e-5, atol=1e-7)
     # --- expert path: oracle needs only the experts actually used
-    tok = list(range(T)) if max_oracle_tokens is None else list(range(min(T, max_oracle_tokens)))
+    # the oracle runs on all tokens, or on a sample spread evenly over them (first and last included)
+    tok = list(range(T)) if max_oracle_tokens is None or max_oracle_tokens >= T else \
+        sorted(set(int(x) for x in np.linspace(0, T - 1, max_oracle_tokens).round()))
     ids_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_ids, rt["ids"])[tok]
     w_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_w, rt["w"])[tok]
     used = np.unique(ids_use)

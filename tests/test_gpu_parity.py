@@ -49,17 +49,20 @@ def test_config3_routing_regimes(regime, T):
     assert r["rel_l2"] < 2e-3, r
 
 
-def test_more_than_64_tokens_is_chunked():
-    """T > 64 runs as consecutive launches of <= 64 tokens; each chunk must match the oracle and the one-call result."""
+@pytest.mark.parametrize("shape,per_launch", [(SMALL_SIG, 128), (TINY, 64)])
+def test_more_tokens_than_one_launch_is_chunked(shape, per_launch):
+    """More tokens than one launch takes (128 under sparse routing, else 64) run as consecutive launches; each chunk
+    must match the oracle and the one-call result."""
     from paper_2609_04244_b200 import MoEPlan
     from tests.parity import check_against_oracle
-    shape, T = SMALL_SIG, 100
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=per_launch + 36)
+    assert plan.tokens_per_launch() == per_launch
+    T = per_launch + 36
     d = wl.make_layer(shape, T, device="cuda")
-    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T)
     args = (d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
     full = plan.forward(d["hidden"], *args)
     plan.sync_status()
-    for lo, hi in ((0, 64), (64, 100)):
+    for lo, hi in ((0, per_launch), (per_launch, T)):
         dbg = plan.forward_debug(d["hidden"][lo:hi].contiguous(), *args)
         plan.sync_status()
         assert torch.equal(dbg["out"], full[lo:hi])
@@ -67,6 +70,13 @@ def test_more_than_64_tokens_is_chunked():
         r = check_against_oracle(shape, hi - lo, dd, dbg, max_oracle_tokens=12)
         assert r["rel_l2"] < 2e-3, r
     plan.close()
+
+
+@pytest.mark.parametrize("shape,T", [(SMALL_SIG, 128), (SMALL_SIG, 97), (RAGGED, 128)])
+def test_up_to_128_tokens_in_one_launch(shape, T):
+    """65..128 tokens in a single launch: token sets of two 64-bit words, up to eight passes of 16 compacted tokens."""
+    r = run_case(shape, T)
+    assert r["rel_l2"] < 2e-3, r
 
 
 def test_host_activation_entry_point_matches_device_entry_point():
