@@ -74,7 +74,7 @@ struct moe_plan {
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
     int split_slack_kib = 100;
-    int route_all_tokens = 16;
+    int route_all_tokens = 8;
     int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
     int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
     int use_pdl = 1;                // programmatic dependent launch

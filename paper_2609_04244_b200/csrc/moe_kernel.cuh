@@ -387,26 +387,32 @@ __device__ __forceinline__ uint32_t orderable(float f) {
 //     the orderable keys (one redux), warp-wide minimum of the indices holding it (one redux), removal of the winner;
 //     lane j keeps slot j.  The softmax normaliser is only summed when the weights are not renormalised (it cancels
 //     otherwise), with the largest logit -- slot 0 -- as the shift.
-__device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, int ksplit, int tid, int nthreads,
-                                             uint32_t* s_key, float* s_val, bool write_global) {
+// EPT elements per thread and turn, each the sum of up to KP K-split parts: EPT * KP = 16 loads in flight per thread
+// (each turn costs an L2 round trip, so few turns matter more than anything else here).
+template <int EPT, int KP>
+__device__ __forceinline__ void route_scores_t(const Params& P, int t0, int nt, int ksplit, int tid, int nthreads,
+                                               uint32_t* s_key, float* s_val, bool write_global) {
     const int E = P.E;
     const bool softmax = (P.scoring == 0);
-    for (int p0 = tid; p0 < nt * E; p0 += 2 * nthreads) {      // two elements per turn: all their loads in flight at once
-        float part[2][8];                                        // router logit = sum of the K-split parts, fixed order
-        float bias[2];
+    for (int p0 = tid; p0 < nt * E; p0 += EPT * nthreads) {
+        float part[EPT][KP];                                     // router logit = sum of the K-split parts, fixed order
+        float bias[EPT];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < EPT; ++j) {
             const int p = p0 + j * nthreads;
 #pragma unroll
-            for (int kp = 0; kp < 8; ++kp)
+            for (int kp = 0; kp < KP; ++kp)
                 part[j][kp] = (p < nt * E && kp < ksplit) ? __ldcg(P.lpart + ((size_t)kp * P.T + t0) * E + p) : 0.f;
             bias[j] = (!softmax && P.bias && p < nt * E) ? __ldg(P.bias + (p - div_small(p, E) * E)) : 0.f;
         }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < EPT; ++j) {
             const int p = p0 + j * nthreads;
             if (p < nt * E) {
-                const float l = (((part[j][0] + part[j][1]) + (part[j][2] + part[j][3])) + ((part[j][4] + part[j][5]) + (part[j][6] + part[j][7])));
+                float l;                                         // pairwise tree over the parts (absent parts are zeros)
+                if constexpr (KP == 2) l = part[j][0] + part[j][1];
+                else if constexpr (KP == 4) l = (part[j][0] + part[j][1]) + (part[j][2] + part[j][3]);
+                else l = ((part[j][0] + part[j][1]) + (part[j][2] + part[j][3])) + ((part[j][4] + part[j][5]) + (part[j][6] + part[j][7]));
                 if (write_global) P.logits[(size_t)t0 * E + p] = l;
                 if (softmax) {
                     s_val[p] = l;
@@ -419,6 +425,12 @@ __device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, in
             }
         }
     }
+}
+__device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, int ksplit, int tid, int nthreads,
+                                             uint32_t* s_key, float* s_val, bool write_global) {
+    if (ksplit <= 2) route_scores_t<8, 2>(P, t0, nt, ksplit, tid, nthreads, s_key, s_val, write_global);
+    else if (ksplit <= 4) route_scores_t<4, 4>(P, t0, nt, ksplit, tid, nthreads, s_key, s_val, write_global);
+    else route_scores_t<2, 8>(P, t0, nt, ksplit, tid, nthreads, s_key, s_val, write_global);
 }
 
 template <int NPER>
@@ -693,26 +705,38 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             __syncthreads();
         }
         if (tid == 0) MOE_STAMP(6);
-        if (warp == 0) {                                   // active list in ascending expert order: entry = expert | pass << 16
+        if constexpr (kCompact) {
+            // active list in ascending expert order, entry = expert | pass << 16 (passes of N tokens): every warp takes
+            // 32-expert chunks; the chunks' totals meet in shared memory (the idle weight ring)
+            int* s_tot = reinterpret_cast<int*>(smem);
+            const int nch = (E + 31) / 32;
+            for (int c = warp; c < nch; c += kWarps) {
+                const int e = c * 32 + lane;
+                const int np = (e < E) ? (mask_count(load_mask(s_mask, e)) + N - 1) / N : 0;
+                const int tot = __reduce_add_sync(0xffffffffu, np);
+                if (lane == 0) s_tot[c] = tot;
+            }
+            __syncthreads();
+            for (int c = warp; c < nch; c += kWarps) {
+                const int e = c * 32 + lane;
+                const int np = (e < E) ? (mask_count(load_mask(s_mask, e)) + N - 1) / N : 0;
+                int incl = np;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                const int base = __reduce_add_sync(0xffffffffu, (lane < c) ? s_tot[lane] : 0);   // nch <= 16 chunks
+                const int u0 = base + incl - np;
+                for (int ps = 0; ps < np; ++ps) s_act[u0 + ps] = e | (ps << 16);
+                if (np) s_uidx[e] = u0;
+                if (c == nch - 1 && lane == 31) { misc[1] = (uint32_t)(base + incl); s_act[base + incl] = 0; }
+            }
+        } else if (warp == 0) {                            // active list in ascending expert order
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
                 const int e = e0 + lane;
-                const int mc = (e < E) ? mask_count(load_mask(s_mask, e)) : 0;
-                if constexpr (kCompact) {
-                    const int np = (mc + N - 1) / N;               // passes of N tokens
-                    int incl = np;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-                    const int u0 = base + incl - np;
-                    for (int ps = 0; ps < np; ++ps) s_act[u0 + ps] = e | (ps << 16);
-                    if (np) s_uidx[e] = u0;
-                    base += __shfl_sync(0xffffffffu, incl, 31);
-                } else {
-                    const bool on = (mc != 0);
-                    const unsigned b = __ballot_sync(0xffffffffu, on);
-                    if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
-                    base += __popc(b);
-                }
+                const bool on = (e < E) && (s_mask[2 * e] != 0ull);
+                const unsigned b = __ballot_sync(0xffffffffu, on);
+                if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
+                base += __popc(b);
             }
             if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
         }
@@ -1258,34 +1282,50 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // unit would stall on the unit's own stores; units can be as short as two k-steps)
         epi_bar(kEpiThreads);
         if (etid == 0) { st_release(P.dn_flag + cta, tag); MOE_STAMP(13); }
-        // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block) over all CTAs
-        const int grp = (warp - kEpiWarp0) >> 2, gtid = etid & (kEpiGroupThreads - 1);
-        for (int task0 = cta * kEpiGroups; task0 < T * HB && !wt.dead; task0 += G * kEpiGroups) {
-            const int task = task0 + grp;
-            const bool mine = task < T * HB;
-            const int t = mine ? task / HB : 0, hb = mine ? task - t * HB : 0;
+        // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block): task = cta + i * G.
+        // First every (task, slot) of this CTA waits for the CTA that stored its down-projection result -- all of
+        // them in parallel, one thread each -- then the tasks are summed two at a time so that their loads overlap.
+        const int grp = (warp - kEpiWarp0) >> 2;
+        const int n_tasks = T * HB, n_mine = (cta < n_tasks) ? (n_tasks - cta + G - 1) / G : 0;
+        {
             bool got = true;
-            if (mine && gtid < K) {
+            for (int idx = etid; idx < n_mine * K; idx += kEpiThreads) {
+                const int i = div_small(idx, K), j = idx - i * K, task = cta + i * G;
+                const int t = div_small(task, HB), hb = task - t * HB;
                 // the CTA that owns unit (expert, hb) of the down projection = the one whose range holds its first k-step
-                const int ex = s_ids[t * K + gtid];
+                const int ex = s_ids[t * K + j];
                 const int ps = kCompact ? mask_rank(load_mask(s_mask, ex), t) / N : 0;   // the pass that holds token t
                 const unsigned unit = (unsigned)((s_uidx[ex] + ps) * HB + hb);
                 const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
                 const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
-                got = wt.flag(P.dn_flag + owner, tag, 7);
+                got = wt.flag(P.dn_flag + owner, tag, 7) && got;
             }
-            if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
-            if (!mine) continue;
-            float acc = 0.f;
-            const float* yp = P.y + (size_t)t * K * H + hb * kBlock + row;
+            if (!epi_all(got, kEpiThreads)) wt.dead = true;
+        }
+        for (int i0 = grp; i0 < n_mine && !wt.dead; i0 += 2 * kEpiGroups) {
+            const int i1 = i0 + kEpiGroups;
+            const bool two = i1 < n_mine;
+            const int task0 = cta + i0 * G, task1 = cta + (two ? i1 : i0) * G;
+            const int t0 = div_small(task0, HB), hb0 = task0 - t0 * HB, t1 = div_small(task1, HB), hb1 = task1 - t1 * HB;
+            const float* yp0 = P.y + (size_t)t0 * K * H + hb0 * kBlock + row;
+            const float* yp1 = P.y + (size_t)t1 * K * H + hb1 * kBlock + row;
+            float acc0 = 0.f, acc1 = 0.f;
             for (int j0 = 0; j0 < K; j0 += 8) {
-                float v[8];
+                float v0[8], v1[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (j0 + j < K) ? __ldcg(yp + (size_t)(j0 + j) * H) : 0.f;
+                for (int j = 0; j < 8; ++j) {
+                    v0[j] = (j0 + j < K) ? __ldcg(yp0 + (size_t)(j0 + j) * H) : 0.f;
+                    v1[j] = (j0 + j < K && two) ? __ldcg(yp1 + (size_t)(j0 + j) * H) : 0.f;
+                }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) if (j0 + j < K) acc = fmaf(s_w[t * K + j0 + j], v[j], acc);
+                for (int j = 0; j < 8; ++j)
+                    if (j0 + j < K) {
+                        acc0 = fmaf(s_w[t0 * K + j0 + j], v0[j], acc0);
+                        acc1 = fmaf(s_w[t1 * K + j0 + j], v1[j], acc1);
+                    }
             }
-            P.out[(size_t)t * H + hb * kBlock + row] = __float2bfloat16_rn(acc);
+            P.out[(size_t)t0 * H + hb0 * kBlock + row] = __float2bfloat16_rn(acc0);
+            if (two) P.out[(size_t)t1 * H + hb1 * kBlock + row] = __float2bfloat16_rn(acc1);
         }
         if (etid == 0) MOE_STAMP(14);
     }
