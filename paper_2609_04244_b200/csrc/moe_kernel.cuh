@@ -623,7 +623,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const uint32_t* bp = reinterpret_cast<const uint32_t*>(P.hidden + (size_t)(tok < T ? tok : 0) * H);
                 float c[4] = {0.f, 0.f, 0.f, 0.f};
                 const int k_lo = kp * kpart_len + warp * kper, k_hi = min((kp + 1) * kpart_len, k_lo + kper);
-#pragma unroll 4
+#pragma unroll 8
                 for (int k = k_lo; k < k_hi; k += 16) {
                     const int o = (k >> 1) + tq;                          // 32-bit word holding elements k+2tq, k+2tq+1
                     const uint32_t a0 = __ldg(a0p + o), a1 = __ldg(a1p + o), a2 = __ldg(a0p + o + 4), a3 = __ldg(a1p + o + 4);
@@ -670,8 +670,9 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // tokens (one warp's worth each), publish ids and weights, and everybody reads all of them after a second
         // arrival counter (two more L2 round trips).  The idle weight ring holds the keys and score values.
         const bool route_all = (T <= P.route_all_tokens) && (T * E <= 8192);
-        const int n_route_ctas = min(G, (T + kWarps - 1) / kWarps);
-        const int rt0 = route_all ? 0 : min(T, cta * kWarps), rnt = route_all ? T : min(T - rt0, kWarps);
+        const int tpc = (T + G - 1) / G;                   // tokens per selecting CTA when the grid shares them (1 up to G tokens)
+        const int n_route_ctas = (T + tpc - 1) / tpc;
+        const int rt0 = route_all ? 0 : min(T, cta * tpc), rnt = route_all ? T : min(T - rt0, tpc);
         uint32_t* s_key = reinterpret_cast<uint32_t*>(smem);
         float* s_val = reinterpret_cast<float*>(smem) + rnt * E;
         const bool wg = route_all ? (cta == 0) : true;
@@ -990,6 +991,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         int buf = 0, hs_e = -1;
         uint32_t tph = 0;
         float accg[TCG], accu[TCG];
+        // columns of the current (expert, pass): token set (first word), columns in use, and per lane the token and
+        // the y row of column cb + lane
+        int col_entry = -1, cnt = TCG, tok_lane = cb + lane, yoff_lane = 0;
+        unsigned long long mask = 0ull;
+        auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
 
         // While the first weight tiles are in flight: the routed (token, slot) pairs grouped by expert, tokens
         // ascending -- entry r of expert e is the r-th token routed to e and the top-k slot e holds for it.
@@ -1047,16 +1053,19 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int entry = w.e, e = entry & 0xFFFF, colbase = (entry >> 16) * N, mb = w.mb, kb0 = w.kb;
                 const int ustart = s - kb0, uend = ustart + KB;
                 const int pend = uend < hi ? uend : hi;
-                const unsigned long long mask = s_mask[2 * e];  // tokens 0..63 (all there are unless compacted)
-                // lane l of every warp looks after column cb + l: its token and (down projection) where its result goes
-                int cnt = TCG, tok_lane = cb + lane, yoff_lane = 0;
-                if constexpr (kCompact) cnt = min(N, __popcll(mask) + __popcll(s_mask[2 * e + 1]) - colbase);
-                auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
-                if (lane < TCG && col_on(lane)) {
-                    const int r = kCompact ? colbase + cb + lane : __popcll(mask & ((1ull << (cb + lane)) - 1ull));
-                    const unsigned pr = s_pair[s_poff[e] + r];
-                    tok_lane = (int)(pr & 0xFFu);
-                    yoff_lane = (tok_lane * K + (int)(pr >> 8)) * H;   // first element of the (token, slot) row of y
+                // lane l of every warp looks after column cb + l: its token and (down projection) where its result goes;
+                // consecutive units of a range mostly belong to the same (expert, pass), whose columns are kept
+                if (entry != col_entry) {
+                    col_entry = entry;
+                    mask = s_mask[2 * e];                      // tokens 0..63 (all there are unless compacted)
+                    cnt = TCG; tok_lane = cb + lane; yoff_lane = 0;
+                    if constexpr (kCompact) cnt = min(N, __popcll(mask) + __popcll(s_mask[2 * e + 1]) - colbase);
+                    if (lane < TCG && col_on(lane)) {
+                        const int r = kCompact ? colbase + cb + lane : __popcll(mask & ((1ull << (cb + lane)) - 1ull));
+                        const unsigned pr = s_pair[s_poff[e] + r];
+                        tok_lane = (int)(pr & 0xFFu);
+                        yoff_lane = (tok_lane * K + (int)(pr >> 8)) * H;   // first element of the (token, slot) row of y
+                    }
                 }
                 if (!up && entry != hs_e) {
                     // activation scales of this expert's intermediate tile -> shared memory (once per expert and pass)
