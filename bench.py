@@ -47,6 +47,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--config", default="c2_qwen3_30b_a3b")
+    ap.add_argument("--schedule", default="", help="schedule table written by paper_2609_04244_b200.tune (JSON)")
     ap.add_argument("--tokens", type=int, default=1)
     ap.add_argument("--regime", default="natural", choices=["natural", "same", "disjoint"])
     ap.add_argument("--layers", type=int, default=0, help="distinct layer copies to rotate over (0 = auto)")
@@ -249,7 +250,12 @@ def main():
     L = args.layers or max(2, min(16, -(-2 * 126 * 2**20 // per_step) + 1))
     L = max(1, min(L, int(0.6 * free_b // layer_bytes)))
     layers = [wl.make_layer(shape, T, regime=args.regime, layer=rank * 64 + l, device=dev) for l in range(L)]
-    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T)
+    schedule = None
+    if args.schedule:
+        import json as _json
+        with open(args.schedule) as f:
+            schedule = _json.load(f)
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T, schedule=schedule)
     info = plan.info(T)
     outs = [torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev) for _ in range(L)]
 

@@ -170,6 +170,25 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
  * done, 15 exit.  Section 3.3 of the paper argues which of these gaps must hide under the weight stream. */
 int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint64_t* host_out);
 
+/*
+ * Schedule knobs (Section 3.4: shape and schedule are fixed ahead of time; the paper finds its schedule with an
+ * offline search, and so does paper_2609_04244_b200/tune.py through these two calls).  T = 0 sets a per-token-count
+ * knob for every token count; the last two knobs are plan-wide and ignore T.  Changing MOE_KNOB_COMPACT_MIN changes
+ * which kernel variant a token count gets and with it the scratch layout: query moe_workspace_bytes() again.
+ *   MOE_KNOB_STAGES            pipeline stages of the shared-memory ring; 0 = as many as fit (default)
+ *   MOE_KNOB_SPLIT_SLACK_KIB   keep a projection's units whole while that costs the busiest CTA at most this many KiB
+ *                              of extra weight stream, split them across CTAs (split-K) otherwise (default 100)
+ *   MOE_KNOB_ROUTE_ALL_TOKENS  up to this many tokens every CTA selects the experts of all tokens; beyond, the grid
+ *                              shares the tokens and exchanges the result (default 8)
+ *   MOE_KNOB_COMPACT_MIN       fewest tokens (2..9) for which each expert's tokens are compacted into its MMA columns (9)
+ *   MOE_KNOB_PDL               programmatic dependent launch on/off (1)
+ * Results do not depend on STAGES, ROUTE_ALL_TOKENS or PDL; SPLIT_SLACK_KIB and COMPACT_MIN change the order of fp32
+ * partial sums (never the routing or the quantised input).
+ */
+enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4 };
+int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value);
+int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value);
+
 /* Set the device-side wait limit in milliseconds (default 1000).  A wait that runs out makes the kernel
  * record MOE_ERR_TIMEOUT and return; it never traps. */
 int moe_plan_set_timeout_ms(moe_plan_t plan, int ms);

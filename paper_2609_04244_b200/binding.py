@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_tokens_per_launch", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_tokens_per_launch", "moe_plan_set_knob", "moe_plan_get_knob", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -66,6 +66,10 @@ def load_library():
     lib.moe_debug_stamps.argtypes = [vp, vp, vp, vp]
     lib.moe_plan_info.restype = i
     lib.moe_plan_info.argtypes = [vp, i] + [ctypes.POINTER(i)] * 4
+    lib.moe_plan_set_knob.restype = i
+    lib.moe_plan_set_knob.argtypes = [vp, i, i, i]
+    lib.moe_plan_get_knob.restype = i
+    lib.moe_plan_get_knob.argtypes = [vp, i, i, ctypes.POINTER(i)]
     lib.moe_tokens_per_launch.restype = i
     lib.moe_tokens_per_launch.argtypes = [vp]
     lib.moe_plan_set_timeout_ms.restype = i
@@ -159,6 +163,20 @@ def moe_debug_stamps(plan, workspace, grid: int, stream=None):
     return buf
 
 
+KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4}
+
+
+def moe_plan_set_knob(plan, T: int, knob, value: int) -> None:
+    """Set a schedule knob (name from KNOBS or its number) for token count T (0 = every token count)."""
+    _check(load_library().moe_plan_set_knob(plan, int(T), KNOBS.get(knob, knob), int(value)))
+
+
+def moe_plan_get_knob(plan, T: int, knob) -> int:
+    v = ctypes.c_int()
+    _check(load_library().moe_plan_get_knob(plan, int(T), KNOBS.get(knob, knob), ctypes.byref(v)))
+    return v.value
+
+
 def moe_tokens_per_launch(plan) -> int:
     return int(load_library().moe_tokens_per_launch(plan))
 
@@ -172,11 +190,39 @@ def moe_plan_info(plan, T: int) -> dict:
 class MoEPlan:
     """Owns a plan handle and a workspace sized for `T_max` tokens on the current CUDA device."""
 
-    def __init__(self, H, E, I, top_k, scoring=SCORE_SOFTMAX, renorm=1, routed_scale=1.0, T_max=64):
+    def __init__(self, H, E, I, top_k, scoring=SCORE_SOFTMAX, renorm=1, routed_scale=1.0, T_max=64, schedule=None):
         self.H, self.E, self.I, self.top_k = H, E, I, top_k
+        self.T_max = T_max
         self.handle = moe_plan(H, E, I, top_k, scoring, renorm, routed_scale)
-        self.workspace = torch.empty(moe_workspace_bytes(self.handle, T_max), dtype=torch.uint8, device="cuda")
-        moe_workspace_init(self.handle, self.workspace)
+        self.workspace = None
+        if schedule:
+            self.apply_schedule(schedule)
+        self._size_workspace()
+
+    def _size_workspace(self):
+        need = moe_workspace_bytes(self.handle, self.T_max)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(need, dtype=torch.uint8, device="cuda")
+            moe_workspace_init(self.handle, self.workspace)
+
+    def set_knob(self, T, knob, value):
+        """Schedule knob for token count T (0 = all); the scratch is re-sized if the knob changes its layout."""
+        torch.cuda.synchronize()
+        moe_plan_set_knob(self.handle, T, knob, value)
+        if self.workspace is not None:
+            self._size_workspace()
+
+    def get_knob(self, T, knob):
+        return moe_plan_get_knob(self.handle, T, knob)
+
+    def apply_schedule(self, schedule):
+        """Apply a schedule table as written by paper_2609_04244_b200.tune: {"plan": {knob: value}, "per_tokens":
+        {"T": {knob: value}}}; unknown token counts keep the defaults."""
+        for knob, value in schedule.get("plan", {}).items():
+            self.set_knob(0, knob, value)
+        for T, knobs in schedule.get("per_tokens", {}).items():
+            for knob, value in knobs.items():
+                self.set_knob(int(T), knob, value)
 
     def forward(self, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, out=None, stream=None):
         T = hidden.shape[0]

@@ -73,11 +73,15 @@ struct moe_plan {
     float routed_scale;
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
-    int split_slack_kib = 100;
-    int route_all_tokens = 8;
+    // schedule knobs (Section 3.4: fixed ahead of time; moe_plan_set_knob / the offline tuner change them)
+    int split_slack_kib[moe::kMaxTokens + 1];   // per token count: whole units vs split-K (see range_quantum)
+    int route_all_tokens[moe::kMaxTokens + 1];  // per token count: largest T for which every CTA routes all tokens
+    int stages_cap[moe::kMaxTokens + 1];        // per token count: 0 = as many pipeline stages as shared memory holds
     int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
-    int stages_cap = 0;             // 0 = as many pipeline stages as shared memory holds
     int use_pdl = 1;                // programmatic dependent launch
+    moe_plan() {
+        for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = 100; route_all_tokens[t] = 8; stages_cap[t] = 0; }
+    }
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
 
@@ -123,7 +127,8 @@ struct moe_plan {
     }
 
     int stages_for(int N, int T) const {
-        for (int s = (stages_cap > 0 && stages_cap < moe::kMaxStages) ? stages_cap : moe::kMaxStages; s >= 2; --s) {
+        const int cap_s = stages_cap[T <= moe::kMaxTokens ? T : moe::kMaxTokens];
+        for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s) {
             const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s, compact(T));
             if (L.total + 1024 <= smem_optin) return s;
         }
@@ -190,8 +195,8 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.T = T; P.H = p->H; P.E = p->E; P.I = p->I; P.K = p->K; P.scoring = p->scoring; P.renorm = p->renorm;
     P.routed_scale = p->routed_scale;
     P.stages = stages;
-    P.split_slack_kib = p->split_slack_kib;
-    P.route_all_tokens = p->route_all_tokens;
+    P.split_slack_kib = p->split_slack_kib[T];
+    P.route_all_tokens = p->route_all_tokens[T];
     P.nr = p->nr(T);
     P.grid_magic = (1ull << 40) / (unsigned long long)p->sms + 1ull;
     P.timeout_ns = p->timeout_ns;
@@ -275,6 +280,49 @@ extern "C" {
 
 const char* moe_last_error(void) { return g_err; }
 
+int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
+    if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (T < 0 || T > moe::kMaxTokens) return fail(MOE_ERR_ARG, "T must be 0 (all token counts) or 1..%d", moe::kMaxTokens);
+    const int lo = T ? T : 0, hi = T ? T : moe::kMaxTokens;
+    switch (knob) {
+        case MOE_KNOB_STAGES:
+            if (value != 0 && (value < 2 || value > moe::kMaxStages)) return fail(MOE_ERR_ARG, "stages must be 0 (as many as fit) or 2..%d", moe::kMaxStages);
+            for (int t = lo; t <= hi; ++t) plan->stages_cap[t] = value;
+            return MOE_OK;
+        case MOE_KNOB_SPLIT_SLACK_KIB:
+            if (value < 0 || value > (1 << 20)) return fail(MOE_ERR_ARG, "split slack out of range");
+            for (int t = lo; t <= hi; ++t) plan->split_slack_kib[t] = value;
+            return MOE_OK;
+        case MOE_KNOB_ROUTE_ALL_TOKENS:
+            if (value < 0 || value > 64) return fail(MOE_ERR_ARG, "route-all token count must be 0..64");
+            for (int t = lo; t <= hi; ++t) plan->route_all_tokens[t] = value;
+            return MOE_OK;
+        case MOE_KNOB_COMPACT_MIN:
+            if (value < 2 || value > 9) return fail(MOE_ERR_ARG, "compaction threshold must be 2..9 tokens");
+            plan->compact_min = value;
+            return MOE_OK;
+        case MOE_KNOB_PDL:
+            plan->use_pdl = value != 0;
+            return MOE_OK;
+        default:
+            return fail(MOE_ERR_ARG, "unknown knob %d", knob);
+    }
+}
+
+int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
+    if (!plan || !value) return fail(MOE_ERR_ARG, "plan or value is NULL");
+    if (T < 0 || T > moe::kMaxTokens) return fail(MOE_ERR_ARG, "T must be 0..%d", moe::kMaxTokens);
+    const int t = T ? T : 1;
+    switch (knob) {
+        case MOE_KNOB_STAGES: *value = plan->stages_cap[t]; return MOE_OK;
+        case MOE_KNOB_SPLIT_SLACK_KIB: *value = plan->split_slack_kib[t]; return MOE_OK;
+        case MOE_KNOB_ROUTE_ALL_TOKENS: *value = plan->route_all_tokens[t]; return MOE_OK;
+        case MOE_KNOB_COMPACT_MIN: *value = plan->compact_min; return MOE_OK;
+        case MOE_KNOB_PDL: *value = plan->use_pdl; return MOE_OK;
+        default: return fail(MOE_ERR_ARG, "unknown knob %d", knob);
+    }
+}
+
 int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float routed_scale, moe_plan_t* out) {
     if (!out) return fail(MOE_ERR_ARG, "out is NULL");
     *out = nullptr;
@@ -305,11 +353,12 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     p->smem_optin = (int)prop.sharedMemPerBlockOptin;
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
     // schedule overrides for experiments (the paper tunes its schedule offline, Section 3.4)
-    if (const char* v = getenv("MOE_B200_STAGES")) p->stages_cap = atoi(v);
-    if (const char* v = getenv("MOE_B200_PDL")) p->use_pdl = atoi(v) != 0;
-    if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) p->split_slack_kib = atoi(v);
-    if (const char* v = getenv("MOE_B200_COMPACT_MIN")) p->compact_min = atoi(v) < 2 ? 2 : (atoi(v) > 9 ? 9 : atoi(v));
-    if (const char* v = getenv("MOE_B200_ROUTE_ALL")) p->route_all_tokens = atoi(v) < 0 ? 0 : (atoi(v) > 64 ? 64 : atoi(v));
+    // environment overrides for experiments (the same knobs moe_plan_set_knob sets)
+    if (const char* v = getenv("MOE_B200_STAGES")) moe_plan_set_knob(p, 0, MOE_KNOB_STAGES, atoi(v));
+    if (const char* v = getenv("MOE_B200_PDL")) moe_plan_set_knob(p, 0, MOE_KNOB_PDL, atoi(v));
+    if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_SLACK_KIB, atoi(v));
+    if (const char* v = getenv("MOE_B200_COMPACT_MIN")) moe_plan_set_knob(p, 0, MOE_KNOB_COMPACT_MIN, atoi(v));
+    if (const char* v = getenv("MOE_B200_ROUTE_ALL")) moe_plan_set_knob(p, 0, MOE_KNOB_ROUTE_ALL_TOKENS, atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, 64);
     if (st < 2 || p->stages_for(p->n_hw(p->chunk()), p->chunk()) < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
