@@ -164,7 +164,7 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
 
 /* Diagnostics: synchronise `stream` and copy the phase time stamps of the last launch on this workspace to
  * HOST memory host_out[grid*16] (nanoseconds of the GPU's global timer).  Per CTA: 0 start, 1 input quantised,
- * 2 router logits done, 3 arrived at the routing flag, 4 routing published grid-wide, 5 scales cached,
+ * 2 router logits done, 3 arrived at the routing flag, 4 routing published grid-wide, 5 selection keys ready,
  * 6 top-k done, 7 routing metadata done, 8 first weight tile requested, 9 first ring of requests issued,
  * 10 first weight tile landed, 11 first accumulator read, 12 up phase done, 13 down phase done, 14 reduction
  * done, 15 exit.  Section 3.3 of the paper argues which of these gaps must hide under the weight stream. */

@@ -667,7 +667,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // input scales, transposed to [K block][token]: the first load is issued here and consumed after the routing loads
         const float xs0 = (tid < T * KBu) ? __ldcg(P.xs + tid) : 0.f;
         // few tokens: every CTA selects for all of them (no second grid-wide wait); many tokens: CTAs share the
-        // tokens (one warp's worth each), publish ids and weights, and everybody reads all of them after a second
+        // tokens (one each, up to the grid size), publish ids and weights, and everybody reads all of them after a second
         // arrival counter (two more L2 round trips).  The idle weight ring holds the keys and score values.
         const bool route_all = (T <= P.route_all_tokens) && (T * E <= 8192);
         const int tpc = (T + G - 1) / G;                   // tokens per selecting CTA when the grid shares them (1 up to G tokens)
@@ -680,6 +680,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         if (tid < T * KBu) { const int tt = div_small(tid, KBu); s_xs[(tid - tt * KBu) * TS + tt] = xs0; }
         for (int i = tid + kThreads; i < T * KBu; i += kThreads) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
         __syncthreads();
+        if (tid == 0) MOE_STAMP(5);
         for (int tl = warp; tl < rnt; tl += kWarps) {
             const int t = rt0 + tl;
             if (E <= 128) route_select<4>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
