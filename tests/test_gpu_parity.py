@@ -37,13 +37,14 @@ def test_config2_qwen3_like(T):
     assert r["rel_l2"] < 2e-3, r
 
 
-@pytest.mark.parametrize("regime,T", [("same", 4), ("disjoint", 4), ("disjoint", 32), ("natural", 64), ("same", 40), ("same", 64)])
+@pytest.mark.parametrize("regime,T", [("same", 4), ("disjoint", 4), ("disjoint", 32), ("natural", 64), ("same", 40), ("same", 64),
+                                      ("natural", 128), ("same", 128)])
 def test_config3_routing_regimes(regime, T):
     """Natural, maximum-reuse and maximum-bytes routing; 40 and 64 tokens on the same 8 experts walk each expert in
-    three and four passes of 16 compacted tokens."""
+    three and four passes of 16 compacted tokens, 128 tokens in eight."""
     r = run_case(wl.SHAPES["c2_qwen3_30b_a3b"], T, regime=regime, max_oracle_tokens=8)
-    if regime == "same":
-        assert r["unique_experts"] == 8
+    if regime == "same":      # (at 128 tokens the forcing term of the generator no longer wins for every token)
+        assert r["unique_experts"] == 8 if T <= 64 else r["unique_experts"] <= 16
     if regime == "disjoint":
         assert r["unique_experts"] == min(128, 8 * T)
     assert r["rel_l2"] < 2e-3, r
