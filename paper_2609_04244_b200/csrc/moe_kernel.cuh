@@ -678,7 +678,16 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const bool wg = route_all ? (cta == 0) : true;
         route_scores(P, rt0, rnt, ksplit, tid, kThreads, s_key, s_val, wg);
         if (tid < T * KBu) { const int tt = div_small(tid, KBu); s_xs[(tid - tt * KBu) * TS + tt] = xs0; }
-        for (int i = tid + kThreads; i < T * KBu; i += kThreads) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
+        for (int i0 = tid + kThreads; i0 < T * KBu; i0 += 8 * kThreads) {          // the rest, eight loads in flight per thread
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (i0 + j * kThreads < T * KBu) ? __ldcg(P.xs + i0 + j * kThreads) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = i0 + j * kThreads;
+                if (i < T * KBu) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = v[j]; }
+            }
+        }
         __syncthreads();
         if (tid == 0) MOE_STAMP(5);
         for (int tl = warp; tl < rnt; tl += kWarps) {
@@ -697,11 +706,20 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             __syncthreads();
             alive = (misc[2] != 0u);
             if (alive) {
-                for (int i = tid; i < T * K; i += kThreads) {
-                    const int id = __ldcg(P.ids + i);
-                    s_ids[i] = id;
-                    s_w[i] = __ldcg(P.wts + i);
-                    mask_add(s_mask, id, div_small(i, K));
+                for (int i0 = tid; i0 < T * K; i0 += 4 * kThreads) {                 // eight loads in flight per thread
+                    int id[4];
+                    float wv[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int i = i0 + j * kThreads;
+                        id[j] = (i < T * K) ? __ldcg(P.ids + i) : 0;
+                        wv[j] = (i < T * K) ? __ldcg(P.wts + i) : 0.f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int i = i0 + j * kThreads;
+                        if (i < T * K) { s_ids[i] = id[j]; s_w[i] = wv[j]; mask_add(s_mask, id[j], div_small(i, K)); }
+                    }
                 }
             }
             __syncthreads();
