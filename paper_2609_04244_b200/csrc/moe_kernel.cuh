@@ -16,11 +16,12 @@
 //
 // Warp roles (Section 3.3, warp specialisation): warps 0 and 2 = TMA producers (weight tiles,
 // activation tiles), warps 1 and 3 = tcgen05 MMA issuers (even and odd k-steps), warps 4..7 = accumulator/epilogue warps (one TMEM lane
-// quadrant each); all eight warps share phase R.  Weights are the MMA "A"
-// operand (M = 128 weight rows), the whole token tile is the "B" operand with
-// N = 16/32/64 (Eq. 9), K = 32 per instruction, four instructions per 128-wide
-// K block; each K block is accumulated in TMEM on its own and scaled by
-// (weight block scale x activation group scale) in registers.
+// quadrant each; twice that for 32/64 token columns); all warps share phase R.  Weights are the MMA "A"
+// operand (M = 128 weight rows), tokens are the "B" operand with N = 16/32/64 (Eq. 9), K = 32 per instruction,
+// four instructions per 128-wide K block; each K block is accumulated in TMEM on its own and scaled by
+// (weight block scale x activation group scale) in registers.  Up to 8 tokens the B columns are the step's tokens;
+// beyond that, under sparse routing, the columns of a unit are the tokens routed to the unit's expert (compacted:
+// gathered activation tile, compact intermediate tile, passes of N tokens for crowded experts).
 #pragma once
 
 #include <cuda.h>
