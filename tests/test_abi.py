@@ -47,3 +47,13 @@ def test_plan_argument_validation_happens_before_any_device_work():
     assert b"H and I" in lib.moe_last_error() or len(lib.moe_last_error()) > 0
     assert lib.moe_workspace_bytes(None, 4) == 0
     assert lib.moe_forward(None, 1, *([None] * 9), 0, None) == -1
+
+
+def test_plan_helpers_reject_a_null_plan_without_touching_a_device():
+    lib = binding.load_library()
+    v = ctypes.c_int(-5)
+    assert lib.moe_plan_set_knob(None, 0, 0, 4) == -1
+    assert lib.moe_plan_get_knob(None, 0, 0, ctypes.byref(v)) == -1 and v.value == -5
+    assert lib.moe_tokens_per_launch(None) == 0
+    assert lib.moe_workspace_bytes(None, 8) == 0
+    assert b"NULL" in lib.moe_last_error()
