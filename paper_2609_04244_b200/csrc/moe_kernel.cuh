@@ -521,8 +521,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
-    constexpr int kTmemBufs = (N == 16) ? 8 : 4;                 // 8 x 32 = 256, 4 x 64 = 256, 4 x 128 = 512 columns
-    constexpr int kBufShift = (N == 16) ? 3 : 2;
+    constexpr int kTmemBufs = (N <= 32) ? 8 : 4;                 // 8 x 32 = 256, 8 x 64 = 512, 4 x 128 = 512 columns
+    constexpr int kBufShift = (N <= 32) ? 3 : 2;
     const uint32_t bar_fullb = smem_u32(bars + 2 * kMaxStages);  // activation tile landed (second producer)
     const uint32_t bar_tfull = smem_u32(bars + 3 * kMaxStages), bar_tempty = smem_u32(bars + 3 * kMaxStages + kMaxTmemBufs);
     const uint32_t bar_drain = smem_u32(bars + 3 * kMaxStages + 2 * kMaxTmemBufs);
@@ -545,7 +545,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     // launch was not made with the programmatic-serialization attribute).
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // Set-up that touches only this CTA's shared and tensor memory runs before the wait on the previous launch.
-    constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 128/256/512
+    constexpr uint32_t kTmemCols = kTmemBufs * 2 * N;            // buffers x (gate N + up N) columns: 256/512/512
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq); tma_prefetch_desc(&tmHq);
         for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, kCompact ? 32 : 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -1004,6 +1004,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
         const int cb = ((warp - kEpiWarp0) >> 2) * TCG;        // first token column of this accumulator group
+        // column of register slot n: the group's columns in order -- except in the 32-column compacted variant, where
+        // the two groups take alternating blocks of 8 columns: the columns in use are the first `cnt`, and this way both
+        // groups share them (slots in use stay contiguous from 0: a group's second block fills only after its first)
+        constexpr bool kInterleave = kCompact && kEpiGroups == 2;
+        auto colx = [&](int n) -> int { return kInterleave ? ((n & 8) << 1) + (cb >> 1) + (n & 7) : cb + n; };
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         volatile uint32_t* s_giveup = misc + 3;
         bool first_acc = true;
@@ -1012,10 +1017,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         uint32_t tph = 0;
         float accg[TCG], accu[TCG];
         // columns of the current (expert, pass): token set (first word), columns in use, and per lane the token and
-        // the y row of column cb + lane
-        int col_entry = -1, cnt = TCG, tok_lane = cb + lane, yoff_lane = 0;
+        // the y row of column colx(lane)
+        int col_entry = -1, cnt = TCG, tok_lane = colx(lane), yoff_lane = 0;
         unsigned long long mask = 0ull;
-        auto col_on = [&](int n) -> bool { return kCompact ? (cb + n < cnt) : (bool)((mask >> (cb + n)) & 1ull); };
+        auto col_on = [&](int n) -> bool { return kCompact ? (colx(n) < cnt) : (bool)((mask >> (colx(n))) & 1ull); };
 
         // While the first weight tiles are in flight: the routed (token, slot) pairs grouped by expert, tokens
         // ascending -- entry r of expert e is the r-th token routed to e and the top-k slot e holds for it.
@@ -1078,10 +1083,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (entry != col_entry) {
                     col_entry = entry;
                     mask = s_mask[2 * e];                      // tokens 0..63 (all there are unless compacted)
-                    cnt = TCG; tok_lane = cb + lane; yoff_lane = 0;
+                    cnt = TCG; tok_lane = colx(lane); yoff_lane = 0;
                     if constexpr (kCompact) cnt = min(N, __popcll(mask) + __popcll(s_mask[2 * e + 1]) - colbase);
                     if (lane < TCG && col_on(lane)) {
-                        const int r = kCompact ? colbase + cb + lane : __popcll(mask & ((1ull << (cb + lane)) - 1ull));
+                        const int r = kCompact ? colbase + colx(lane) : __popcll(mask & ((1ull << (colx(lane))) - 1ull));
                         const unsigned pr = s_pair[s_poff[e] + r];
                         tok_lane = (int)(pr & 0xFFu);
                         yoff_lane = (tok_lane * K + (int)(pr >> 8)) * H;   // first element of the (token, slot) row of y
@@ -1098,7 +1103,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if constexpr (kCompact) {
                     if (up) {
                         // input scales of this piece's K blocks, gathered for the unit's tokens: [K block][column]
-                        if (q == 0 && lane < TCG) s_utok[cb + lane] = tok_lane;   // each group's first warp: its columns
+                        if (q == 0 && lane < TCG) s_utok[colx(lane)] = tok_lane;   // each group's first warp: its columns
                         epi_bar(kEpiThreads);
                         for (int idx = etid; idx < (pend - s) * N; idx += kEpiThreads) {
                             const int c = idx & (N - 1);
@@ -1129,39 +1134,44 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     if constexpr (kCompact) {
                         // one load as wide as the routed columns need (warp-uniform): a TMEM load costs about the
                         // same whatever its width
-                        const int need = cnt - cb;
+                        // slots in use: the group's columns below cnt
+                        const int need = kInterleave ? min(8, max(0, cnt - (cb >> 1))) + min(8, max(0, cnt - 16 - (cb >> 1))) : cnt - cb;
                         if (need <= 4) {
-                            tmem_ld<4>(tcol + cb, dg);
-                            if (up) tmem_ld<4>(tcol + N + cb, du);
+                            tmem_ld<4>(tcol + colx(0), dg);
+                            if (up) tmem_ld<4>(tcol + N + colx(0), du);
                         } else if (need <= 8) {
-                            tmem_ld<8>(tcol + cb, dg);
-                            if (up) tmem_ld<8>(tcol + N + cb, du);
+                            tmem_ld<8>(tcol + colx(0), dg);
+                            if (up) tmem_ld<8>(tcol + N + colx(0), du);
+                        } else if constexpr (kInterleave) {
+                            tmem_ld<8>(tcol + colx(0), dg);
+                            tmem_ld<8>(tcol + colx(8), dg + 8);
+                            if (up) { tmem_ld<8>(tcol + N + colx(0), du); tmem_ld<8>(tcol + N + colx(8), du + 8); }
                         } else {
-                            tmem_ld<16>(tcol + cb, dg);
-                            if (up) tmem_ld<16>(tcol + N + cb, du);
+                            tmem_ld<16>(tcol + colx(0), dg);
+                            if (up) tmem_ld<16>(tcol + N + colx(0), du);
                         }
                     } else {
 #pragma unroll
                         for (int c = 0; c < TCG; c += CH) {
-                            tmem_ld<CH>(tcol + cb + c, dg + c);
-                            if (up) tmem_ld<CH>(tcol + N + cb + c, du + c);
+                            tmem_ld<CH>(tcol + colx(c), dg + c);
+                            if (up) tmem_ld<CH>(tcol + N + colx(c), du + c);
                         }
                     }
                 };
                 auto add_scaled = [&](const float* dg, const float* du, float wsg, float wsu, int i) {
 #pragma unroll
                     for (int c = 0; c < TCG; c += CH) {
-                        if (kCompact && cb + c >= cnt) break;
+                        if (kCompact && colx(c) >= cnt) break;
                         float as[CH];
                         if constexpr (CH >= 4) {
 #pragma unroll
                             for (int jj = 0; jj < CH; jj += 4) {
-                                const float4 v = *reinterpret_cast<const float4*>(as_p + i * as_step + cb + c + jj);
+                                const float4 v = *reinterpret_cast<const float4*>(as_p + i * as_step + colx(c) + jj);
                                 as[jj] = v.x; as[jj + 1] = v.y; as[jj + 2] = v.z; as[jj + 3] = v.w;
                             }
                         } else {
 #pragma unroll
-                            for (int jj = 0; jj < CH; ++jj) as[jj] = as_p[i * as_step + cb + c + jj];
+                            for (int jj = 0; jj < CH; ++jj) as[jj] = as_p[i * as_step + colx(c) + jj];
                         }
 #pragma unroll
                         for (int jj = 0; jj < CH; ++jj) {
@@ -1208,7 +1218,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // (units of the down projection can be as short as two k-steps)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                        if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
                             const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
                             __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
@@ -1225,10 +1235,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     float* dst = part + (size_t)cta * pcols * kBlock;
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                        if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {                        // only tokens routed to this expert matter
-                            __stcg(dst + (cb + n) * kBlock + row, accg[n]);
-                            if (up) __stcg(dst + (N + cb + n) * kBlock + row, accu[n]);
+                            __stcg(dst + (colx(n)) * kBlock + row, accg[n]);
+                            if (up) __stcg(dst + (N + colx(n)) * kBlock + row, accu[n]);
                         }
                     }
                     epi_bar(kEpiThreads);
@@ -1255,10 +1265,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TCG; ++n) {
-                            if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                            if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                             if (col_on(n)) {
-                                accg[n] += __ldcg(src + (cb + n) * kBlock + row);
-                                if (up) accu[n] += __ldcg(src + (N + cb + n) * kBlock + row);
+                                accg[n] += __ldcg(src + (colx(n)) * kBlock + row);
+                                if (up) accu[n] += __ldcg(src + (N + colx(n)) * kBlock + row);
                             }
                         }
                     }
@@ -1267,27 +1277,27 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // SiLU(gate)*up, 128-wide amax, FP8 requantisation, one global store  (Section 3.3)
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                        if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {                        // warp-uniform: other tokens cost nothing
                             const float g = accg[n];
                             const float a = __fdiv_rn(g, 1.0f + expf(-g)) * accu[n];
                             accg[n] = a;
                             // |a| as an integer orders like the float: one warp-wide integer max instead of a shuffle tree
                             const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a)));
-                            if (lane == 0) s_red[q * N + cb + n] = __uint_as_float(m);
+                            if (lane == 0) s_red[q * N + colx(n)] = __uint_as_float(m);
                         }
                     }
                     epi_bar(kEpiThreads);
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                        if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
-                            const float amax = fmaxf(fmaxf(s_red[cb + n], s_red[N + cb + n]), fmaxf(s_red[2 * N + cb + n], s_red[3 * N + cb + n]));
+                            const float amax = fmaxf(fmaxf(s_red[colx(n)], s_red[N + colx(n)]), fmaxf(s_red[2 * N + colx(n)], s_red[3 * N + colx(n)]));
                             const float sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
                             const float2 v = make_float2(__fdiv_rn(accg[n], sc), 0.f);
                             const uint8_t code = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
-                            P.hq[((size_t)e * P.nr + colbase + cb + n) * I + mb * kBlock + row] = code;
-                            if (row == 0) P.hs[((size_t)e * IB + mb) * P.nr + colbase + cb + n] = sc;
+                            P.hq[((size_t)e * P.nr + colbase + colx(n)) * I + mb * kBlock + row] = code;
+                            if (row == 0) P.hs[((size_t)e * IB + mb) * P.nr + colbase + colx(n)] = sc;
                         }
                     }
                     fence_proxy_async();
@@ -1297,7 +1307,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     // per-slot result of this expert for its routed tokens
 #pragma unroll
                     for (int n = 0; n < TCG; ++n) {
-                        if (kCompact && cb + n >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
+                        if (kCompact && colx(n) >= cnt) break;               // compacted columns are contiguous: stop at the first unused one
                         if (col_on(n)) {
                             const int yo = __shfl_sync(0xffffffffu, yoff_lane, n);
                             __stcg(P.y + (size_t)yo + mb * kBlock + row, accg[n]);
