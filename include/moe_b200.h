@@ -179,7 +179,8 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *   MOE_KNOB_SPLIT_SLACK_KIB   keep a projection's units whole while that costs the busiest CTA at most this many KiB
  *                              of extra weight stream, split them across CTAs (split-K) otherwise (default 100)
  *   MOE_KNOB_ROUTE_ALL_TOKENS  up to this many tokens every CTA selects the experts of all tokens; beyond, the grid
- *                              shares the tokens and exchanges the result (default 8)
+ *                              shares the tokens and exchanges the result (default 8; up to 8 tokens every CTA always
+ *                              selects for all of them, so smaller values act as 8)
  *   MOE_KNOB_COMPACT_MIN       fewest tokens (2..9) for which each expert's tokens are compacted into its MMA columns (9)
  *   MOE_KNOB_PDL               programmatic dependent launch on/off (1)
  * Results do not depend on STAGES, ROUTE_ALL_TOKENS or PDL; SPLIT_SLACK_KIB and COMPACT_MIN change the order of fp32

@@ -670,7 +670,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // few tokens: every CTA selects for all of them (no second grid-wide wait); many tokens: CTAs share the
         // tokens (one each, up to the grid size), publish ids and weights, and everybody reads all of them after a second
         // arrival counter (two more L2 round trips).  The idle weight ring holds the keys and score values.
-        const bool route_all = (T <= P.route_all_tokens) && (T * E <= 8192);
+        constexpr bool kAlwaysAll = (TC <= 8);             // the token-column variants serve at most 8 tokens: no shared routing code in them
+        const bool route_all = kAlwaysAll || ((T <= P.route_all_tokens) && (T * E <= 8192));
         const int tpc = (T + G - 1) / G;                   // tokens per selecting CTA when the grid shares them (1 up to G tokens)
         const int n_route_ctas = (T + tpc - 1) / tpc;
         const int rt0 = route_all ? 0 : min(T, cta * tpc), rnt = route_all ? T : min(T - rt0, tpc);
@@ -698,7 +699,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             else route_select<16>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
         }
         __syncthreads();
-        if (!route_all) {
+        if (!kAlwaysAll && !route_all) {
             if (tid == 0) {
                 if (cta < n_route_ctas) red_release_add(P.ctrl + kRouteCnt2 + par, 1u);
                 const bool ok = wt.flag(P.ctrl + kRouteCnt2 + par, (unsigned)n_route_ctas, 12);

@@ -32,7 +32,7 @@ REL_L2_REJECT = 2e-3
 PER_TOKEN_GRID = {
     "split_slack_kib": [0, 50, 100, 200, 400],
     "stages": [0, 8, 6],
-    "route_all_tokens": [4, 8, 16],
+    "route_all_tokens": [8, 16, 32],
 }
 PLAN_GRID = {"compact_min": [9, 5]}
 
@@ -79,7 +79,7 @@ def _rel_l2(a, b):
 def relevant_knobs(T, per_launch):
     """Knobs that can matter for T tokens: the route-all threshold only where it changes the routing mode."""
     grid = dict(PER_TOKEN_GRID)
-    if not 4 < min(T, per_launch) <= 16:
+    if not 8 < min(T, per_launch) <= 32:
         grid["route_all_tokens"] = [8]
     return grid
 
