@@ -526,7 +526,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const uint32_t bar_fullb = smem_u32(bars + 2 * kMaxStages);  // activation tile landed (second producer)
     const uint32_t bar_tfull = smem_u32(bars + 3 * kMaxStages), bar_tempty = smem_u32(bars + 3 * kMaxStages + kMaxTmemBufs);
     const uint32_t bar_drain = smem_u32(bars + 3 * kMaxStages + 2 * kMaxTmemBufs);
-    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] routing published, [3] give-up flag of the accumulator warps
+    uint32_t* misc = (uint32_t*)(smem + L.misc_off);  // [0] tmem base, [1] U, [2] routing published, [3] give-up flag of the accumulator warps, [4],[5] k-steps issued by the two MMA issuers
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
@@ -552,7 +552,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4 * kEpiGroups); }
         mbar_init(bar_drain, 1);
         mbar_init(bar_drain + 16, 1);
-        misc[3] = 0u;
+        misc[3] = 0u; misc[4] = 0u; misc[5] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
@@ -940,9 +940,14 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         __syncwarp();
     }
     // ------------------------------------------------------------------ role: MMA issuers
-    // Two issuing threads (warp 1: even k-steps, warp 3: odd k-steps), each with its own TMEM buffers (k-step mod 4)
+    // Two issuing threads (warp 1: even k-steps, warp 3: odd k-steps), each with its own TMEM buffers (k-step mod 8)
     // and its own commits: issuing four tcgen05.mma per 16 KiB tile from one thread alone costs more time than the
     // tile takes to arrive from HBM.
+    // The two share the stage ring, and a stage's previous user may have been the other issuer.  A parity wait cannot
+    // tell "my phase is complete" from "the phase before the previous one is complete", so an issuer that runs ahead
+    // (tiles land out of order) must not wait on a stage whose previous phase the other issuer has not seen complete:
+    // each publishes the number of k-steps it has issued, and nobody gets S/2 or more k-steps ahead of the other (a
+    // lap of the ring is at least S/2 k-steps, so the previous user of any of my stages is then done with them).
     else if (warp == 1 || warp == 3) {
         if (lane == 0 && alive) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
@@ -953,12 +958,25 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             uint32_t ph = 0;                     // full-barrier parity of stage `st`
             auto advance = [&](int n) { st += n; while (st >= S) { st -= S; ph ^= 1u; } };
             bool first = true;
+            int other_seen = 0;                  // k-steps the other issuer was last seen to have issued
             if (who == 1) advance(n_up > 0 ? 2 : 1);               // skip k-step 0
             for (int ks = who; ks < n_up + n_dn && !wt.dead; ks += 2) {
                 const bool up = ks < n_up;
                 const int buf = ks & (kTmemBufs - 1);
                 const uint32_t tph = (uint32_t)((ks >> kBufShift) & 1) ^ 1u;
                 if (!wt.mbar(bar_tempty + 8 * buf, tph, 3)) break;
+                {
+                    // the other issuer's k-steps up to q = ks - S/2 must be issued: the last of them is q or q - 1
+                    const int q = ks - (S >> 1);
+                    const int thr = ((q & 1) != who) ? q + 1 : q;                      // its progress count once that one is issued
+                    if (other_seen < thr) {                                             // (re-read only when the cached count is too old)
+                        volatile uint32_t* other = misc + 4 + (who ^ 1);
+                        bool ok = true;
+                        for (uint32_t i = 1; (other_seen = (int)*other) < thr; ++i)
+                            if ((i & 255u) == 0 && wt.expired(13)) { ok = false; break; }
+                        if (!ok) break;
+                    }
+                }
                 const int st0 = st;
                 const uint32_t ph0 = ph;
                 const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)L.stage_bytes;
@@ -989,6 +1007,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     umma_commit(bar_empty + 8 * st0);
                 }
                 umma_commit(bar_tfull + 8 * buf);              // accumulator of this K block complete
+                *(volatile uint32_t*)(misc + 4 + who) = (uint32_t)(ks + 1);     // every k-step below ks + 1 of mine is issued
                 // move past the rest of this k-step and the other issuer's k-step
                 advance(1);
                 if (ks + 1 < n_up + n_dn) advance(ks + 1 < n_up ? 2 : 1);
