@@ -175,7 +175,9 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  * offline search, and so does paper_2609_04244_b200/tune.py through these two calls).  T = 0 sets a per-token-count
  * knob for every token count; the last two knobs are plan-wide and ignore T.  Changing MOE_KNOB_COMPACT_MIN changes
  * which kernel variant a token count gets and with it the scratch layout: query moe_workspace_bytes() again.
- *   MOE_KNOB_STAGES            pipeline stages of the shared-memory ring; 0 = as many as fit (default)
+ *   MOE_KNOB_STAGES            pipeline stages of the shared-memory ring, 2..16 (capped by what fits); 0 = the
+ *                              library's choice for the token count (default): 6 or 8 for short weight streams, all
+ *                              that fit for steps of a few tiles and for long streams
  *   MOE_KNOB_SPLIT_SLACK_KIB   keep a projection's units whole while that costs the busiest CTA at most this many KiB
  *                              of extra weight stream, split them across CTAs (split-K) otherwise (default 100)
  *   MOE_KNOB_ROUTE_ALL_TOKENS  up to this many tokens every CTA selects the experts of all tokens; beyond, the grid

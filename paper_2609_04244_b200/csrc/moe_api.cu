@@ -2,6 +2,7 @@
 #include "moe_kernel.cuh"
 
 #include <cstdarg>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -79,6 +80,7 @@ struct moe_plan {
     int stages_cap[moe::kMaxTokens + 1];        // per token count: 0 = as many pipeline stages as shared memory holds
     int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
     int use_pdl = 1;                // programmatic dependent launch
+    int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
     moe_plan() {
         for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = 100; route_all_tokens[t] = 8; stages_cap[t] = 0; }
     }
@@ -126,8 +128,22 @@ struct moe_plan {
         return L;
     }
 
+    // Default depth of the stage ring when the knob is 0.  Measured on this machine (config 2 and the paper's shapes,
+    // T = 1..64, ring depths 12/10/8/6): a CTA whose whole step is a handful of tiles wants every tile requested at
+    // once; short streams run 2-7 % faster on a ring of 6, medium ones 1-2 % faster on 8; long streams want all the
+    // depth that fits.  "Length" = weight tiles per CTA for the expected number of distinct experts (text after Eq. 5).
+    int default_stages(int T) const {
+        const double U = E * (1.0 - std::pow(1.0 - (double)K / E, (double)T));
+        const double tiles = 3.0 * U * (I / 128) * (H / 128) / sms;
+        if (tiles <= 18.0) return 0;
+        if (tiles <= 105.0) return 6;
+        if (tiles <= 450.0) return 8;
+        return 0;
+    }
+
     int stages_for(int N, int T) const {
-        const int cap_s = stages_cap[T <= moe::kMaxTokens ? T : moe::kMaxTokens];
+        int cap_s = stages_cap[T <= moe::kMaxTokens ? T : moe::kMaxTokens];
+        if (cap_s == 0 && auto_stages) cap_s = default_stages(T);
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s) {
             const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s, compact(T));
             if (L.total + 1024 <= smem_optin) return s;
@@ -356,6 +372,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     // environment overrides for experiments (the same knobs moe_plan_set_knob sets)
     if (const char* v = getenv("MOE_B200_STAGES")) moe_plan_set_knob(p, 0, MOE_KNOB_STAGES, atoi(v));
     if (const char* v = getenv("MOE_B200_PDL")) moe_plan_set_knob(p, 0, MOE_KNOB_PDL, atoi(v));
+    if (const char* v = getenv("MOE_B200_AUTO_STAGES")) p->auto_stages = atoi(v) != 0;
     if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_SLACK_KIB, atoi(v));
     if (const char* v = getenv("MOE_B200_COMPACT_MIN")) moe_plan_set_knob(p, 0, MOE_KNOB_COMPACT_MIN, atoi(v));
     if (const char* v = getenv("MOE_B200_ROUTE_ALL")) moe_plan_set_knob(p, 0, MOE_KNOB_ROUTE_ALL_TOKENS, atoi(v));

@@ -31,7 +31,7 @@ REL_L2_REJECT = 2e-3
 
 PER_TOKEN_GRID = {
     "split_slack_kib": [0, 50, 100, 200, 400],
-    "stages": [0, 8, 6],
+    "stages": [0, 16, 8, 6],
     "route_all_tokens": [8, 16, 32],
 }
 PLAN_GRID = {"compact_min": [9, 5]}
