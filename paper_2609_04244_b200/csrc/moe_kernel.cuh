@@ -1042,8 +1042,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         unsigned long long mask = 0ull;
         auto col_on = [&](int n) -> bool { return kCompact ? (colx(n) < cnt) : (bool)((mask >> (colx(n))) & 1ull); };
 
-        // While the first weight tiles are in flight: the routed (token, slot) pairs grouped by expert, tokens
-        // ascending -- entry r of expert e is the r-th token routed to e and the top-k slot e holds for it.
+        // The routed (token, slot) pairs grouped by expert, tokens ascending -- entry r of expert e is the r-th token
+        // routed to e and the top-k slot e holds for it.  The compacted variants need it from the first up unit on and
+        // build it while the first weight tiles are in flight; the others only need it for the down projection and
+        // build it while they wait for the first intermediate tile to be published.
+        auto build_pairs = [&]() {
         if (warp == kEpiWarp0) {
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
@@ -1061,6 +1064,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             s_pair[s_poff[ex] + mask_rank(load_mask(s_mask, ex), t)] = (unsigned short)(t | ((pi - t * K) << 8));
         }
         epi_bar(kEpiThreads);
+        };
+        if constexpr (kCompact) build_pairs();
 
         for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
             const bool up = (phase == 0);
@@ -1072,6 +1077,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const int pcols = up ? 2 * N : N;
             if (!up && etid == 0) MOE_STAMP(12);
             if (hi <= lo) continue;
+            if (!kCompact && !up) { build_pairs(); col_entry = -1; }
             Walk w;
             w.init(lo, KB, MB, s_act);
 
@@ -1105,7 +1111,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     mask = s_mask[2 * e];                      // tokens 0..63 (all there are unless compacted)
                     cnt = TCG; tok_lane = colx(lane); yoff_lane = 0;
                     if constexpr (kCompact) cnt = min(N, __popcll(mask) + __popcll(s_mask[2 * e + 1]) - colbase);
-                    if (lane < TCG && col_on(lane)) {
+                    if ((kCompact || !up) && lane < TCG && col_on(lane)) {
                         const int r = kCompact ? colbase + colx(lane) : __popcll(mask & ((1ull << (colx(lane))) - 1ull));
                         const unsigned pr = s_pair[s_poff[e] + r];
                         tok_lane = (int)(pr & 0xFFu);
