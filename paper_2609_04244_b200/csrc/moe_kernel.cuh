@@ -1349,7 +1349,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         if (etid == 0) { st_release(P.dn_flag + cta, tag); MOE_STAMP(13); }
         // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block): task = cta + i * G.
         // First every (task, slot) of this CTA waits for the CTA that stored its down-projection result -- all of
-        // them in parallel, one thread each -- then the tasks are summed two at a time so that their loads overlap.
+        // them in parallel, one thread each -- then the tasks are summed two (four for 16 token columns and more) at a time so that their loads overlap.
         const int grp = (warp - kEpiWarp0) >> 2;
         const int n_tasks = T * HB, n_mine = (cta < n_tasks) ? (n_tasks - cta + G - 1) / G : 0;
         {
@@ -1367,30 +1367,36 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
             if (!epi_all(got, kEpiThreads)) wt.dead = true;
         }
-        for (int i0 = grp; i0 < n_mine && !wt.dead; i0 += 2 * kEpiGroups) {
-            const int i1 = i0 + kEpiGroups;
-            const bool two = i1 < n_mine;
-            const int task0 = cta + i0 * G, task1 = cta + (two ? i1 : i0) * G;
-            const int t0 = div_small(task0, HB), hb0 = task0 - t0 * HB, t1 = div_small(task1, HB), hb1 = task1 - t1 * HB;
-            const float* yp0 = P.y + (size_t)t0 * K * H + hb0 * kBlock + row;
-            const float* yp1 = P.y + (size_t)t1 * K * H + hb1 * kBlock + row;
-            float acc0 = 0.f, acc1 = 0.f;
-            for (int j0 = 0; j0 < K; j0 += 8) {
-                float v0[8], v1[8];
+        constexpr int RT = (TC >= 16) ? 4 : 2;                 // tasks summed together: RT x 8 loads in flight per thread
+        for (int i0 = grp; i0 < n_mine && !wt.dead; i0 += RT * kEpiGroups) {
+            int tt[RT], hh[RT];
+            const float* yp[RT];
+            float acc[RT];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    v0[j] = (j0 + j < K) ? __ldcg(yp0 + (size_t)(j0 + j) * H) : 0.f;
-                    v1[j] = (j0 + j < K && two) ? __ldcg(yp1 + (size_t)(j0 + j) * H) : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (j0 + j < K) {
-                        acc0 = fmaf(s_w[t0 * K + j0 + j], v0[j], acc0);
-                        acc1 = fmaf(s_w[t1 * K + j0 + j], v1[j], acc1);
-                    }
+            for (int r = 0; r < RT; ++r) {
+                const int i = i0 + r * kEpiGroups;
+                const int task = cta + (i < n_mine ? i : i0) * G;  // (absent tasks repeat the first: loads stay legal, nothing is stored)
+                tt[r] = div_small(task, HB);
+                hh[r] = task - tt[r] * HB;
+                yp[r] = P.y + (size_t)tt[r] * K * H + hh[r] * kBlock + row;
+                acc[r] = 0.f;
             }
-            P.out[(size_t)t0 * H + hb0 * kBlock + row] = __float2bfloat16_rn(acc0);
-            if (two) P.out[(size_t)t1 * H + hb1 * kBlock + row] = __float2bfloat16_rn(acc1);
+            for (int j0 = 0; j0 < K; j0 += 8) {
+                float v[RT][8];
+#pragma unroll
+                for (int r = 0; r < RT; ++r)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        v[r][j] = (j0 + j < K && i0 + r * kEpiGroups < n_mine) ? __ldcg(yp[r] + (size_t)(j0 + j) * H) : 0.f;
+#pragma unroll
+                for (int r = 0; r < RT; ++r)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j0 + j < K) acc[r] = fmaf(s_w[tt[r] * K + j0 + j], v[r][j], acc[r]);
+            }
+#pragma unroll
+            for (int r = 0; r < RT; ++r)
+                if (i0 + r * kEpiGroups < n_mine) P.out[(size_t)tt[r] * H + hh[r] * kBlock + row] = __float2bfloat16_rn(acc[r]);
         }
         if (etid == 0) MOE_STAMP(14);
     }
