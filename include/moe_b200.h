@@ -173,7 +173,7 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
 /*
  * Schedule knobs (Section 3.4: shape and schedule are fixed ahead of time; the paper finds its schedule with an
  * offline search, and so does paper_2609_04244_b200/tune.py through these two calls).  T = 0 sets a per-token-count
- * knob for every token count; the last two knobs are plan-wide and ignore T.  Changing MOE_KNOB_COMPACT_MIN changes
+ * knob for every token count; COMPACT_MIN and PDL are plan-wide and ignore T.  Changing MOE_KNOB_COMPACT_MIN changes
  * which kernel variant a token count gets and with it the scratch layout: query moe_workspace_bytes() again.
  *   MOE_KNOB_STAGES            pipeline stages of the shared-memory ring, 2..16 (capped by what fits); 0 = the
  *                              library's choice for the token count (default): 6 or 8 for short weight streams, all
@@ -185,10 +185,16 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              selects for all of them, so smaller values act as 8)
  *   MOE_KNOB_COMPACT_MIN       fewest tokens (2..9) for which each expert's tokens are compacted into its MMA columns (9)
  *   MOE_KNOB_PDL               programmatic dependent launch on/off (1)
- * Results do not depend on STAGES, ROUTE_ALL_TOKENS or PDL; SPLIT_SLACK_KIB and COMPACT_MIN change the order of fp32
- * partial sums (never the routing or the quantised input).
+ *   MOE_KNOB_SPLIT_WEIGHT      where tokens are compacted: cut the k-step lists into per-CTA ranges of equal WEIGHT, a
+ *                              k-step of an expert with many tokens weighing more (its epilogue work grows with the
+ *                              columns in use), instead of ranges of equal length.  0 = equal length, 1..8 = strength
+ *                              of the per-column term in quarters of the fitted value, -1 = the library's choice
+ *                              (default: 4 from 24 tokens on, from 16 where I <= 256, else 0)
+ * Results do not depend on STAGES, ROUTE_ALL_TOKENS or PDL; SPLIT_SLACK_KIB, COMPACT_MIN and SPLIT_WEIGHT change the
+ * order of fp32 partial sums (never the routing or the quantised input).
  */
-enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4 };
+enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4,
+       MOE_KNOB_SPLIT_WEIGHT = 5 };
 int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value);
 int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value);
 

@@ -163,7 +163,7 @@ def moe_debug_stamps(plan, workspace, grid: int, stream=None):
     return buf
 
 
-KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4}
+KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4, "split_weight": 5}
 
 
 def moe_plan_set_knob(plan, T: int, knob, value: int) -> None:

@@ -75,6 +75,7 @@ struct moe_plan {
     int device, sms, smem_optin;
     unsigned long long timeout_ns;
     // schedule knobs (Section 3.4: fixed ahead of time; moe_plan_set_knob / the offline tuner change them)
+    int split_weight[moe::kMaxTokens + 1];      // compacted variants: per-column cost in the range split, quarters of the fitted weight (0 off .. 8; -1 = library's choice)
     int split_slack_kib[moe::kMaxTokens + 1];   // per token count: whole units vs split-K (see range_quantum)
     int route_all_tokens[moe::kMaxTokens + 1];  // per token count: largest T for which every CTA routes all tokens
     int stages_cap[moe::kMaxTokens + 1];        // per token count: 0 = as many pipeline stages as shared memory holds
@@ -82,7 +83,7 @@ struct moe_plan {
     int use_pdl = 1;                // programmatic dependent launch
     int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
     moe_plan() {
-        for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = 100; route_all_tokens[t] = 8; stages_cap[t] = 0; }
+        for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
     }
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
@@ -95,6 +96,15 @@ struct moe_plan {
         return (T <= 32 || (long long)T * K <= 20ll * E) ? 32 : 64;
     }
     bool compact(int T) const { return T >= compact_min && n_hw(T) <= 32; }
+    // ranges of equal weight (instead of equal k-step counts) where tokens are compacted and experts can be crowded
+    // (its set-up costs about a microsecond; it pays from two dozen tokens on, earlier where the experts' slices are
+    // so short -- I <= 256 -- that the per-column epilogue work is a large share of a unit)
+    int split_weight_for(int T) const {
+        if (!compact(T)) return 0;
+        if (split_weight[T] >= 0) return split_weight[T];
+        return (T >= 24 || (T >= 16 && I <= 256)) ? 4 : 0;
+    }
+    bool weighted(int T) const { return split_weight_for(T) > 0; }
     int nr(int T) const { const int N = n_hw(T); return compact(T) ? (T + N - 1) / N * N : N; }   // token rows per expert in hq / hs
     // tokens per launch: 128 while 128 tokens can still be compacted (sparse routing), otherwise 64
     int chunk() const { return compact(moe::kMaxTokens) ? moe::kMaxTokens : 64; }
@@ -145,7 +155,7 @@ struct moe_plan {
         int cap_s = stages_cap[T <= moe::kMaxTokens ? T : moe::kMaxTokens];
         if (cap_s == 0 && auto_stages) cap_s = default_stages(T);
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s) {
-            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s, compact(T));
+            const moe::SmemLayout L = moe::smem_layout(N, T, K, E, H, I, s, compact(T), weighted(T));
             if (L.total + 1024 <= smem_optin) return s;
         }
         return 0;
@@ -169,12 +179,12 @@ using Plan = struct moe_plan;
 
 namespace {
 
-template <int N, int TC>
+template <int N, int TC, bool WS = false>
 int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx, const CUtensorMap& mh,
            const moe::Params& P, int smem_bytes, cudaStream_t stream) {
     static int configured_device = -1;
     if (configured_device != p->device) {
-        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
+        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
             return fail(MOE_ERR_CUDA, "cudaFuncSetAttribute(max dynamic smem) failed: %s", cudaGetErrorString(cudaGetLastError()));
         configured_device = p->device;
     }
@@ -188,17 +198,17 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
     attr[0].val.programmaticStreamSerializationAllowed = 1;            // kernel's tail; the kernel itself waits for it
     cfg.attrs = attr;
     cfg.numAttrs = p->use_pdl ? 1 : 0;
-    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_decode_kernel<N, TC>, m13, m2, mx, mh, P);
+    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_decode_kernel<N, TC, WS>, m13, m2, mx, mh, P);
     if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
     return MOE_OK;
 }
 
-template <int N, int TC>
+template <int N, int TC, bool WS = false>
 bool resident(int smem_optin, int smem_bytes) {
     int blocks = 0;
-    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return false;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, moe::moe_decode_kernel<N, TC>, 128 + 128 * (TC >= 32 ? 2 : 1), smem_bytes) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return false;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, moe::moe_decode_kernel<N, TC, WS>, 128 + 128 * (TC >= 32 ? 2 : 1), smem_bytes) != cudaSuccess) return false;
     return blocks >= 1;
 }
 
@@ -212,6 +222,7 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.routed_scale = p->routed_scale;
     P.stages = stages;
     P.split_slack_kib = p->split_slack_kib[T];
+    P.split_weight = p->split_weight_for(T);
     P.route_all_tokens = p->route_all_tokens[T];
     P.nr = p->nr(T);
     P.grid_magic = (1ull << 40) / (unsigned long long)p->sms + 1ull;
@@ -250,6 +261,10 @@ int dispatch(Plan* p, int T, const CUtensorMap& m13, const CUtensorMap& m2, cons
         if (T <= 4) return launch<16, 4>(p, m13, m2, mx, mh, P, smem_bytes, stream);
         if (T <= 8) return launch<16, 8>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     }
+    if (p->weighted(T)) {
+        if (p->n_hw(T) == 16) return launch<16, 16, true>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+        return launch<32, 32, true>(p, m13, m2, mx, mh, P, smem_bytes, stream);
+    }
     if (p->n_hw(T) == 16) return launch<16, 16>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     if (p->n_hw(T) == 32) return launch<32, 32>(p, m13, m2, mx, mh, P, smem_bytes, stream);
     return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
@@ -263,7 +278,7 @@ int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const floa
     if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
     const int stages = p->stages_for(N, T);
     if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages, p->compact(T));
+    const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages, p->compact(T), p->weighted(T));
     uint8_t* w = static_cast<uint8_t*>(ws);
 
     CUtensorMap m13, m2, mx, mh;
@@ -320,6 +335,10 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
         case MOE_KNOB_PDL:
             plan->use_pdl = value != 0;
             return MOE_OK;
+        case MOE_KNOB_SPLIT_WEIGHT:
+            if (value < -1 || value > 8) return fail(MOE_ERR_ARG, "split weight must be -1 (library's choice), 0 (off) or 1..8");
+            for (int t = lo; t <= hi; ++t) plan->split_weight[t] = value;
+            return MOE_OK;
         default:
             return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
@@ -335,6 +354,7 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_ROUTE_ALL_TOKENS: *value = plan->route_all_tokens[t]; return MOE_OK;
         case MOE_KNOB_COMPACT_MIN: *value = plan->compact_min; return MOE_OK;
         case MOE_KNOB_PDL: *value = plan->use_pdl; return MOE_OK;
+        case MOE_KNOB_SPLIT_WEIGHT: *value = plan->split_weight[t]; return MOE_OK;
         default: return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
 }
@@ -350,6 +370,11 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
         const long long ks = (long long)E * (H / 128) * (I / 128);
         if (ks * 256 >= (1ll << 31) || (long long)E * 2 * I * H / 128 >= (1ll << 31))
             return fail(MOE_ERR_SHAPE, "layer too large for 32-bit k-step indices");
+        // weighted range split of the compacted variants: a k-step weighs < 256, a unit list holds up to
+        // E + kMaxTokens * top_k / 16 virtual experts, one virtual expert's weight goes through div_small()
+        const long long per_expert = (long long)(H / 128) * (I / 128);
+        if (per_expert * 256 >= (1ll << 22) || (ks + (long long)(moe::kMaxTokens * top_k / 16 + 1) * per_expert) * 256 >= (1ll << 32))
+            return fail(MOE_ERR_SHAPE, "layer too large for the 32-bit range weights");
     }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
@@ -365,7 +390,7 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     p->H = H; p->E = E; p->I = I; p->K = top_k; p->scoring = scoring; p->renorm = renorm ? 1 : 0;
     p->routed_scale = routed_scale;
     p->device = dev;
-    p->sms = prop.multiProcessorCount;
+    p->sms = prop.multiProcessorCount < moe::kMaxGrid ? prop.multiProcessorCount : moe::kMaxGrid;   // one CTA per SM, up to the size of the kernel's range tables
     p->smem_optin = (int)prop.sharedMemPerBlockOptin;
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
     // schedule overrides for experiments (the paper tunes its schedule offline, Section 3.4)
@@ -375,13 +400,14 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (const char* v = getenv("MOE_B200_AUTO_STAGES")) p->auto_stages = atoi(v) != 0;
     if (const char* v = getenv("MOE_B200_SPLIT_SLACK_KIB")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_SLACK_KIB, atoi(v));
     if (const char* v = getenv("MOE_B200_COMPACT_MIN")) moe_plan_set_knob(p, 0, MOE_KNOB_COMPACT_MIN, atoi(v));
+    if (const char* v = getenv("MOE_B200_SPLIT_WEIGHT")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_WEIGHT, atoi(v));
     if (const char* v = getenv("MOE_B200_ROUTE_ALL")) moe_plan_set_knob(p, 0, MOE_KNOB_ROUTE_ALL_TOKENS, atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, 64);
     if (st < 2 || p->stages_for(p->n_hw(p->chunk()), p->chunk()) < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
-    const int smem = moe::smem_layout(64, 64, top_k, E, H, I, st, false).total + 1024;
+    const int smem = moe::smem_layout(64, 64, top_k, E, H, I, st, false, false).total + 1024;
     const int optin = p->smem_optin;
-    if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) ||
+    if (!resident<64, 64>(optin, smem) || !resident<32, 32>(optin, smem) || !resident<16, 16>(optin, smem) || !resident<32, 32, true>(optin, smem) || !resident<16, 16, true>(optin, smem) ||
         !resident<16, 8>(optin, smem) || !resident<16, 4>(optin, smem) || !resident<16, 2>(optin, smem) ||
         !resident<16, 1>(optin, smem)) {
         delete p;
@@ -479,7 +505,7 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     const int N = plan->n_hw(T);
     const int stages = plan->stages_for(N, T);
     if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages, plan->compact(T));
+    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages, plan->compact(T), plan->weighted(T));
     uint8_t* w = static_cast<uint8_t*>(ws);
     CUtensorMap m13, m2, mx, mh;       // encoded on the stack: no descriptor cache, nothing allocated
     if (!encode_2d(&m13, W13_fp8, (uint64_t)plan->E * 2 * plan->I, plan->H, 128) ||
@@ -572,7 +598,7 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
     if (grid) *grid = plan->sms;
     if (stages) *stages = st;
     if (n_hw) *n_hw = N;
-    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st, plan->compact(Tc)).total + 1024;
+    if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st, plan->compact(Tc), plan->weighted(Tc)).total + 1024;
     return MOE_OK;
 }
 

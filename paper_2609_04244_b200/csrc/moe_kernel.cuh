@@ -43,8 +43,10 @@ constexpr int kMaxTopK = 32;
 constexpr int kMaxExperts = 512;
 constexpr int kMaxTokens = 128;       // per launch when tokens are compacted per expert; 64 when all tokens are MMA columns
 constexpr int kMaxPasses = 8;         // kMaxTokens / 16
+constexpr int kMaxUnits = kMaxExperts + kMaxTokens * kMaxTopK / 16;   // virtual experts (expert, pass) of one launch
 constexpr int kMaxTmemBufs = 8;      // accumulator buffers in TMEM (one K block each): 8 for N=16, 4 for N=32/64
 constexpr int kStampsPerCta = 16;
+constexpr int kMaxGrid = 255;         // CTAs the weighted range tables of the compacted variants can hold
 
 // control words at the head of the workspace
 // (the two arrival counters are used by alternate launches: a launch counts in one and clears the other)
@@ -57,6 +59,7 @@ struct Params {
     float routed_scale;
     int stages;
     int split_slack_kib;            // see range_quantum()
+    int split_weight;               // compacted variants: weight of the per-column cost in the range split, in quarters (0: equal k-steps)
     int route_all_tokens;           // up to this many tokens every CTA selects for all of them
     int nr;                         // token rows per expert in hq / hs: the MMA N, or T rounded up to 16 when tokens are compacted per expert
     unsigned long long grid_magic;  // floor(2^40 / grid) + 1: division by the grid size as a multiplication
@@ -273,9 +276,9 @@ struct Waiter {
 // shared-memory layout
 // ---------------------------------------------------------------------------------------------
 struct SmemLayout {
-    int ring_off, stage_bytes, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, poff_off, pair_off, misc_off, total;
+    int ring_off, stage_bytes, lo_off, kw_off, pv_off, pv_stride, bar_off, ids_off, w_off, mask_off, act_off, uidx_off, xs_off, hs_off, as_off, red_off, poff_off, pair_off, misc_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages, bool compact) {
+__host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, int H, int I, int stages, bool compact, bool weighted) {
     SmemLayout L;
     L.stage_bytes = kATileBytes + N * kBlock;
     L.ring_off = 0;
@@ -295,6 +298,10 @@ __host__ __device__ inline SmemLayout smem_layout(int N, int T, int K, int E, in
     L.red_off = o;  o += kMaxWarps * 64 * 4;        // cross-warp reduction scratch
     L.poff_off = o; o += E * 4;                     // expert -> first entry of its (token, slot) pairs
     L.pair_off = o; o += ((T * K * 2 + 15) & ~15);  // (token | slot << 8) of every routed pair, grouped by expert, tokens ascending
+    L.lo_off = o;   o += weighted ? 2 * (kMaxGrid + 1) * 4 : 0;   // weighted ranges: first k-step of every CTA's range, per projection
+    L.kw_off = o;   o += weighted ? 2 * 33 * 4 : 0;               // weighted ranges: weight of a k-step by columns in use, per projection
+    L.pv_stride = E + (T * K) / N + 2;                           // weighted ranges: weight of the k-steps before every virtual expert, per projection
+    L.pv_off = o;   o += weighted ? 2 * L.pv_stride * 4 : 0;
     L.total = o;
     return L;
 }
@@ -313,6 +320,21 @@ __device__ __forceinline__ int div_small(int a, int d) {          // 0 <= a < 2^
     return q;
 }
 __device__ __forceinline__ int range_lo(int Sq, int c, int q, unsigned long long magic) { return (int)div_grid((unsigned)Sq * (unsigned)c, magic) * q; }
+
+// Ranges of equal weight (compacted variants): `pv[u]` = weight of all k-steps before virtual expert u, pv[U] the total,
+// every virtual expert holding n_u k-steps of equal weight.  The range of CTA c starts at the first k-step whose
+// preceding weight reaches total * c / G.  Rounded toward zero throughout: the target stays below the total and grows
+// with c; every CTA computes the same values, which is all the split needs.
+__device__ __forceinline__ unsigned split_target(unsigned total, int c, float rG) {
+    return __float2uint_rz(__uint2float_rz(total) * (__int2float_rz(c) * rG));
+}
+__device__ __forceinline__ int split_point(const unsigned* pv, int a, unsigned target, int n_u, int KB, int q) {   // a = largest u with pv[u] <= target
+    const int w = div_small((int)(pv[a + 1] - pv[a]), n_u);
+    const int j = min(n_u, div_small((int)(target - pv[a]) + w - 1, w));
+    int lo = a * n_u + j;
+    if (q != 1) lo = div_small(lo, KB) * KB;                                     // whole units only
+    return lo;
+}
 
 // Split a projection's units across CTAs (split-K, partial sums exchanged through L2) or keep units whole?
 // Whole units cost no exchange but load the busiest CTA with ceil(units/G) units; take them when that surplus,
@@ -493,9 +515,11 @@ __device__ __forceinline__ uint32_t quant4(float x0, float x1, float x2, float x
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // N  = MMA N (token tile, 16/32/64); TC = token columns the accumulator warps actually read (power of two >= T).
+// WS = ranges of equal weight instead of equal k-step counts (compacted variants only; a variant of its own because
+//      even unexecuted code in the accumulator loops costs the small-batch cases a microsecond or two).
 // ---------------------------------------------------------------------------------------------
 // Accumulator warps: one group of 4 warps for TC <= 16, two groups (each half of the token columns) for TC >= 32.
-template <int N, int TC>
+template <int N, int TC, bool WS = false>
 __global__ void __launch_bounds__(128 + 128 * (TC >= 32 ? 2 : 1), 1)
 moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                   const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ CUtensorMap tmHq,
@@ -516,7 +540,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock, KBd = IB;
     const int S = P.stages;
-    const SmemLayout L = smem_layout(N, T, K, E, H, I, S, kCompact);
+    const SmemLayout L = smem_layout(N, T, K, E, H, I, S, kCompact, WS);
     const int TS = (T + 3) & ~3;                              // token stride of the transposed input scales
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
@@ -653,6 +677,17 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
+    static_assert(!WS || (TC >= 16 && TC == N && N <= 32), "weighted ranges exist for the compacted variants only");
+    constexpr bool wsplit = WS;   // ranges of equal weight instead of equal k-step counts (see below)
+    if constexpr (kCompact) {
+        // weight of one k-step of a unit with c columns in use, c = 0..N, per projection (computed while thread 0 waits)
+        if (wsplit && tid >= 32 && tid <= 32 + N) {
+            const int c = tid - 32;
+            unsigned* s_kw = (unsigned*)(smem + L.kw_off);
+            s_kw[c] = 64u + (unsigned)((P.split_weight * (c / 4 + min(64, div_small(4 * c, KBu)))) >> 2);
+            s_kw[33 + c] = 64u + (unsigned)((P.split_weight * (c + min(64, div_small(8 * c, KBd)))) >> 2);
+        }
+    }
     if (tid == 0) {
         MOE_STAMP(3);
         red_release_add(P.ctrl + kRouteCnt + par, 1u);      // all CTAs' logits and xq published once this reaches G
@@ -727,7 +762,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             __syncthreads();
         }
         if (tid == 0) MOE_STAMP(6);
-        if constexpr (kCompact) {
+        if constexpr (kCompact && !WS) {
             // active list in ascending expert order, entry = expert | pass << 16 (passes of N tokens): every warp takes
             // 32-expert chunks; the chunks' totals meet in shared memory (the idle weight ring)
             int* s_tot = reinterpret_cast<int*>(smem);
@@ -751,6 +786,65 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (np) s_uidx[e] = u0;
                 if (c == nch - 1 && lane == 31) { misc[1] = (uint32_t)(base + incl); s_act[base + incl] = 0; }
             }
+        } else if constexpr (kCompact) {
+            // active list in ascending expert order, entry = expert | pass << 16 (passes of N tokens): every warp takes
+            // 32-expert chunks; the chunks' totals meet in shared memory (the idle weight ring).  The same scan carries
+            // the weights of the range split (see below): s_pv[ph][u] = weight of all k-steps before virtual expert u.
+            int* s_tot = reinterpret_cast<int*>(smem);                          // [3][32] chunk totals: passes, up weight, down weight
+            unsigned* s_pv = (unsigned*)(smem + L.pv_off);                      // [2][pv_stride]
+            const int PVS = L.pv_stride;
+            const int nch = (E + 31) / 32;
+            const unsigned n_up_u = (unsigned)(IB * KBu), n_dn_u = (unsigned)(HB * KBd);   // k-steps of one virtual expert
+            const unsigned* s_kw = (const unsigned*)(smem + L.kw_off);
+            const unsigned wfu = wsplit ? s_kw[N] * n_up_u : 0u, wfd = wsplit ? s_kw[33 + N] * n_dn_u : 0u;   // a full pass
+            constexpr int kIters = (kMaxExperts / 32 + kWarps - 1) / kWarps;    // chunks per warp (unrolled: the arrays stay in registers)
+            int np_l[kIters];
+            unsigned wu_l[kIters], wd_l[kIters];
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int c = warp + it * kWarps;
+                if (c >= nch) break;
+                const int e = c * 32 + lane;
+                const int m = (e < E) ? mask_count(load_mask(s_mask, e)) : 0;
+                const int full = m / N, rem = m - full * N;
+                const unsigned wru = (wsplit && rem) ? s_kw[rem] * n_up_u : 0u, wrd = (wsplit && rem) ? s_kw[33 + rem] * n_dn_u : 0u;
+                np_l[it] = full + (rem != 0); wu_l[it] = (unsigned)full * wfu + wru; wd_l[it] = (unsigned)full * wfd + wrd;
+                const int tot = __reduce_add_sync(0xffffffffu, np_l[it]);
+                if (lane == 0) s_tot[c] = tot;
+                if (wsplit) {
+                    const unsigned tu = __reduce_add_sync(0xffffffffu, wu_l[it]), td = __reduce_add_sync(0xffffffffu, wd_l[it]);
+                    if (lane == 0) { s_tot[32 + c] = (int)tu; s_tot[64 + c] = (int)td; }
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int c = warp + it * kWarps;
+                if (c >= nch) break;
+                const int e = c * 32 + lane;
+                const int np = np_l[it];
+                int incl = np;
+                unsigned iu = wu_l[it], id = wd_l[it];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                const int base = __reduce_add_sync(0xffffffffu, (lane < c) ? s_tot[lane] : 0);   // nch <= 16 chunks
+                const int u0 = base + incl - np;
+                for (int ps = 0; ps < np; ++ps) s_act[u0 + ps] = e | (ps << 16);
+                if (np) s_uidx[e] = u0;
+                if (c == nch - 1 && lane == 31) { misc[1] = (uint32_t)(base + incl); s_act[base + incl] = 0; }
+                if (wsplit) {
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned vu = __shfl_up_sync(0xffffffffu, iu, o), vd = __shfl_up_sync(0xffffffffu, id, o);
+                        if (lane >= o) { iu += vu; id += vd; }
+                    }
+                    const unsigned bu = __reduce_add_sync(0xffffffffu, (lane < c) ? (unsigned)s_tot[32 + lane] : 0u);
+                    const unsigned bd = __reduce_add_sync(0xffffffffu, (lane < c) ? (unsigned)s_tot[64 + lane] : 0u);
+                    const unsigned pu0 = bu + iu - wu_l[it], pd0 = bd + id - wd_l[it];
+                    for (int ps = 0; ps < np; ++ps) { s_pv[u0 + ps] = pu0 + (unsigned)ps * wfu; s_pv[PVS + u0 + ps] = pd0 + (unsigned)ps * wfd; }
+                    if (c == nch - 1 && lane == 31) { s_pv[base + incl] = bu + iu; s_pv[PVS + base + incl] = bd + id; }
+                }
+            }
         } else if (warp == 0) {                            // active list in ascending expert order
             int base = 0;
             for (int e0 = 0; e0 < E; e0 += 32) {
@@ -770,8 +864,43 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     const unsigned long long gm = P.grid_magic;
     const int q_up = range_quantum(U * IB, KBu, G, 32, P.split_slack_kib, gm), q_dn = range_quantum(U * HB, KBd, G, 16, P.split_slack_kib, gm);
     const int Sq_up = (q_up == 1) ? S_up : U * IB, Sq_dn = (q_dn == 1) ? S_dn : U * HB;      // quanta per list
-    const int up_lo = range_lo(Sq_up, cta, q_up, gm), up_hi = range_lo(Sq_up, cta + 1, q_up, gm);
-    const int dn_lo = range_lo(Sq_dn, cta, q_dn, gm), dn_hi = range_lo(Sq_dn, cta + 1, q_dn, gm);
+    // Range of CTA c in projection ph (0 up, 1 down).  Token-column variants: equal numbers of k-steps (closed form).
+    // Compacted variants: the accumulator warps pay per column in use, so a k-step of an expert with many tokens is
+    // dearer than one of an expert with few; there the list is cut into ranges of equal WEIGHT, a k-step of a unit
+    // with `cnt` columns in use weighing 64 + cnt/4 + 4 cnt/(K blocks) going up and 64 + cnt + 8 cnt/(K blocks) going
+    // down (fitted to the measured per-CTA phase times; the second term is the per-unit epilogue spread over the
+    // unit's k-steps).  Every CTA computes the same table of range starts once.
+    int* s_lo = (int*)(smem + L.lo_off);
+    const unsigned* s_pv = (const unsigned*)(smem + L.pv_off);
+    const float rG = __frcp_rz(__int2float_rz(G));
+    if constexpr (kCompact) {
+        if (alive && wsplit) {
+            // this CTA's own four range ends, one warp each (two 32-way steps find the virtual expert: U <= 1024);
+            // the accumulator warps fill in the other CTAs' while the first weight tiles are in flight
+            if (warp < 4) {
+                const int ph = warp >> 1, c = cta + (warp & 1);
+                const unsigned* p1 = s_pv + ph * L.pv_stride;
+                const int n_u = ph ? HB * KBd : IB * KBu;
+                int lo_ks = U * n_u;
+                if (c < G) {
+                    const unsigned target = split_target(p1[U], c, rG);
+                    const int stride = (U + 31) >> 5;
+                    const int b1 = __popc(__ballot_sync(0xffffffffu, lane * stride < U && p1[lane * stride] <= target)) - 1;   // p1[0] = 0
+                    const int i2 = b1 * stride + lane;
+                    const int a = b1 * stride + __popc(__ballot_sync(0xffffffffu, lane < stride && i2 < U && p1[i2] <= target)) - 1;
+                    lo_ks = split_point(p1, a, target, n_u, ph ? KBd : KBu, ph ? q_dn : q_up);
+                }
+                if (lane == 0) s_lo[ph * (kMaxGrid + 1) + c] = lo_ks;
+            }
+            __syncthreads();
+        }
+    }
+    auto rlo = [&](int ph, int c) -> int {
+        if constexpr (kCompact) { if (wsplit) return s_lo[ph * (kMaxGrid + 1) + c]; }
+        return ph ? range_lo(Sq_dn, c, q_dn, gm) : range_lo(Sq_up, c, q_up, gm);
+    };
+    const int up_lo = alive ? rlo(0, cta) : 0, up_hi = alive ? rlo(0, cta + 1) : 0;
+    const int dn_lo = alive ? rlo(1, cta) : 0, dn_hi = alive ? rlo(1, cta + 1) : 0;
 
     // ------------------------------------------------------------------ role: TMA producers
     // Stage sequence: an up k-step contributes two stages (gate tile, up tile), a down k-step one.  A stage = one
@@ -1065,13 +1194,30 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         }
         epi_bar(kEpiThreads);
         };
-        if constexpr (kCompact) build_pairs();
+        if constexpr (kCompact) {
+            if (wsplit) {                                  // every CTA's range starts (ordered before their first use by build_pairs' barriers)
+                for (int i = etid; i < 2 * (G + 1); i += kEpiThreads) {
+                    const int ph = (i > G) ? 1 : 0, c = i - ph * (G + 1);
+                    const unsigned* p1 = s_pv + ph * L.pv_stride;
+                    const int n_u = ph ? HB * KBd : IB * KBu;
+                    int lo_ks = U * n_u;
+                    if (c < G) {
+                        const unsigned target = split_target(p1[U], c, rG);
+                        int a = 0, b = U - 1;              // largest u with p1[u] <= target
+                        while (a < b) { const int m = (a + b + 1) >> 1; if (p1[m] <= target) a = m; else b = m - 1; }
+                        lo_ks = split_point(p1, a, target, n_u, ph ? KBd : KBu, ph ? q_dn : q_up);
+                    }
+                    s_lo[ph * (kMaxGrid + 1) + c] = lo_ks;
+                }
+            }
+            build_pairs();
+        }
 
         for (int phase = 0; phase < 2 && !wt.dead; ++phase) {
             const bool up = (phase == 0);
             const int lo = up ? up_lo : dn_lo, hi = up ? up_hi : dn_hi;
             const int KB = up ? KBu : KBd, MB = up ? IB : HB;  // K blocks per unit, row blocks per expert
-            const int Sq_all = up ? Sq_up : Sq_dn, q_all = up ? q_up : q_dn;
+            const int rph = up ? 0 : 1;
             float* part = up ? P.part_up : P.part_dn;
             unsigned* pflag = up ? P.pu_flag : P.pd_flag;
             const int pcols = up ? 2 * N : N;
@@ -1279,15 +1425,15 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                     for (int base = cta + 1; base < G; base += kEpiThreads) {
                         const int c = base + etid;
                         if (c < G) {
-                            const int clo = range_lo(Sq_all, c, q_all, gm), chi = range_lo(Sq_all, c + 1, q_all, gm);
+                            const int clo = rlo(rph, c), chi = rlo(rph, c + 1);
                             if (clo < uend && chi > clo) got = wt.flag(pflag + c, tag, 6) && got;
                         }
-                        if (range_lo(Sq_all, min(base + kEpiThreads, G), q_all, gm) >= uend) break;
+                        if (rlo(rph, min(base + kEpiThreads, G)) >= uend) break;
                     }
-                    while (c_end < G && range_lo(Sq_all, c_end, q_all, gm) < uend) ++c_end;
+                    while (c_end < G && rlo(rph, c_end) < uend) ++c_end;
                     if (!epi_all(got, kEpiThreads)) { wt.dead = true; break; }
                     for (int c = cta + 1; c < c_end; ++c) {
-                        if (range_lo(Sq_all, c + 1, q_all, gm) == range_lo(Sq_all, c, q_all, gm)) continue;
+                        if (rlo(rph, c + 1) == rlo(rph, c)) continue;
                         const float* src = part + (size_t)c * pcols * kBlock;
 #pragma unroll
                         for (int n = 0; n < TCG; ++n) {
@@ -1361,8 +1507,16 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 const int ex = s_ids[t * K + j];
                 const int ps = kCompact ? mask_rank(load_mask(s_mask, ex), t) / N : 0;   // the pass that holds token t
                 const unsigned unit = (unsigned)((s_uidx[ex] + ps) * HB + hb);
-                const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;          // first quantum of the unit
-                const unsigned owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
+                unsigned owner;
+                if (kCompact && wsplit) {
+                    const int xk = (int)unit * KBd;                                    // first k-step of the unit
+                    int a = 0, b = G - 1;                                              // the CTA whose range holds it
+                    while (a < b) { const int m = (a + b + 1) >> 1; if (rlo(1, m) <= xk) a = m; else b = m - 1; }
+                    owner = (unsigned)a;
+                } else {
+                    const unsigned x = (q_dn == 1) ? unit * (unsigned)KBd : unit;      // first quantum of the unit
+                    owner = ((x + 1u) * (unsigned)G - 1u) / (unsigned)Sq_dn;
+                }
                 got = wt.flag(P.dn_flag + owner, tag, 7) && got;
             }
             if (!epi_all(got, kEpiThreads)) wt.dead = true;

@@ -2,7 +2,8 @@
 numerical check are rejected, the rest are ranked by CUDA-graph timing over token counts and routing regimes).
 
 The kernel's schedule knobs are those of `moe_plan_set_knob` (include/moe_b200.h): pipeline stages, the whole-unit vs
-split-K threshold, the token count up to which every CTA routes all tokens, the compaction threshold.  For one layer
+split-K threshold, the token count up to which every CTA routes all tokens, equal-weight ranges, the compaction
+threshold.  For one layer
 shape this module times every candidate on seeded synthetic layers (the inputs of `workloads`), validates each
 candidate's output against the default schedule's output of the same step, and writes a table that
 `MoEPlan(..., schedule=table)` / `MoEPlan.apply_schedule(table)` / `bench.py --schedule FILE` apply:
@@ -33,6 +34,7 @@ PER_TOKEN_GRID = {
     "split_slack_kib": [0, 50, 100, 200, 400],
     "stages": [0, 16, 8, 6],
     "route_all_tokens": [8, 16, 32],
+    "split_weight": [-1, 0, 4],
 }
 PLAN_GRID = {"compact_min": [9, 5]}
 
@@ -81,6 +83,8 @@ def relevant_knobs(T, per_launch):
     grid = dict(PER_TOKEN_GRID)
     if not 8 < min(T, per_launch) <= 32:
         grid["route_all_tokens"] = [8]
+    if min(T, per_launch) < 9:                       # equal-weight ranges exist only where tokens are compacted
+        grid["split_weight"] = [-1]
     return grid
 
 
@@ -169,7 +173,7 @@ def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=
 
 
 def plan_default(knob):
-    return {"split_slack_kib": 100, "stages": 0, "route_all_tokens": 8}[knob]
+    return {"split_slack_kib": 100, "stages": 0, "route_all_tokens": 8, "split_weight": -1}[knob]
 
 
 def main(argv=None):

@@ -82,10 +82,13 @@ def _only_order_within_band(a, b, key, tau):
     return all(x == y or abs(key[x] - key[y]) <= tau for x, y in zip(a, b))
 
 
-def run_case(shape, T, regime="natural", layer=0, dist="gauss", routed_scale=1.0, max_oracle_tokens=None, repeat=1):
+def run_case(shape, T, regime="natural", layer=0, dist="gauss", routed_scale=1.0, max_oracle_tokens=None, repeat=1,
+             knobs=None):
     d = wl.make_layer(shape, T, regime=regime, layer=layer, device="cuda", dist=dist)
     plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, routed_scale, T_max=T)
     try:
+        for knob, value in (knobs or {}).items():
+            plan.set_knob(0, knob, value)
         dbg = plan.forward_debug(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
         plan.sync_status()
         res = check_against_oracle(shape, T, d, dbg, routed_scale, max_oracle_tokens)

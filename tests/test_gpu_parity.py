@@ -50,6 +50,18 @@ def test_config3_routing_regimes(regime, T):
     assert r["rel_l2"] < 2e-3, r
 
 
+@pytest.mark.parametrize("weight,slack", [(0, 100), (4, 100), (8, 0), (4, 1 << 20)])
+@pytest.mark.parametrize("shape,regime,T", [(SMALL_SIG, "natural", 12), (SMALL_SIG, "same", 40), (RAGGED, "natural", 24),
+                                            (RAGGED, "same", 128), (wl.SHAPES["c2_qwen3_30b_a3b"], "same", 64),
+                                            (wl.SHAPES["c2_qwen3_30b_a3b"], "natural", 33)])
+def test_ranges_of_equal_weight(shape, regime, T, weight, slack):
+    """Where tokens are compacted the per-CTA ranges are cut by weight (a k-step of a crowded expert weighs more), in
+    both compacted variants, with units split across CTAs (slack 0) and kept whole (huge slack); weight 0 is the
+    equal-length cut.  Every setting must match the oracle and repeat bit-identically."""
+    r = run_case(shape, T, regime=regime, max_oracle_tokens=8, repeat=2, knobs={"split_weight": weight, "split_slack_kib": slack})
+    assert r["rel_l2"] < 2e-3, r
+
+
 @pytest.mark.parametrize("shape,per_launch", [(SMALL_SIG, 128), (TINY, 64)])
 def test_more_tokens_than_one_launch_is_chunked(shape, per_launch):
     """More tokens than one launch takes (128 under sparse routing, else 64) run as consecutive launches; each chunk

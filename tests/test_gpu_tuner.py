@@ -24,6 +24,11 @@ def test_knobs_round_trip_and_reject_bad_values():
         plan.set_knob(8, "stages", 1)
     with pytest.raises(Exception):
         plan.set_knob(8, "compact_min", 40)
+    assert plan.get_knob(16, "split_weight") == -1
+    plan.set_knob(16, "split_weight", 8)
+    assert plan.get_knob(16, "split_weight") == 8 and plan.get_knob(12, "split_weight") == -1
+    with pytest.raises(Exception):
+        plan.set_knob(16, "split_weight", 9)
     plan.close()
 
 
