@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/; keyed by (config, tokens).  None where no capture exists.
 NCU_TRAFFIC_BYTES = {
     ("c2_qwen3_30b_a3b", 1): 38.700e6 + 0.036e6,     # profiles/moe_decode_kernel_c2_qwen3_t1.md
-    ("c2_qwen3_30b_a3b", 64): 601.8e6 + 5.3e6,       # profiles/moe_decode_kernel_c2_qwen3_t64.md
-    ("c4_mixtral_8x7b", 64): 1416.2e6 + 7.8e6,       # profiles/moe_decode_kernel_c4_mixtral_t64.md
+    ("c2_qwen3_30b_a3b", 64): 601.9e6 + 5.6e6,       # profiles/moe_decode_kernel_c2_qwen3_t64.md
+    ("c4_mixtral_8x7b", 64): 1416.3e6 + 6.8e6,       # profiles/moe_decode_kernel_c4_mixtral_t64.md
     ("c5_deepseek_v3[E=16]", 1): 356.76e6 + 4.67e6,  # profiles/moe_decode_kernel_c5like_e16_t1.md
     ("c5_deepseek_v3[E=64]", 8): 1680.1e6 + 4.8e6,   # profiles/moe_decode_kernel_c5like_e64_t8.md
 }
