@@ -465,7 +465,8 @@ __device__ __forceinline__ void route_select(const Params& P, int t, int lane, c
 #pragma unroll
     for (int i = 0; i < NPER; ++i) key[i] = (i * 32 + lane < E) ? s_key[i * 32 + lane] : 0u;    // 0 is below every real key
     int my_id = 0;
-    for (int j = 0; j < K; ++j) {
+#pragma unroll 1
+    for (int j = 0; j < K; ++j) {                              // (a serial chain: unrolling buys nothing, and code fetched once per launch is dear)
         uint32_t m = key[0];
 #pragma unroll
         for (int i = 1; i < NPER; ++i) m = max(m, key[i]);
@@ -580,6 +581,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
+#pragma unroll 1
     for (int e = tid; e < 2 * E; e += kThreads) s_mask[e] = 0ull;
     int ksplit = 1;                                              // parts of H per router tile: enough to occupy the grid
     {
@@ -594,6 +596,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const int kper = (kpart_len / 16 + kWarps - 1) / kWarps * 16;
             const int k_lo = kp * kpart_len + warp * kper, k_hi = min((kp + 1) * kpart_len, k_lo + kper);
             const int lines = (k_hi - k_lo + 63) / 64;                        // 128-byte lines per row
+#pragma unroll 1
             for (int idx = lane; idx < 16 * lines; idx += 32) {
                 const int r = eb * 16 + (idx & 15);
                 if (r < E) prefetch_l2(P.Wr + (size_t)r * H + k_lo + (idx >> 4) * 64);
@@ -607,6 +610,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (tid == 0) MOE_STAMP(0);
     const unsigned par = tag & 1u;
     unsigned* e_cnt = P.e_cnt + par * kMaxPasses * E;       // counters of this launch: [pass][expert]
+#pragma unroll 1
     for (int e = cta * kThreads + tid; e < kMaxPasses * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * kMaxPasses * E + e] = 0u;
     if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
@@ -615,6 +619,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     {
         // input quantisation: one warp per (token, 128-column group)  (Section 4.1)
         const int groups = T * KBu;
+#pragma unroll 1
         for (int p = (G - 1 - cta) * kWarps + warp; p < groups; p += G * kWarps) {   // from the last CTA down: the first ones have router tiles
             const int t = p / KBu, g = p % KBu;
             const uint2 raw = *reinterpret_cast<const uint2*>(P.hidden + (size_t)t * H + g * kBlock + lane * 4);
@@ -639,6 +644,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             const int g = lane >> 2, tq = lane & 3;
             const int kpart_len = H / ksplit;
             const int kper = (kpart_len / 16 + kWarps - 1) / kWarps * 16;   // K range of one warp (multiple of 16)
+#pragma unroll 1
             for (int wi = cta; wi < nEB * nTB * ksplit; wi += G) {
                 const int item = wi / ksplit, kp = wi - item * ksplit;
                 const int eb = item / nTB, tb = item - eb * nTB;
@@ -727,6 +733,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         }
         __syncthreads();
         if (tid == 0) MOE_STAMP(5);
+#pragma unroll 1
         for (int tl = warp; tl < rnt; tl += kWarps) {
             const int t = rt0 + tl;
             if (E <= 128) route_select<4>(P, t, lane, s_key + tl * E, s_val + tl * E, s_ids, s_w, s_mask, wg, route_all);
@@ -847,6 +854,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
         } else if (warp == 0) {                            // active list in ascending expert order
             int base = 0;
+#pragma unroll 1
             for (int e0 = 0; e0 < E; e0 += 32) {
                 const int e = e0 + lane;
                 const bool on = (e < E) && (s_mask[2 * e] != 0ull);
@@ -1178,6 +1186,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         auto build_pairs = [&]() {
         if (warp == kEpiWarp0) {
             int base = 0;
+#pragma unroll 1
             for (int e0 = 0; e0 < E; e0 += 32) {
                 const int c = (e0 + lane < E) ? mask_count(load_mask(s_mask, e0 + lane)) : 0;
                 int incl = c;
@@ -1188,6 +1197,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
         }
         epi_bar(kEpiThreads);
+#pragma unroll 1
         for (int pi = etid; pi < T * K; pi += kEpiThreads) {
             const int t = div_small(pi, K), ex = s_ids[pi];
             s_pair[s_poff[ex] + mask_rank(load_mask(s_mask, ex), t)] = (unsigned short)(t | ((pi - t * K) << 8));
@@ -1196,6 +1206,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         };
         if constexpr (kCompact) {
             if (wsplit) {                                  // every CTA's range starts (ordered before their first use by build_pairs' barriers)
+#pragma unroll 1
                 for (int i = etid; i < 2 * (G + 1); i += kEpiThreads) {
                     const int ph = (i > G) ? 1 : 0, c = i - ph * (G + 1);
                     const unsigned* p1 = s_pv + ph * L.pv_stride;
@@ -1500,6 +1511,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         const int n_tasks = T * HB, n_mine = (cta < n_tasks) ? (n_tasks - cta + G - 1) / G : 0;
         {
             bool got = true;
+#pragma unroll 1
             for (int idx = etid; idx < n_mine * K; idx += kEpiThreads) {
                 const int i = div_small(idx, K), j = idx - i * K, task = cta + i * G;
                 const int t = div_small(task, HB), hb = task - t * HB;
