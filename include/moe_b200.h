@@ -179,7 +179,8 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              library's choice for the token count (default): 6 or 8 for short weight streams, all
  *                              that fit for steps of a few tiles and for long streams
  *   MOE_KNOB_SPLIT_SLACK_KIB   keep a projection's units whole while that costs the busiest CTA at most this many KiB
- *                              of extra weight stream, split them across CTAs (split-K) otherwise (default 100)
+ *                              of extra weight stream, split them across CTAs (split-K) otherwise (default 200 up to 8 tokens,
+ *                              100 beyond)
  *   MOE_KNOB_ROUTE_ALL_TOKENS  up to this many tokens every CTA selects the experts of all tokens; beyond, the grid
  *                              shares the tokens and exchanges the result (default 8; up to 8 tokens every CTA always
  *                              selects for all of them, so smaller values act as 8)

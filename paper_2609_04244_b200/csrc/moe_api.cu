@@ -83,7 +83,7 @@ struct moe_plan {
     int use_pdl = 1;                // programmatic dependent launch
     int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
     moe_plan() {
-        for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
+        for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = t <= 8 ? 200 : 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
     }
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors

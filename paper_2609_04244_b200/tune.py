@@ -31,7 +31,7 @@ from .binding import MoEPlan
 REL_L2_REJECT = 2e-3
 
 PER_TOKEN_GRID = {
-    "split_slack_kib": [0, 50, 100, 200, 400],
+    "split_slack_kib": [200, 0, 100, 300, 400],
     "stages": [0, 16, 8, 6],
     "route_all_tokens": [8, 16, 32],
     "split_weight": [-1, 0, 4],
@@ -160,7 +160,7 @@ def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=
         valid = [r for r in results if r["us"] is not None]
         best = min(valid, key=lambda r: r["us"])
         # keep the defaults unless the best candidate is clearly (1 %) faster: timing noise is of that order
-        chosen = best["knobs"] if best["us"] < 0.99 * default_us else {n: plan_default(n) for n in names}
+        chosen = best["knobs"] if best["us"] < 0.99 * default_us else {n: plan_default(n, T) for n in names}
         table["per_tokens"][str(T)] = chosen
         table["measured_us"][str(T)] = {"default": round(default_us, 2), "best": round(best["us"], 2),
                                         "rejected": len(results) - len(valid),
@@ -172,8 +172,8 @@ def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=
     return table
 
 
-def plan_default(knob):
-    return {"split_slack_kib": 100, "stages": 0, "route_all_tokens": 8, "split_weight": -1}[knob]
+def plan_default(knob, T=1):
+    return {"split_slack_kib": 200 if T <= 8 else 100, "stages": 0, "route_all_tokens": 8, "split_weight": -1}[knob]
 
 
 def main(argv=None):

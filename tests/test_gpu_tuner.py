@@ -15,10 +15,10 @@ SHAPE = wl.MoEShape("tune_small", 7, H=512, E=32, I=256, top_k=4, scoring=wl.SCO
 
 def test_knobs_round_trip_and_reject_bad_values():
     plan = MoEPlan(SHAPE.H, SHAPE.E, SHAPE.I, SHAPE.top_k, SHAPE.scoring, SHAPE.renorm, T_max=16)
-    assert plan.get_knob(8, "split_slack_kib") == 100 and plan.get_knob(8, "stages") == 0
+    assert plan.get_knob(8, "split_slack_kib") == 200 and plan.get_knob(8, "stages") == 0
     plan.set_knob(8, "split_slack_kib", 0)
     plan.set_knob(0, "stages", 6)
-    assert plan.get_knob(8, "split_slack_kib") == 0 and plan.get_knob(4, "split_slack_kib") == 100
+    assert plan.get_knob(8, "split_slack_kib") == 0 and plan.get_knob(4, "split_slack_kib") == 200
     assert plan.get_knob(16, "stages") == 6 and plan.info(8)["stages"] == 6
     with pytest.raises(Exception):
         plan.set_knob(8, "stages", 1)
