@@ -57,14 +57,17 @@ enum { MOE_SCORE_SOFTMAX = 0, MOE_SCORE_SIGMOID_BIAS = 1 };
 /* Largest number of tokens one kernel launch can handle; a plan's own limit is moe_tokens_per_launch(). */
 #define MOE_MAX_TOKENS_PER_LAUNCH 128
 
+/* Size of the scratch array built into the library's device image for moe_forward_noalloc (24 MiB). */
+#define MOE_NOALLOC_SCRATCH_BYTES (24u << 20)
+
 /*
  * moe_plan: fix the layer shape and routing policy (Section 3.4: shape and
  * schedule are fixed ahead of time, token count is a run-time argument).
  *   H hidden size, E experts, I intermediate size, top_k experts per token,
  *   scoring MOE_SCORE_*, renorm != 0 renormalises the selected weights.
  * Queries the current device, checks that the persistent grid (one CTA per SM)
- * is co-resident (Section 3.2, "verifies the realized occupancy") and stores
- * host-side state only.  *out receives the plan; free it with moe_plan_destroy.
+ * is actually co-resident, one CTA per SM, rather than assuming it (Section
+ * 3.2), and stores host-side state only.  *out receives the plan; free it with moe_plan_destroy.
  */
 int moe_plan(int H, int E, int I, int top_k, int scoring, int renorm, moe_plan_t* out);
 
@@ -122,7 +125,11 @@ int moe_forward_host(moe_plan_t plan, int T,
  * part of the library's device image: every GPU that loads the library holds these 24 MiB until the process exits.
  *   - Same tensor arguments as moe_forward; there is no workspace argument.  1 <= T <= 64.
  *   - A layer shape whose scratch for T tokens exceeds the array is rejected with MOE_ERR_WORKSPACE and a message
- *     giving both sizes (the five benchmark shapes fit for T <= 16).
+ *     giving both sizes (the five benchmark shapes fit for T <= 16).  Up to 8 tokens the fused-unit kernel variant
+ *     is used where its (larger) scratch fits, the general variant otherwise; results agree within rounding.
+ *   - A device-side wait that ran out is recorded in the array, like in a workspace: read it with
+ *     moe_sync_status(plan, NULL, stream) BEFORE the next moe_forward_noalloc call on the device (every call starts by
+ *     clearing the array's control words, and with them the record).
  *   - The plan's device must be the current device.  The FIRST call on a device looks up the array's device
  *     address (cudaGetSymbolAddress); make that first call outside any stream capture.
  *   - The call itself allocates nothing: no cudaMalloc/cudaFree, no descriptor cache; TMA descriptors are built on
@@ -152,7 +159,8 @@ int moe_forward_debug(moe_plan_t plan, int T,
                       int32_t* topk_ids, float* topk_w, uint8_t* xq, float* xs, float* logits);
 
 /* Synchronise `stream`, read the workspace's device status word and return MOE_OK, MOE_ERR_TIMEOUT or
- * MOE_ERR_CUDA.  After MOE_ERR_TIMEOUT the workspace must be re-initialised. */
+ * MOE_ERR_CUDA.  After MOE_ERR_TIMEOUT the workspace must be re-initialised.  workspace == NULL reads the built-in
+ * array of moe_forward_noalloc on the plan's device (MOE_ERR_ARG if that entry point has never run there). */
 int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream);
 
 /* Tokens one launch of this plan handles: 128 when the routing is sparse enough (128 * top_k <= 20 * E) for the
@@ -162,8 +170,18 @@ int moe_tokens_per_launch(moe_plan_t plan);
 /* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);
 
+/* Introspection: which kernel variant T tokens get.  *fused = 1 for the fused-unit variant (1..8 tokens: a work unit
+ * is one expert's 128-wide intermediate block through gate/up AND its down-projection column block, shared by the
+ * *cluster CTAs of a thread-block cluster; Section 3.2's hand-over of the intermediate tile stays on chip), 0 for the
+ * general variant (*cluster = 1).  Either out may be NULL. */
+int moe_plan_variant(moe_plan_t plan, int T, int* fused, int* cluster);
+
 /* Diagnostics: synchronise `stream` and copy the phase time stamps of the last launch on this workspace to
- * HOST memory host_out[grid*16] (nanoseconds of the GPU's global timer).  Per CTA: 0 start, 1 input quantised,
+ * HOST memory host_out[SMs*16] (nanoseconds of the GPU's global timer); the launch must have run with MOE_KNOB_STAMPS
+ * set.  Fused-unit variant, per CTA: 0 start, 1 router rows published, 2 input quantised, 3 all logits gathered, 4 top-k
+ * done, 5 routing metadata done, 6 first weight tile requested, 7 first weight tile landed, 8 first accumulator read,
+ * 9 first partial sums parked, 10 first intermediate tile ready, 11 last down tile stored, 12 all CTAs done, 13
+ * reduction done, 14 SM id (not a time), 15 exit.  General variant, per CTA: 0 start, 1 input quantised,
  * 2 router logits done, 3 arrived at the routing flag, 4 routing published grid-wide, 5 selection keys ready,
  * 6 top-k done, 7 routing metadata done, 8 first weight tile requested, 9 first ring of requests issued,
  * 10 first weight tile landed, 11 first accumulator read, 12 up phase done, 13 down phase done, 14 reduction
@@ -191,11 +209,20 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              columns in use), instead of ranges of equal length.  0 = equal length, 1..8 = strength
  *                              of the per-column term in quarters of the fitted value, -1 = the library's choice
  *                              (default: 4 from 24 tokens on, from 16 where I <= 256, else 0)
- * Results do not depend on STAGES, ROUTE_ALL_TOKENS or PDL; SPLIT_SLACK_KIB, COMPACT_MIN and SPLIT_WEIGHT change the
- * order of fp32 partial sums (never the routing or the quantised input).
+ *   MOE_KNOB_FUSED             (plan-wide) fused-unit variant for 1..8 tokens: 1 = wherever it can run, 0 = never,
+ *                              -1 = the library's choice (default).  Changes the scratch layout: query
+ *                              moe_workspace_bytes() again.
+ *   MOE_KNOB_CLUSTER           fused-unit variant: CTAs that share one unit (thread-block cluster size) 1, 2, 4 or 8;
+ *                              0 = the library's choice (default): the size for which the busiest CTA streams the fewest
+ *                              tiles at the expected number of distinct experts.  MOE_ERR_OCCUPANCY if the device cannot
+ *                              hold such clusters.  With MOE_KNOB_STAGES = 0 the fused variant takes as many stages as
+ *                              leave half of the SM's shared memory to the next launch's CTA.
+ *   MOE_KNOB_STAMPS            (plan-wide) kernels record the phase time stamps moe_debug_stamps() reads; off by default
+ * Results do not depend on STAGES, ROUTE_ALL_TOKENS, PDL or STAMPS; SPLIT_SLACK_KIB, COMPACT_MIN, SPLIT_WEIGHT, FUSED and
+ * CLUSTER change the order of fp32 partial sums (never the routing or the quantised input).
  */
 enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4,
-       MOE_KNOB_SPLIT_WEIGHT = 5 };
+       MOE_KNOB_SPLIT_WEIGHT = 5, MOE_KNOB_FUSED = 6, MOE_KNOB_CLUSTER = 7, MOE_KNOB_STAMPS = 8 };
 int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value);
 int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value);
 

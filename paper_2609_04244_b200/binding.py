@@ -16,7 +16,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID_BIAS = 1
 
 EXPORTS = ["moe_plan", "moe_plan_ex", "moe_plan_destroy", "moe_workspace_bytes", "moe_workspace_init", "moe_forward",
-           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_tokens_per_launch", "moe_plan_set_knob", "moe_plan_get_knob", "moe_plan_set_timeout_ms", "moe_last_error"]
+           "moe_forward_noalloc", "moe_forward_host", "moe_forward_debug", "moe_sync_status", "moe_debug_stamps", "moe_plan_info", "moe_plan_variant", "moe_tokens_per_launch", "moe_plan_set_knob", "moe_plan_get_knob", "moe_plan_set_timeout_ms", "moe_last_error"]
 
 _lib = None
 
@@ -66,6 +66,8 @@ def load_library():
     lib.moe_debug_stamps.argtypes = [vp, vp, vp, vp]
     lib.moe_plan_info.restype = i
     lib.moe_plan_info.argtypes = [vp, i] + [ctypes.POINTER(i)] * 4
+    lib.moe_plan_variant.restype = i
+    lib.moe_plan_variant.argtypes = [vp, i] + [ctypes.POINTER(i)] * 2
     lib.moe_plan_set_knob.restype = i
     lib.moe_plan_set_knob.argtypes = [vp, i, i, i]
     lib.moe_plan_get_knob.restype = i
@@ -158,12 +160,14 @@ def moe_sync_status(plan, workspace, stream=None) -> None:
 def moe_debug_stamps(plan, workspace, grid: int, stream=None):
     """Phase time stamps [grid, 16] (ns) of the last launch on this workspace; see include/moe_b200.h."""
     import numpy as np
-    buf = np.zeros((grid, 16), dtype=np.uint64)
+    sms = torch.cuda.get_device_properties(workspace.device).multi_processor_count   # the call fills one row per SM
+    buf = np.zeros((max(sms, grid), 16), dtype=np.uint64)
     _check(load_library().moe_debug_stamps(plan, _p(workspace), _stream(stream), ctypes.c_void_p(buf.ctypes.data)))
-    return buf
+    return buf[:grid]
 
 
-KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4, "split_weight": 5}
+KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4, "split_weight": 5,
+         "fused": 6, "cluster": 7, "stamps": 8}
 
 
 def moe_plan_set_knob(plan, T: int, knob, value: int) -> None:
@@ -184,7 +188,15 @@ def moe_tokens_per_launch(plan) -> int:
 def moe_plan_info(plan, T: int) -> dict:
     g, s, n, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     _check(load_library().moe_plan_info(plan, T, ctypes.byref(g), ctypes.byref(s), ctypes.byref(n), ctypes.byref(b)))
-    return {"grid": g.value, "stages": s.value, "n_hw": n.value, "smem_bytes": b.value}
+    f, c = moe_plan_variant(plan, T)
+    return {"grid": g.value, "stages": s.value, "n_hw": n.value, "smem_bytes": b.value, "fused": f, "cluster": c}
+
+
+def moe_plan_variant(plan, T: int):
+    """(fused, cluster): whether T tokens get the fused-unit kernel variant, and the CTAs that share one unit."""
+    f, c = ctypes.c_int(), ctypes.c_int()
+    _check(load_library().moe_plan_variant(plan, T, ctypes.byref(f), ctypes.byref(c)))
+    return bool(f.value), c.value
 
 
 class MoEPlan:
@@ -252,8 +264,9 @@ class MoEPlan:
     def sync_status(self, stream=None):
         moe_sync_status(self.handle, self.workspace, stream)
 
-    def stamps(self, stream=None):
-        return moe_debug_stamps(self.handle, self.workspace, self.info(1)["grid"], stream)
+    def stamps(self, T=1, stream=None):
+        """Phase time stamps of the last launch (of T tokens); needs the "stamps" knob set before that launch."""
+        return moe_debug_stamps(self.handle, self.workspace, self.info(T)["grid"], stream)
 
     def info(self, T):
         return moe_plan_info(self.handle, T)

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libmoe_b200.so")
 SOURCES = ["moe_api.cu"]
-DEPS = ["moe_api.cu", "moe_kernel.cuh", os.path.join("..", "..", "include", "moe_b200.h")]
+DEPS = ["moe_api.cu", "moe_kernel.cuh", "moe_fused_kernel.cuh", os.path.join("..", "..", "include", "moe_b200.h")]
 
 
 def _nvcc() -> str:

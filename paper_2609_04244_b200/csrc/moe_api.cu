@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/moe_b200.h: plan, workspace layout, TMA descriptors, launch.
 #include "moe_kernel.cuh"
+#include "moe_fused_kernel.cuh"
 
 #include <cstdarg>
 #include <cmath>
@@ -57,7 +58,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
     size_t ctrl, e_cnt, dn_flag, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
-    size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, total;
+    size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, ll, yp, total;
 };
 
 struct MapKey {
@@ -82,6 +83,12 @@ struct moe_plan {
     int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
     int use_pdl = 1;                // programmatic dependent launch
     int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
+    // fused-unit variants (1..8 tokens, moe_fused_kernel.cuh)
+    int fused_mode = -1;            // 1: wherever they apply, 0: never, -1: the library's choice
+    int cluster_knob[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // CTAs per unit for T = 1..8; 0 = the library's choice
+    int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
+    int smem_per_sm = 0;
+    int take_stamps = 0;            // kernels record their phase time stamps (diagnostics)
     moe_plan() {
         for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = t <= 8 ? 200 : 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
     }
@@ -110,7 +117,8 @@ struct moe_plan {
     int chunk() const { return compact(moe::kMaxTokens) ? moe::kMaxTokens : 64; }
     int cap(int T) const { return T < chunk() ? T : chunk(); }
 
-    WsLayout layout(int T_max) const {
+    WsLayout layout(int T_max) const { return layout(T_max, fused(cap(T_max))); }
+    WsLayout layout(int T_max, bool with_fused) const {
         const int Tc = cap(T_max), N = n_hw(Tc), NR = nr(Tc), G = sms;
         WsLayout L;
         size_t o = 0;
@@ -134,8 +142,50 @@ struct moe_plan {
         L.y = o;        o += align_up((size_t)Tc * K * H * 4, 256);
         L.stage_in = o;  o += align_up((size_t)Tc * H * 2, 256);    // device copies of host-resident input/output
         L.stage_out = o; o += align_up((size_t)Tc * H * 2, 256);    // (moe_forward_host)
+        // fused variants: tagged router logits, and one down-projection partial per (token, slot, intermediate block)
+        L.ll = o;       o += with_fused ? align_up((size_t)Tc * E * 8, 256) : 0;
+        L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 4, 256) : 0;
         L.total = o;
         return L;
+    }
+
+    // ---- fused-unit variants -------------------------------------------------------------------------------------
+    static int fused_tc(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
+    // shared memory that still lets two CTAs share an SM (the next launch's CTAs become resident under this one)
+    int fused_smem_budget() const { const int half = smem_per_sm / 2 - 1024; return half < smem_optin ? half : smem_optin; }
+    int fused_stages(int T) const {
+        const int cap_s = stages_cap[T];
+        const int budget = cap_s > 0 ? smem_optin : fused_smem_budget();
+        for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s)
+            if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) return s;
+        return 0;
+    }
+    // CTAs per unit.  A unit (expert, 128-wide intermediate block) is 3 * H/128 weight tiles; clusters take units
+    // round-robin, so the busiest CTA streams ceil(units / clusters) * ceil(3 * (H/128) / C) tiles: take the C that
+    // makes that smallest for the expected number of distinct experts (text after Eq. 5), the smaller C on a tie.
+    int fused_cluster(int T) const {
+        const int KB = H / 128;
+        const int knob = cluster_knob[T];
+        if (knob > 0) return (knob <= 8 && max_clusters[knob] > 0 && knob <= KB) ? knob : 0;
+        const double U = E * (1.0 - std::pow(1.0 - (double)K / E, (double)T));
+        const long long units = (long long)std::llround(U) * (I / 128);
+        int best = 0;
+        long long best_cost = 0;
+        for (int C = 1; C <= 4; C *= 2) {
+            if (max_clusters[C] <= 0 || C > KB) continue;
+            const long long rounds = (units + max_clusters[C] - 1) / max_clusters[C];
+            const long long cost = rounds * ((3 * KB + C - 1) / C);
+            if (!best || cost < best_cost) { best = C; best_cost = cost; }
+        }
+        return best;
+    }
+    int fused_grid(int T) const { const int C = fused_cluster(T); return C ? C * max_clusters[C] : 0; }
+    bool fused_possible(int T) const {
+        return T >= 1 && T <= 8 && T < compact_min && H <= 8192 && fused_cluster(T) > 0 && fused_stages(T) >= 2;
+    }
+    bool fused(int T) const {
+        if (fused_mode == 0 || !fused_possible(T)) return false;
+        return true;
     }
 
     // Default depth of the stage ring when the knob is 0.  Measured on this machine (config 2 and the paper's shapes,
@@ -182,12 +232,7 @@ namespace {
 template <int N, int TC, bool WS = false>
 int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx, const CUtensorMap& mh,
            const moe::Params& P, int smem_bytes, cudaStream_t stream) {
-    static int configured_device = -1;
-    if (configured_device != p->device) {
-        if (cudaFuncSetAttribute(moe::moe_decode_kernel<N, TC, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_optin) != cudaSuccess)
-            return fail(MOE_ERR_CUDA, "cudaFuncSetAttribute(max dynamic smem) failed: %s", cudaGetErrorString(cudaGetLastError()));
-        configured_device = p->device;
-    }
+    // (the opt-in shared-memory size of every variant was set by resident<>() when the plan was made)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p->sms, 1, 1);
     cfg.blockDim = dim3(128 + 128 * (TC >= 32 ? 2 : 1), 1, 1);
@@ -202,6 +247,47 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
     if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
     return MOE_OK;
+}
+
+// Fused-unit variants: grid = clusters x C CTAs, cluster size chosen at run time.
+template <int TC>
+int launch_fused(Plan* p, int grid, int C, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx,
+                 const moe::Params& P, int smem_bytes, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p->use_pdl ? 2 : 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_fused_kernel<TC>, m13, m2, mx, P);
+    if (err == cudaSuccess) err = cudaGetLastError();
+    if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
+    return MOE_OK;
+}
+
+// Clusters of C CTAs of the fused kernel that are co-resident when every SM holds ONE of its CTAs (the other half of
+// the SM may still belong to the previous launch); 0 when such a cluster cannot be launched at all.
+template <int TC>
+int fused_clusters(int C, int smem_optin, int sms) {
+    if (cudaFuncSetAttribute(moe::moe_fused_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) { cudaGetLastError(); return 0; }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((sms / C) * C, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = smem_optin;                         // a footprint that admits one CTA per SM
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, moe::moe_fused_kernel<TC>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n < sms / C ? n : sms / C;
 }
 
 template <int N, int TC, bool WS = false>
@@ -248,7 +334,9 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.pu_flag = reinterpret_cast<unsigned*>(w + L.pu_flag);
     P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
     P.y = reinterpret_cast<float*>(w + L.y);
-    P.stamps = reinterpret_cast<unsigned long long*>(w + L.stamps);
+    P.ll = reinterpret_cast<unsigned long long*>(w + L.ll);
+    P.yp = reinterpret_cast<float*>(w + L.yp);
+    P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
     return P;
 }
 
@@ -270,31 +358,56 @@ int dispatch(Plan* p, int T, const CUtensorMap& m13, const CUtensorMap& m2, cons
     return launch<64, 64>(p, m13, m2, mx, mh, P, smem_bytes, stream);
 }
 
-int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
-                  const float* W13s, const void* W2, const float* W2s, void* out, void* ws, size_t ws_bytes,
-                  cudaStream_t stream) {
+// One launch: T tokens (at most the plan's tokens per launch) on workspace `ws` laid out as `L`.  `fused` selects the
+// fused-unit variant (L must then hold its scratch).  `cache_maps` = keep the encoded TMA descriptors in the plan.
+int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, const void* hidden, const void* Wr, const float* bias,
+             const void* W13, const float* W13s, const void* W2, const float* W2s, void* out, void* ws, cudaStream_t stream) {
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    auto map = [&](CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+        return cache_maps ? p->get_map(m, ptr, rows, cols, box_rows) : encode_2d(m, ptr, rows, cols, box_rows);
+    };
+    CUtensorMap m13, m2, mx, mh;
+    if (fused) {
+        const int TC = Plan::fused_tc(T), C = p->fused_cluster(T), grid = p->fused_grid(T), stages = p->fused_stages(T);
+        if (C < 1 || grid < C || stages < 2) return fail(MOE_ERR_OCCUPANCY, "the fused variant cannot be launched for T=%d", T);
+        if (!map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) || !map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
+            !map(&mx, w + L.xq, moe::kMaxTokens, p->H, moe::kFusedN))
+            return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+        const moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
+        const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
+        switch (TC) {
+            case 1: return launch_fused<1>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 2: return launch_fused<2>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 4: return launch_fused<4>(p, grid, C, m13, m2, mx, P, smem, stream);
+            default: return launch_fused<8>(p, grid, C, m13, m2, mx, P, smem, stream);
+        }
+    }
     const int N = p->n_hw(T);
-    const WsLayout L = p->layout(T);
-    if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
     const int stages = p->stages_for(N, T);
     if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
     const moe::SmemLayout SL = moe::smem_layout(N, T, p->K, p->E, p->H, p->I, stages, p->compact(T), p->weighted(T));
-    uint8_t* w = static_cast<uint8_t*>(ws);
-
-    CUtensorMap m13, m2, mx, mh;
-    if (!p->get_map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) ||
-        !p->get_map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
-        !p->get_map(&mx, w + L.xq, moe::kMaxTokens, p->H, N) ||
-        !p->get_map(&mh, w + L.hq, (uint64_t)p->E * p->nr(T), p->I, N))
+    if (!map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) || !map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
+        !map(&mx, w + L.xq, moe::kMaxTokens, p->H, N) || !map(&mh, w + L.hq, (uint64_t)p->E * p->nr(T), p->I, N))
         return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     const moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
     return dispatch(p, T, m13, m2, mx, mh, P, SL.total + 1024, stream);
+}
+
+int forward_chunk(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
+                  const float* W13s, const void* W2, const float* W2s, void* out, void* ws, size_t ws_bytes,
+                  cudaStream_t stream) {
+    const bool fused = p->fused(T);
+    const WsLayout L = p->layout(T, fused);
+    if (ws_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", ws_bytes, L.total, T);
+    return run_step(p, T, fused, L, true, hidden, Wr, bias, W13, W13s, W2, W2s, out, ws, stream);
 }
 
 int check_forward_args(Plan* p, int T, const void* hidden, const void* Wr, const float* bias, const void* W13,
                        const float* W13s, const void* W2, const float* W2s, void* out, void* ws) {
     if (!p) return fail(MOE_ERR_ARG, "plan is NULL");
     if (T < 1) return fail(MOE_ERR_ARG, "T must be >= 1 (got %d)", T);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) return fail(MOE_ERR_ARG, "the plan's device (%d) must be the current device", p->device);
     if (!hidden || !Wr || !W13 || !W13s || !W2 || !W2s || !out) return fail(MOE_ERR_ARG, "a tensor pointer is NULL");
     if (!ws) return fail(MOE_ERR_WORKSPACE, "workspace is NULL");
     if (p->scoring == MOE_SCORE_SIGMOID_BIAS && bias && !aligned16(bias)) return fail(MOE_ERR_ALIGN, "sel_bias not 16-byte aligned");
@@ -339,6 +452,18 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             if (value < -1 || value > 8) return fail(MOE_ERR_ARG, "split weight must be -1 (library's choice), 0 (off) or 1..8");
             for (int t = lo; t <= hi; ++t) plan->split_weight[t] = value;
             return MOE_OK;
+        case MOE_KNOB_FUSED:
+            if (value < -1 || value > 1) return fail(MOE_ERR_ARG, "fused must be -1 (library's choice), 0 or 1");
+            plan->fused_mode = value;
+            return MOE_OK;
+        case MOE_KNOB_CLUSTER:
+            if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return fail(MOE_ERR_ARG, "cluster size must be 0 (library's choice), 1, 2, 4 or 8");
+            if (value > 0 && plan->max_clusters[value] <= 0) return fail(MOE_ERR_OCCUPANCY, "clusters of %d CTAs cannot be launched on this device", value);
+            for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->cluster_knob[t] = value;
+            return MOE_OK;
+        case MOE_KNOB_STAMPS:
+            plan->take_stamps = value != 0;
+            return MOE_OK;
         default:
             return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
@@ -355,6 +480,9 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_COMPACT_MIN: *value = plan->compact_min; return MOE_OK;
         case MOE_KNOB_PDL: *value = plan->use_pdl; return MOE_OK;
         case MOE_KNOB_SPLIT_WEIGHT: *value = plan->split_weight[t]; return MOE_OK;
+        case MOE_KNOB_FUSED: *value = plan->fused_mode; return MOE_OK;
+        case MOE_KNOB_CLUSTER: *value = t <= 8 ? plan->cluster_knob[t] : 0; return MOE_OK;
+        case MOE_KNOB_STAMPS: *value = plan->take_stamps; return MOE_OK;
         default: return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
 }
@@ -385,13 +513,14 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     cudaDeviceProp prop;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
         return fail(MOE_ERR_CUDA, "cannot query the current device");
-    if (prop.major != 10) return fail(MOE_ERR_UNSUPPORTED_ARCH, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+    if (prop.major != 10 || prop.minor != 0) return fail(MOE_ERR_UNSUPPORTED_ARCH, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
     Plan* p = new Plan();
     p->H = H; p->E = E; p->I = I; p->K = top_k; p->scoring = scoring; p->renorm = renorm ? 1 : 0;
     p->routed_scale = routed_scale;
     p->device = dev;
     p->sms = prop.multiProcessorCount < moe::kMaxGrid ? prop.multiProcessorCount : moe::kMaxGrid;   // one CTA per SM, up to the size of the kernel's range tables
     p->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    p->smem_per_sm = (int)prop.sharedMemPerMultiprocessor;
     p->timeout_ns = 1000ull * 1000ull * 1000ull;
     // schedule overrides for experiments (the paper tunes its schedule offline, Section 3.4)
     // environment overrides for experiments (the same knobs moe_plan_set_knob sets)
@@ -402,6 +531,15 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     if (const char* v = getenv("MOE_B200_COMPACT_MIN")) moe_plan_set_knob(p, 0, MOE_KNOB_COMPACT_MIN, atoi(v));
     if (const char* v = getenv("MOE_B200_SPLIT_WEIGHT")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_WEIGHT, atoi(v));
     if (const char* v = getenv("MOE_B200_ROUTE_ALL")) moe_plan_set_knob(p, 0, MOE_KNOB_ROUTE_ALL_TOKENS, atoi(v));
+    // fused-unit variants: which cluster sizes can be co-resident (Section 3.2: the realised occupancy is checked, not assumed)
+    for (int C = 1; C <= 8; C *= 2) {
+        const int n1 = fused_clusters<1>(C, p->smem_optin, p->sms), n2 = fused_clusters<2>(C, p->smem_optin, p->sms);
+        const int n4 = fused_clusters<4>(C, p->smem_optin, p->sms), n8 = fused_clusters<8>(C, p->smem_optin, p->sms);
+        const int a = n1 < n2 ? n1 : n2, b = n4 < n8 ? n4 : n8;
+        p->max_clusters[C] = a < b ? a : b;
+    }
+    if (const char* v = getenv("MOE_B200_FUSED")) moe_plan_set_knob(p, 0, MOE_KNOB_FUSED, atoi(v));
+    if (const char* v = getenv("MOE_B200_CLUSTER")) moe_plan_set_knob(p, 0, MOE_KNOB_CLUSTER, atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, 64);
     if (st < 2 || p->stages_for(p->n_hw(p->chunk()), p->chunk()) < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
@@ -460,7 +598,6 @@ int moe_forward(moe_plan_t plan, int T, const void* hidden_bf16, const void* Wr_
 // ---------------------------------------------------------------------------------------------------------------
 // Entry point for callers that must not allocate: the scratch lives in a fixed array in the device image.
 // ---------------------------------------------------------------------------------------------------------------
-#define MOE_NOALLOC_SCRATCH_BYTES (24u << 20)
 static __device__ __align__(256) unsigned char g_noalloc_scratch[MOE_NOALLOC_SCRATCH_BYTES];
 
 namespace {
@@ -474,7 +611,10 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
     if (T < 1 || T > 64)
         return fail(MOE_ERR_ARG, "moe_forward_noalloc handles 1..64 tokens per call (got %d)", T);
-    const WsLayout L = plan->layout(T);
+    // the fused variant where its scratch fits the array, the general kernel where only that one's does
+    bool fused = plan->fused(T);
+    WsLayout L = plan->layout(T, fused);
+    if (fused && L.total > MOE_NOALLOC_SCRATCH_BYTES) { fused = false; L = plan->layout(T, false); }
     if (L.total > MOE_NOALLOC_SCRATCH_BYTES)
         return fail(MOE_ERR_WORKSPACE, "this shape with T=%d needs %zu bytes of scratch; the built-in array holds %u",
                     T, L.total, (unsigned)MOE_NOALLOC_SCRATCH_BYTES);
@@ -502,19 +642,8 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     if (cudaMemsetAsync(ws, 0, L.flags_end, s) != cudaSuccess)
         return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
 
-    const int N = plan->n_hw(T);
-    const int stages = plan->stages_for(N, T);
-    if (stages < 2) return fail(MOE_ERR_OCCUPANCY, "shared memory too small for a 2-stage pipeline");
-    const moe::SmemLayout SL = moe::smem_layout(N, T, plan->K, plan->E, plan->H, plan->I, stages, plan->compact(T), plan->weighted(T));
-    uint8_t* w = static_cast<uint8_t*>(ws);
-    CUtensorMap m13, m2, mx, mh;       // encoded on the stack: no descriptor cache, nothing allocated
-    if (!encode_2d(&m13, W13_fp8, (uint64_t)plan->E * 2 * plan->I, plan->H, 128) ||
-        !encode_2d(&m2, W2_fp8, (uint64_t)plan->E * plan->H, plan->I, 128) ||
-        !encode_2d(&mx, w + L.xq, moe::kMaxTokens, plan->H, N) ||
-        !encode_2d(&mh, w + L.hq, (uint64_t)plan->E * plan->nr(T), plan->I, N))
-        return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-    const moe::Params P = make_params(plan, T, stages, L, w, hidden_bf16, Wr_bf16, sel_bias, W13_scale, W2_scale, out_bf16);
-    return dispatch(plan, T, m13, m2, mx, mh, P, SL.total + 1024, s);
+    // descriptors are encoded on the stack: no descriptor cache, nothing allocated
+    return run_step(plan, T, fused, L, false, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, ws, s);
 }
 
 int moe_forward_host(moe_plan_t plan, int T, const void* hidden_host, const void* Wr_bf16, const float* sel_bias,
@@ -568,7 +697,13 @@ int moe_forward_debug(moe_plan_t plan, int T, const void* hidden_bf16, const voi
 }
 
 int moe_sync_status(moe_plan_t plan, void* workspace, moe_stream_t stream) {
-    if (!plan || !workspace) return fail(MOE_ERR_ARG, "plan or workspace is NULL");
+    if (!plan) return fail(MOE_ERR_ARG, "plan is NULL");
+    if (!workspace) {
+        // the built-in array of moe_forward_noalloc on the plan's device (resolved by that entry point's first call)
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        workspace = (plan->device >= 0 && plan->device < 64) ? g_noalloc_ptr[plan->device] : nullptr;
+        if (!workspace) return fail(MOE_ERR_ARG, "workspace is NULL and moe_forward_noalloc has not run on the plan's device");
+    }
     unsigned ctrl[8] = {0};
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     if (e == cudaSuccess) e = cudaMemcpy(ctrl, workspace, sizeof(ctrl), cudaMemcpyDeviceToHost);
@@ -594,11 +729,29 @@ int moe_tokens_per_launch(moe_plan_t plan) { return plan ? plan->chunk() : 0; }
 
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes) {
     if (!plan || T < 1) return fail(MOE_ERR_ARG, "bad arguments");
-    const int Tc = plan->cap(T), N = plan->n_hw(Tc), st = plan->stages_for(N, Tc);
+    const int Tc = plan->cap(T);
+    if (plan->fused(Tc)) {
+        const int st = plan->fused_stages(Tc);
+        if (grid) *grid = plan->fused_grid(Tc);
+        if (stages) *stages = st;
+        if (n_hw) *n_hw = moe::kFusedN;
+        if (smem_bytes) *smem_bytes = moe::fused_smem_layout(Plan::fused_tc(Tc), Tc, plan->K, plan->E, plan->H, st).total + 1024;
+        return MOE_OK;
+    }
+    const int N = plan->n_hw(Tc), st = plan->stages_for(N, Tc);
     if (grid) *grid = plan->sms;
     if (stages) *stages = st;
     if (n_hw) *n_hw = N;
     if (smem_bytes) *smem_bytes = moe::smem_layout(N, Tc, plan->K, plan->E, plan->H, plan->I, st, plan->compact(Tc), plan->weighted(Tc)).total + 1024;
+    return MOE_OK;
+}
+
+int moe_plan_variant(moe_plan_t plan, int T, int* fused, int* cluster) {
+    if (!plan || T < 1) return fail(MOE_ERR_ARG, "bad arguments");
+    const int Tc = plan->cap(T);
+    const bool f = plan->fused(Tc);
+    if (fused) *fused = f ? 1 : 0;
+    if (cluster) *cluster = f ? plan->fused_cluster(Tc) : 1;
     return MOE_OK;
 }
 

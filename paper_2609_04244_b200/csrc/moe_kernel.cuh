@@ -50,7 +50,7 @@ constexpr int kMaxGrid = 255;         // CTAs the weighted range tables of the c
 
 // control words at the head of the workspace
 // (the two arrival counters are used by alternate launches: a launch counts in one and clears the other)
-enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kExitCnt = 5, kRouteCnt2 = 6, kCtrlWords = 64 };
+enum Ctrl { kEpoch = 0, kStatus = 1, kAbort = 2, kRouteCnt = 3, kExitCnt = 5, kRouteCnt2 = 6, kQuantCnt = 8, kDoneCnt = 10, kCtrlWords = 64 };
 // device status codes
 enum DevStatus { kDevOk = 0, kDevTimeout = 1 };
 
@@ -86,7 +86,9 @@ struct Params {
     unsigned* pu_flag;  // [grid]
     unsigned* pd_flag;  // [grid]
     float* y;           // [T,K,H]
-    unsigned long long* stamps;     // [grid][16] globaltimer stamps of the phases of the last launch (diagnostics)
+    unsigned long long* ll;         // [T,E] fused variants: router logits as {launch tag, fp32 bits} words
+    float* yp;          // [T,K,I/128,H] fused variants: down-projection partial of every (token, slot, intermediate block)
+    unsigned long long* stamps;     // [grid][16] globaltimer stamps of the phases of the last launch; NULL = none taken
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -230,7 +232,7 @@ __device__ __forceinline__ bool epi_all(bool ok, int nthreads) {
     return r != 0;
 }
 
-#define MOE_STAMP(i) do { P.stamps[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
+#define MOE_STAMP(i) do { if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
 
 // K-major, 128-byte swizzled operand tile (rows of 128 bytes, 8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
@@ -612,7 +614,10 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     unsigned* e_cnt = P.e_cnt + par * kMaxPasses * E;       // counters of this launch: [pass][expert]
 #pragma unroll 1
     for (int e = cta * kThreads + tid; e < kMaxPasses * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * kMaxPasses * E + e] = 0u;
-    if (cta == 0 && tid == 0) { P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u; }
+    if (cta == 0 && tid == 0) {
+        P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u;
+        P.ctrl[kQuantCnt + (par ^ 1u)] = 0u; P.ctrl[kDoneCnt + (par ^ 1u)] = 0u;      // (counters of the fused variants, which may share the workspace)
+    }
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
 
     // ------------------------------------------------------------------ phase R: quantise + logits
