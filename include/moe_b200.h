@@ -177,7 +177,7 @@ int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int
 int moe_plan_variant(moe_plan_t plan, int T, int* fused, int* cluster);
 
 /* Diagnostics: synchronise `stream` and copy the phase time stamps of the last launch on this workspace to
- * HOST memory host_out[SMs*16] (nanoseconds of the GPU's global timer); the launch must have run with MOE_KNOB_STAMPS
+ * HOST memory host_out[SMs*32] (nanoseconds of the GPU's global timer; 32 words per CTA, the first 16 in use); the launch must have run with MOE_KNOB_STAMPS
  * set.  Fused-unit variant, per CTA: 0 start, 1 router rows published, 2 input quantised, 3 all logits gathered, 4 top-k
  * done, 5 routing metadata done, 6 first weight tile requested, 7 first weight tile landed, 8 first accumulator read,
  * 9 first partial sums parked, 10 first intermediate tile ready, 11 last down tile stored, 12 all CTAs done, 13

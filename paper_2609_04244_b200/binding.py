@@ -158,10 +158,10 @@ def moe_sync_status(plan, workspace, stream=None) -> None:
 
 
 def moe_debug_stamps(plan, workspace, grid: int, stream=None):
-    """Phase time stamps [grid, 16] (ns) of the last launch on this workspace; see include/moe_b200.h."""
+    """Phase time stamps and wait-time accumulators [grid, 32] (ns) of the last launch on this workspace; see include/moe_b200.h."""
     import numpy as np
     sms = torch.cuda.get_device_properties(workspace.device).multi_processor_count   # the call fills one row per SM
-    buf = np.zeros((max(sms, grid), 16), dtype=np.uint64)
+    buf = np.zeros((max(sms, grid), 32), dtype=np.uint64)
     _check(load_library().moe_debug_stamps(plan, _p(workspace), _stream(stream), ctypes.c_void_p(buf.ctypes.data)))
     return buf[:grid]
 

@@ -128,7 +128,7 @@ struct moe_plan {
         L.pu_flag = o;  o += align_up((size_t)G * 4, 256);
         L.pd_flag = o;  o += align_up((size_t)G * 4, 256);
         L.flags_end = o;
-        L.stamps = o;   o += align_up((size_t)G * 16 * 8, 256);
+        L.stamps = o;   o += align_up((size_t)G * moe::kStampsPerCta * 8, 256);
         L.logits = o;   o += align_up((size_t)Tc * E * 4, 256);
         L.lpart = o;    o += align_up((size_t)8 * Tc * E * 4, 256);
         L.ids = o;      o += align_up((size_t)Tc * K * 4, 256);
@@ -144,7 +144,7 @@ struct moe_plan {
         L.stage_out = o; o += align_up((size_t)Tc * H * 2, 256);    // (moe_forward_host)
         // fused variants: tagged router logits, and one down-projection partial per (token, slot, intermediate block)
         L.ll = o;       o += with_fused ? align_up((size_t)Tc * E * 8, 256) : 0;
-        L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 4, 256) : 0;
+        L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 8, 256) : 0;
         L.total = o;
         return L;
     }
@@ -155,7 +155,7 @@ struct moe_plan {
     int fused_smem_budget() const { const int half = smem_per_sm / 2 - 1024; return half < smem_optin ? half : smem_optin; }
     int fused_stages(int T) const {
         const int cap_s = stages_cap[T];
-        const int budget = cap_s > 0 ? smem_optin : fused_smem_budget();
+        const int budget = smem_optin;
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s)
             if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) return s;
         return 0;
@@ -255,7 +255,7 @@ int launch_fused(Plan* p, int grid, int C, const CUtensorMap& m13, const CUtenso
                  const moe::Params& P, int smem_bytes, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(256, 1, 1);
+    cfg.blockDim = dim3(moe::kFusedThreads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -278,7 +278,7 @@ int fused_clusters(int C, int smem_optin, int sms) {
     if (cudaFuncSetAttribute(moe::moe_fused_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) { cudaGetLastError(); return 0; }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((sms / C) * C, 1, 1);
-    cfg.blockDim = dim3(256, 1, 1);
+    cfg.blockDim = dim3(moe::kFusedThreads, 1, 1);
     cfg.dynamicSmemBytes = smem_optin;                         // a footprint that admits one CTA per SM
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -335,7 +335,9 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.pd_flag = reinterpret_cast<unsigned*>(w + L.pd_flag);
     P.y = reinterpret_cast<float*>(w + L.y);
     P.ll = reinterpret_cast<unsigned long long*>(w + L.ll);
-    P.yp = reinterpret_cast<float*>(w + L.yp);
+    P.ypl = reinterpret_cast<unsigned long long*>(w + L.yp);
+    P.fC = 1; P.fnCl = p->sms;
+    for (int r = 0; r < 9; ++r) { P.fkb[r] = 0; P.fhb[r] = 0; }
     P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
     return P;
 }
@@ -373,7 +375,11 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         if (!map(&m13, W13, (uint64_t)p->E * 2 * p->I, p->H, 128) || !map(&m2, W2, (uint64_t)p->E * p->H, p->I, 128) ||
             !map(&mx, w + L.xq, moe::kMaxTokens, p->H, moe::kFusedN))
             return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-        const moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
+        moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
+        const int KB = p->H / 128;
+        P.fC = C; P.fnCl = grid / C;
+        P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
+        for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
         switch (TC) {
             case 1: return launch_fused<1>(p, grid, C, m13, m2, mx, P, smem, stream);
@@ -575,8 +581,18 @@ int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes,
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return fail(MOE_ERR_ALIGN, "workspace must be 256-byte aligned");
     const WsLayout L = plan->layout(1);
     if (workspace_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace too small");
-    if (cudaMemsetAsync(workspace, 0, L.flags_end, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace, 0, L.flags_end, s) != cudaSuccess)
         return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
+    // Fused variants: their exchange words carry the launch tag, and the tag restarts with the control words -- so no
+    // word of those regions may keep an old tag (or, in fresh memory, something that looks like one).
+    for (int T = 1; T <= 8; ++T) {
+        if (!plan->fused(T)) continue;
+        const WsLayout F = plan->layout(T, true);
+        if (F.total > workspace_bytes) continue;             // a workspace sized for fewer tokens: that layout is never used on it
+        if (cudaMemsetAsync(static_cast<uint8_t*>(workspace) + F.ll, 0, F.total - F.ll, s) != cudaSuccess)
+            return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
     return MOE_OK;
 }
 
@@ -638,8 +654,10 @@ int moe_forward_noalloc(moe_plan_t plan, int T, const void* hidden_bf16, const v
     int rc = check_forward_args(plan, T, hidden_bf16, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, out_bf16, ws);
     if (rc != MOE_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // The array keeps whatever the previous call left: start every call from cleared control words and flags.
-    if (cudaMemsetAsync(ws, 0, L.flags_end, s) != cudaSuccess)
+    // The array keeps whatever the previous call left: start every call from cleared status, counters and flags.  The
+    // launch epoch (the first word) is NOT cleared: it keeps counting across calls, which is what tells this call's
+    // flags and tagged words from the ones earlier calls left in the array.
+    if (cudaMemsetAsync(static_cast<uint8_t*>(ws) + 4, 0, L.flags_end - 4, s) != cudaSuccess)
         return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
 
     // descriptors are encoded on the stack: no descriptor cache, nothing allocated
@@ -720,7 +738,7 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
     const WsLayout L = plan->layout(1);
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     if (e == cudaSuccess)
-        e = cudaMemcpy(host_out, static_cast<const uint8_t*>(workspace) + L.stamps, (size_t)plan->sms * 16 * 8, cudaMemcpyDeviceToHost);
+        e = cudaMemcpy(host_out, static_cast<const uint8_t*>(workspace) + L.stamps, (size_t)plan->sms * moe::kStampsPerCta * 8, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail(MOE_ERR_CUDA, "CUDA error while reading stamps: %s", cudaGetErrorString(e));
     return MOE_OK;
 }

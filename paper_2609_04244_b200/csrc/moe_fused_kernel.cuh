@@ -38,13 +38,16 @@ namespace moe {
 
 constexpr int kFusedN = 16;                                   // MMA N of the fused variants (tokens 0..7 are columns 0..7)
 constexpr int kFusedStage = kATileBytes + kFusedN * kBlock;    // weight tile + activation tile
-constexpr int kFusedTmemCols = 256;                            // 8 accumulator buffers x (gate 16 + up 16) columns
+constexpr int kFusedTmemBufs = 4;                              // accumulator buffers of 2 x 16 columns, one per MMA issuer
+constexpr int kFusedTmemCols = 128;
+constexpr int kFusedThreads = 288;                             // 9 warps
 constexpr int kFusedMaxRows = 4;                               // router rows per CTA: ceil(kMaxExperts / 128)
 
 // ---------------------------------------------------------------------------------------------
 // cluster / distributed-shared-memory wrappers
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_id_x() { uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r; }
 __device__ __forceinline__ uint32_t cluster_nctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -72,6 +75,19 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
+// named barriers over a subset of the CTA's warps
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+__device__ __forceinline__ void named_bar_arrive(int id, int nthreads) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+__device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, %2, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)ok), "r"(id), "r"(nthreads) : "memory");
+    return r != 0;
+}
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
     unsigned long long v;
     asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -92,8 +108,8 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
     int o = 0;
     L.ring_off = o; o += stages * kFusedStage;                 // also the routing scratch (keys and score values) before the stream starts
     L.hq_off = o;   o += 2 * kFusedN * kBlock;                 // intermediate FP8 tile of the unit in flight, double-buffered (1024-byte aligned)
-    L.part_off = o; o += 2 * 2 * TC * kBlock * 4;              // this CTA's partial gate/up sums [slot][gate TC | up TC][128 rows]
-    L.bar_off = o;  o += (3 * kMaxStages + 2 * kMaxTmemBufs + 12) * 8;
+    L.part_off = o; o += 2 * 2 * TC * kBlock * 4;              // this CTA's partial gate/up sums [slot][gate TC | up TC][128 rows]; later the reduction scratch
+    L.bar_off = o;  o += (2 * kMaxStages + 2 * kFusedTmemBufs + 12) * 8;
     L.misc_off = o; o += 64;
     L.ids_off = o;  o += T * K * 4;
     L.w_off = o;    o += T * K * 4;
@@ -112,21 +128,23 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
 
 // ---------------------------------------------------------------------------------------------
 // the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8 >= T).
+// Warps: 0 producer (weight and activation tiles), 1, 2, 3 and 8 MMA issuers, 4..7 accumulator warps; warp 8 keeps
+// house during the routing phase.
 // ---------------------------------------------------------------------------------------------
 template <int TC>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(kFusedThreads, 1)
 moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                  const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ Params P) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
     constexpr int N = kFusedN;
-    constexpr int kThreads = 256, kWarps = 8, kEpiThreads = 128;
-    constexpr int kTmemBufs = 8;
+    constexpr int kMain = 256, kMainWarps = 8, kEpiThreads = 128;     // warps 0..7 share the routing phase; warp 8 keeps house meanwhile
+    constexpr int kBufs = kFusedTmemBufs, kBufCols = 2 * N;          // an accumulator buffer = two 16-column halves
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
-    const int C = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
-    const int cl = cta / C, nCl = G / C;                         // clusters are consecutive CTAs of a 1-D grid
+    const int C = P.fC, nCl = P.fnCl, rank = (int)cluster_ctarank();
+    const int cl = (int)cluster_id_x();
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock;
     const int S = P.stages;
@@ -134,11 +152,11 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     const int TS = (T + 3) & ~3;
 
     uint64_t* bars = (uint64_t*)(smem + L.bar_off);
-    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages), bar_fullb = smem_u32(bars + 2 * kMaxStages);
-    const uint32_t bar_tfull = smem_u32(bars + 3 * kMaxStages), bar_tempty = smem_u32(bars + 3 * kMaxStages + kMaxTmemBufs);
-    const uint32_t bar_x = smem_u32(bars + 3 * kMaxStages + 2 * kMaxTmemBufs);
-    const uint32_t bar_hq = bar_x, bar_xfull = bar_x + 16, bar_xfree = bar_x + 32, bar_drain = bar_x + 48;   // 2 + 2 + 2 + 2 (+ spare)
-    uint32_t* misc = (uint32_t*)(smem + L.misc_off);   // [0] tmem base, [1] U, [2] alive, [3] accumulator give-up, [4],[5] groups issued by the two MMA issuers
+    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
+    const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kBufs);
+    const uint32_t bar_x = smem_u32(bars + 2 * kMaxStages + 2 * kBufs);
+    const uint32_t bar_hq = bar_x, bar_xfull = bar_x + 16, bar_xfree = bar_x + 32, bar_drain = bar_x + 48;   // 2 + 2 + 2 + 4
+    uint32_t* misc = (uint32_t*)(smem + L.misc_off);   // [0] tmem base, [1] U, [3] accumulator give-up, [6] quantised input published (1) or given up (2)
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
@@ -155,25 +173,25 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmW13); tma_prefetch_desc(&tmW2); tma_prefetch_desc(&tmXq);
-        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_fullb + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < kBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_hq + 8 * b, 1);
             mbar_init(bar_xfull + 8 * b, 4 * C);             // one arrival per accumulator warp of every CTA of the cluster
             mbar_init(bar_xfree + 8 * b, 4 * C);
-            mbar_init(bar_drain + 8 * b, 1);
         }
-        misc[3] = 0u; misc[4] = 0u; misc[5] = 0u;
+        for (int b = 0; b < 4; ++b) mbar_init(bar_drain + 8 * b, 1);
+        misc[3] = 0u; misc[6] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kFusedTmemCols); tmem_relinquish(); }
 #pragma unroll 1
-    for (int e = tid; e < 2 * E; e += kThreads) s_mask[e] = 0ull;
+    for (int e = tid; e < 2 * E; e += kFusedThreads) s_mask[e] = 0ull;
     // This CTA's router rows: ask L2 for them now.  (Weights are not written by the previous launch, and a prefetch
     // reads nothing into the SM.)
 #pragma unroll 1
     for (int e = cta; e < E; e += G)
-        for (int l = tid; l < H / 64; l += kThreads) prefetch_l2(reinterpret_cast<const char*>(P.Wr + (size_t)e * H) + l * 128);
+        for (int l = tid; l < H / 64; l += kFusedThreads) prefetch_l2(reinterpret_cast<const char*>(P.Wr + (size_t)e * H) + l * 128);
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
     // every CTA of the cluster has initialised its barriers before anyone arrives on them remotely
     cluster_arrive();
@@ -182,19 +200,16 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 
     Waiter wt;
     wt.init(P.ctrl, P.timeout_ns);
-    const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
-    const unsigned par = tag & 1u;
+    // The launch tag.  A relaxed load: everything the previous launch wrote is visible after the wait above, and an
+    // acquire here would hold back the loads of the router phase for an L2 round trip.
+    unsigned tag;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(tag) : "l"(P.ctrl + kEpoch) : "memory");
+    tag += 1u;
     if (tid == 0) MOE_STAMP(0);
-    // counters of the other launch parity start from zero next time (this launch counts in its own)
-    if (cta == 0 && tid == 0) {
-        P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u;
-        P.ctrl[kQuantCnt + (par ^ 1u)] = 0u; P.ctrl[kDoneCnt + (par ^ 1u)] = 0u;
-    }
-#pragma unroll 1
-    for (int e = cta * kThreads + tid; e < kMaxPasses * E; e += G * kThreads) P.e_cnt[(par ^ 1u) * kMaxPasses * E + e] = 0u;
+    __syncwarp();             // (a lone lane that took a stamp rejoins its warp here, not somewhere inside the next loop)
 
     // ------------------------------------------------------------------ router logits of this CTA's experts (Section 3.3)
-    {
+    if (warp < kMainWarps) {
         const int chunks = H / 8;                                 // 16-byte chunks per row
         int nrows = 0;
 #pragma unroll 1
@@ -204,7 +219,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             for (int t = 0; t < TC; ++t) acc[t] = 0.f;
             const uint4* wrow = reinterpret_cast<const uint4*>(P.Wr + (size_t)e * H);
 #pragma unroll 2
-            for (int c = tid; c < chunks; c += kThreads) {
+            for (int c = tid; c < chunks; c += kMain) {
                 const uint4 wv = __ldg(wrow + c);
                 uint4 xv[TC];
 #pragma unroll
@@ -227,23 +242,22 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 if (lane == 0) s_red[(warp * kFusedMaxRows + nrows) * 8 + t] = acc[t];
             }
         }
-        __syncthreads();
+        named_bar_sync(2, kMain);
         if (tid < nrows * TC) {
             const int r = tid / TC, t = tid - r * TC;
             if (t < T) {
                 float v = 0.f;
 #pragma unroll
-                for (int w = 0; w < kWarps; ++w) v += s_red[(w * kFusedMaxRows + r) * 8 + t];
+                for (int w = 0; w < kMainWarps; ++w) v += s_red[(w * kFusedMaxRows + r) * 8 + t];
                 st_relaxed_u64(P.ll + (size_t)t * E + cta + r * G, ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v));
             }
         }
         if (tid == 0) MOE_STAMP(1);
-    }
-    // ------------------------------------------------------------------ input quantisation (Section 4.1), spread over the grid
-    {
+        __syncwarp();
+        // -------------------------------------------------------------- input quantisation (Section 4.1), spread over the grid
         const int groups = T * KBu;
 #pragma unroll 1
-        for (int p = (G - 1 - cta) * kWarps + warp; p < groups; p += G * kWarps) {   // from the last CTA down: the first ones have router rows
+        for (int p = (G - 1 - cta) * kMainWarps + warp; p < groups; p += G * kMainWarps) {   // from the last CTA down: the first ones have router rows
             const int t = p / KBu, g = p % KBu;
             const uint2 raw = *reinterpret_cast<const uint2*>(P.hidden + (size_t)t * H + g * kBlock + lane * 4);
             const float x0 = __uint_as_float(raw.x << 16), x1 = __uint_as_float(raw.x & 0xFFFF0000u);
@@ -256,27 +270,51 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             if (lane == 0) P.xs[p] = s;
         }
         fence_proxy_async();                                    // generic writes of xq -> the async proxy (bulk-tensor copies) of every CTA
-        __syncthreads();
-        if (tid == 0) { red_release_add(P.ctrl + kQuantCnt + par, 1u); MOE_STAMP(2); }
+        named_bar_arrive(3, kFusedThreads);                     // hand over to the housekeeping warp, do not wait for it
+    } else {
+        // ---------------------------------------------------------- housekeeping warp: everything that costs L2 round
+        // trips but is not needed before the first activation tile.  Publish this CTA's share of the quantised input
+        // (the release waits for the CTA's stores), wait until every CTA has, fetch the input scales.
+        const unsigned par = tag & 1u;
+        if (cta == 0 && lane == 0) {      // counters of the other launch parity start from zero next time
+            P.ctrl[kRouteCnt + (par ^ 1u)] = 0u; P.ctrl[kRouteCnt2 + (par ^ 1u)] = 0u;
+            P.ctrl[kQuantCnt + (par ^ 1u)] = 0u; P.ctrl[kDoneCnt + (par ^ 1u)] = 0u;
+        }
+#pragma unroll 1
+        for (int e = cta * 32 + lane; e < kMaxPasses * E; e += G * 32) P.e_cnt[(par ^ 1u) * kMaxPasses * E + e] = 0u;
+        named_bar_sync(3, kFusedThreads);
+        bool okq = true;
+        if (lane == 0) {
+            red_release_add(P.ctrl + kQuantCnt + par, 1u);
+            MOE_STAMP(2);
+            okq = wt.flag(P.ctrl + kQuantCnt + par, (unsigned)G, 22);
+        }
+        okq = __shfl_sync(0xffffffffu, okq, 0);
+        if (okq) {
+#pragma unroll 1
+            for (int i = lane; i < T * KBu; i += 32) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
+        }
+        __syncwarp();
+        if (lane == 0) misc[6] = okq ? 1u : 2u;
     }
     const uint32_t tmem_base = misc[0];
 
     // ------------------------------------------------------------------ gather all logits: poll the tagged words themselves
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem);
     float* s_val = reinterpret_cast<float*>(smem) + T * E;
-    bool alive;
-    {
+    bool alive = true;
+    if (warp < kMainWarps) {
         const bool softmax = (P.scoring == 0);
         bool ok = true;
 #pragma unroll 1
-        for (int p0 = tid; p0 < T * E && ok; p0 += 8 * kThreads) {          // eight words in flight per thread
+        for (int p0 = tid; p0 < T * E && ok; p0 += 8 * kMain) {              // eight words in flight per thread
             unsigned long long v[8];
             unsigned pending = 0u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) if (p0 + j * kThreads < T * E) pending |= 1u << j;
+            for (int j = 0; j < 8; ++j) if (p0 + j * kMain < T * E) pending |= 1u << j;
             for (uint32_t it = 1; pending; ++it) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(P.ll + p0 + j * kThreads);
+                for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(P.ll + p0 + j * kMain);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) if ((pending & (1u << j)) && (unsigned)(v[j] >> 32) == tag) pending &= ~(1u << j);
                 if (pending && (it & 63u) == 0 && wt.expired(20)) { ok = false; break; }
@@ -284,7 +322,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             if (!ok) break;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int p = p0 + j * kThreads;
+                const int p = p0 + j * kMain;
                 if (p < T * E) {
                     const float l = __uint_as_float((unsigned)v[j]);
                     if (cta == 0) P.logits[p] = l;
@@ -300,83 +338,100 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 }
             }
         }
-        alive = __syncthreads_and(ok && !wt.dead) != 0;
+        alive = named_bar_and(2, kMain, ok && !wt.dead);
         if (tid == 0) MOE_STAMP(3);
-    }
-
-    // ------------------------------------------------------------------ top-k for every token, in every CTA (Section 4.1)
-    if (alive) {
+        __syncwarp();
+        // -------------------------------------------------------------- top-k for every token, in every CTA (Section 4.1)
+        if (alive) {
 #pragma unroll 1
-        for (int t = warp; t < T; t += kWarps) {
-            if (E <= 128) route_select<4>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
-            else if (E <= 256) route_select<8>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
-            else route_select<16>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
+            for (int t = warp; t < T; t += kMainWarps) {
+                if (E <= 128) route_select<4>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
+                else if (E <= 256) route_select<8>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
+                else route_select<16>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
+            }
         }
-    }
-    __syncthreads();
-    if (tid == 0) MOE_STAMP(4);
-    // ------------------------------------------------------------------ routing metadata: active experts (warp 0), routed pairs (warps 4..7)
-    if (alive && warp == 0) {
-        int base = 0;
-#pragma unroll 1
-        for (int e0 = 0; e0 < E; e0 += 32) {
-            const int e = e0 + lane;
-            const bool on = (e < E) && (s_mask[2 * e] != 0ull);
-            const unsigned b = __ballot_sync(0xffffffffu, on);
-            if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
-            base += __popc(b);
-        }
-        if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
-    }
-    if (alive && warp >= kEpiWarp0) {
-        // (token, slot) pairs grouped by expert, tokens ascending: entry r of expert e = its r-th token and the slot e holds for it
-        const int etid = tid - kEpiWarp0 * 32;
-        if (warp == kEpiWarp0) {
+        named_bar_sync(2, kMain);
+        if (tid == 0) MOE_STAMP(4);
+        __syncwarp();
+        // -------------------------------------------------------------- routing metadata: active experts (warp 0), routed pairs (warps 4..7)
+        if (alive && warp == 0) {
             int base = 0;
 #pragma unroll 1
             for (int e0 = 0; e0 < E; e0 += 32) {
-                const int c = (e0 + lane < E) ? __popcll(s_mask[2 * (e0 + lane)]) : 0;
-                int incl = c;
+                const int e = e0 + lane;
+                const bool on = (e < E) && (s_mask[2 * e] != 0ull);
+                const unsigned b = __ballot_sync(0xffffffffu, on);
+                if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
+                base += __popc(b);
+            }
+            if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
+        }
+        if (alive && warp >= kEpiWarp0) {
+            // (token, slot) pairs grouped by expert, tokens ascending: entry r of expert e = its r-th token and the slot e holds for it
+            const int etid = tid - kEpiWarp0 * 32;
+            if (warp == kEpiWarp0) {
+                int base = 0;
+#pragma unroll 1
+                for (int e0 = 0; e0 < E; e0 += 32) {
+                    const int c = (e0 + lane < E) ? __popcll(s_mask[2 * (e0 + lane)]) : 0;
+                    int incl = c;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-                if (e0 + lane < E) s_poff[e0 + lane] = base + incl - c;
-                base += __shfl_sync(0xffffffffu, incl, 31);
+                    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                    if (e0 + lane < E) s_poff[e0 + lane] = base + incl - c;
+                    base += __shfl_sync(0xffffffffu, incl, 31);
+                }
+            }
+            epi_bar(kEpiThreads);
+#pragma unroll 1
+            for (int pi = etid; pi < T * K; pi += kEpiThreads) {
+                const int t = div_small(pi, K), ex = s_ids[pi];
+                s_pair[s_poff[ex] + __popcll(s_mask[2 * ex] & ((1ull << t) - 1ull))] = (unsigned short)(t | ((pi - t * K) << 8));
             }
         }
-        epi_bar(kEpiThreads);
-#pragma unroll 1
-        for (int pi = etid; pi < T * K; pi += kEpiThreads) {
-            const int t = div_small(pi, K), ex = s_ids[pi];
-            s_pair[s_poff[ex] + __popcll(s_mask[2 * ex] & ((1ull << t) - 1ull))] = (unsigned short)(t | ((pi - t * K) << 8));
-        }
     }
-    __syncthreads();
+    alive = __syncthreads_and(alive && !wt.dead) != 0;          // (the housekeeping warp joins here)
+    if (misc[6] != 1u) alive = false;                           // the quantised input never arrived: its wait has recorded why
     if (tid == 0) MOE_STAMP(5);
+    __syncwarp();
     const int U = alive ? (int)misc[1] : 0;
     const int nU = U * IB;                                       // units of this step
-    const int n = (cl < nU) ? (nU - cl + nCl - 1) / nCl : 0;     // units of this cluster: cl, cl + nCl, ...
+    const int n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units of this cluster: cl, cl + nCl, ... (grid_magic divides by the cluster count here)
     // this CTA's share of every unit: K blocks [kb_lo, kb_hi) of the gate/up rows, row blocks [hb_lo, hb_hi) of W2
-    const int kb_lo = rank * KBu / C, kb_hi = (rank + 1) * KBu / C, nk = kb_hi - kb_lo;
-    const int hb_lo = (C - 1 - rank) * HB / C, hb_hi = (C - rank) * HB / C, nh = hb_hi - hb_lo;
+    const int kb_lo = P.fkb[rank], kb_hi = P.fkb[rank + 1], nk = kb_hi - kb_lo;
+    const int hb_lo = P.fhb[rank], hb_hi = P.fhb[rank + 1], nh = hb_hi - hb_lo;
     auto unit_of = [&](int s, int& e, int& ib) { const int u = cl + s * nCl; const int a = div_small(u, IB); ib = u - a * IB; e = s_act[a]; };
 
-    // Stream order of this CTA (same in every role): for s = 0..n: the gate/up k-steps of unit s (if s < n), then the
-    // down tiles of unit s-1 (if s >= 1).  A gate/up k-step is two stages and one accumulation group, a down tile is
-    // one stage and one group.
-    // ------------------------------------------------------------------ role: weight-tile producer
+    // Stream order of this CTA (same in every role): for s = 0..n: the gate/up groups of unit s (if s < n), then the
+    // down groups of unit s-1 (if s >= 1).  A group is what one accumulator buffer holds: two weight tiles -- the gate
+    // and the up tile of one K block (columns [0,16) and [16,32), activation tile next to the gate tile), or two
+    // consecutive row blocks of the W2 column block (activation operand = the on-chip intermediate tile) -- or a
+    // single last W2 tile.  One mbarrier per group in each direction: the group's tiles land on the `full` barrier of
+    // its first stage and are released through that stage's `empty` barrier, so a stage that was the second of a pair
+    // needs no wait of its own (the ring is refilled in order: its pair-mate's release came first).
+    const int NI = (S >> 1) < kBufs ? (S >> 1) : kBufs;           // MMA issuers = accumulator buffers in use
+    const int Ntot = n * (2 * nk + nh);                          // weight tiles of this CTA
+    // ------------------------------------------------------------------ role: producer (weight tiles and activation tiles)
     if (warp == 0) {
         if (lane == 0 && alive && n > 0) {
             const uint64_t stream_once = l2_policy_evict_first();
+            fence_proxy_async();                 // xq was written with ordinary stores by other CTAs (acquired by the housekeeping warp)
             int cur = 0, st = 0;
-            uint32_t ph = 1u;
-            uint32_t dst = smem_u32(smem), full = bar_full, empty = bar_empty;
-            auto put = [&](const CUtensorMap* m, int x, int y) -> bool {
-                if (!wt.mbar(empty, ph, 21)) return false;
-                mbar_expect_tx(full, (uint32_t)kATileBytes);
-                tma_load_2d_hint(dst, m, x, y, full, stream_once);
-                ++cur;
-                dst += kFusedStage; full += 8; empty += 8;
-                if (++st == S) { st = 0; ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; }
+            uint32_t cntpar = 0u, second = 0u;   // per stage: parity of the number of groups it anchored; last filled as the second tile of a pair
+            // one group: 1 or 2 weight tiles (rows y0 / y1 of `m`, column x) and, for gate/up groups, the activation tile of K block xq_kb
+            auto put = [&](const CUtensorMap* m, int x0, int y0, int x1, int y1, int ntiles, int xq_kb) -> bool {
+                const int st0 = st, st1 = (st + 1 == S) ? 0 : st + 1;
+                if (!((second >> st0) & 1u) && !wt.mbar(bar_empty + 8 * st0, ((cntpar >> st0) & 1u) ^ 1u, 21)) return false;
+                if (ntiles == 2 && !((second >> st1) & 1u) && !wt.mbar(bar_empty + 8 * st1, ((cntpar >> st1) & 1u) ^ 1u, 21)) return false;
+                const uint32_t full = bar_full + 8 * st0, dst0 = smem_u32(smem) + (uint32_t)st0 * kFusedStage;
+                mbar_expect_tx(full, (uint32_t)(ntiles * kATileBytes + (xq_kb >= 0 ? N * kBlock : 0)));
+                tma_load_2d_hint(dst0, m, x0, y0, full, stream_once);
+                if (xq_kb >= 0) tma_load_2d(dst0 + kATileBytes, &tmXq, xq_kb * kBlock, 0, full);   // rows 0..15 of xq (tokens beyond T are never read back)
+                if (ntiles == 2) tma_load_2d_hint(smem_u32(smem) + (uint32_t)st1 * kFusedStage, m, x1, y1, full, stream_once);
+                cntpar ^= 1u << st0;
+                second &= ~(1u << st0);
+                if (ntiles == 2) second |= 1u << st1;
+                cur += ntiles;
+                st += ntiles; if (st >= S) st -= S;
                 return true;
             };
             MOE_STAMP(6);
@@ -384,176 +439,117 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 if (s < n) {
                     int e, ib;
                     unit_of(s, e, ib);
-                    for (int k = kb_lo; k < kb_hi; ++k) {
-                        if (!put(&tmW13, k * kBlock, e * 2 * I + ib * kBlock)) break;
-                        if (!put(&tmW13, k * kBlock, e * 2 * I + I + ib * kBlock)) break;
-                    }
+                    const int yg = e * 2 * I + ib * kBlock;
+                    for (int k = kb_lo; k < kb_hi; ++k)
+                        if (!put(&tmW13, k * kBlock, yg, k * kBlock, yg + I, 2, k)) break;
                 }
                 if (s >= 1 && !wt.dead) {
                     int e, ib;
                     unit_of(s - 1, e, ib);
-                    for (int h = hb_lo; h < hb_hi; ++h)
-                        if (!put(&tmW2, ib * kBlock, e * H + h * kBlock)) break;
+                    for (int h = hb_lo; h < hb_hi; h += 2)
+                        if (!put(&tmW2, ib * kBlock, e * H + h * kBlock, ib * kBlock, e * H + (h + 1) * kBlock, (h + 1 < hb_hi) ? 2 : 1, -1)) break;
                 }
             }
-            if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight
-                for (int it = (cur > S ? cur - S : 0); it < cur; ++it)
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
+            if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight: every barrier it may have armed in the last lap
+                for (int s = 0; s < S; ++s)
+                    for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
             }
         }
         __syncwarp();
     }
-    // ------------------------------------------------------------------ role: activation-tile producer
-    else if (warp == 2) {
-        if (lane == 0 && alive && n > 0) {
-            int cur = 0, st = 0;
-            uint32_t ph = 1u;
-            uint32_t dst = smem_u32(smem) + kATileBytes, full = bar_fullb, empty = bar_empty;
-            auto step = [&]() { ++cur; dst += kFusedStage; full += 8; empty += 8; if (++st == S) { st = 0; ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; } };
-            // the quantised input of every token is in the workspace once all CTAs have counted themselves
-            if (wt.flag(P.ctrl + kQuantCnt + par, (unsigned)G, 22)) {
-                fence_proxy_async();
-                for (int s = 0; s <= n && !wt.dead; ++s) {
-                    if (s < n) {
-                        for (int k = kb_lo; k < kb_hi; ++k) {
-                            if (!wt.mbar(empty, ph, 23)) break;
-                            mbar_expect_tx(full, (uint32_t)(N * kBlock));
-                            tma_load_2d(dst, &tmXq, k * kBlock, 0, full);        // rows 0..15 of xq (tokens beyond T are never read back)
-                            step();
-                            if (!wt.mbar(empty, ph, 23)) break;
-                            mbar_arrive(full);                                   // the up tile shares the gate stage's activation tile
-                            step();
-                        }
-                    }
-                    if (s >= 1 && !wt.dead) {
-                        for (int h = hb_lo; h < hb_hi; ++h) {
-                            if (!wt.mbar(empty, ph, 23)) break;
-                            mbar_arrive(full);                                   // the down tile's activation operand is the on-chip intermediate tile
-                            step();
-                        }
-                    }
-                }
-            }
-            if (wt.dead) {
-                for (int it = (cur > S ? cur - S : 0); it < cur; ++it)
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_fullb + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
-            }
-        }
-        __syncwarp();
-    }
-    // ------------------------------------------------------------------ role: MMA issuers (alternate accumulation groups)
-    // The two threads share the stage ring; as in moe_kernel.cuh each publishes how many groups it has issued and
-    // neither runs S/2 or more groups ahead of the other, so a parity wait on a stage is never a lap off.
-    else if (warp == 1 || warp == 3) {
-        if (lane == 0 && alive && n > 0) {
+    // ------------------------------------------------------------------ role: MMA issuers
+    // Measured in this kernel: one group (two waits, a fence, eight tcgen05.mma, two commits) occupies its issuing thread
+    // for about 1100 cycles, far longer than the tensor pipe needs for it.  So up to four threads (warps 1, 2, 3, 8)
+    // take the groups in turn, each with the accumulator buffer of its own number; all of them walk the whole sequence
+    // to keep the stage positions and barrier phases.  Commits are kept few -- one `empty` and one `full` per group,
+    // no `empty` for stages that are never refilled.  With NI issuers and NI buffers nobody runs more than NI groups
+    // ahead of the slowest (a buffer is handed back only after every earlier group was read), and NI <= S/2 groups is
+    // less than a lap of the ring: a parity wait on a stage can never be a phase off.
+    else if (warp < kEpiWarp0 || warp == 8) {
+        const int iss = (warp == 8) ? 3 : warp - 1;
+        if (lane == 0 && alive && n > 0 && iss < NI) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
             const uint32_t ring = smem_u32(smem);
-            const int who = warp >> 1;
-            int st = 0, g = 0;
-            uint32_t ph = 0;
-            auto advance = [&](int k) { st += k; while (st >= S) { st -= S; ph ^= 1u; } };
-            int other_seen = 0;
+            int st = 0, j = 0, turn = 0;
+            uint32_t fpar = 0u;                  // per stage: parity of the next phase of its `full` barrier
+            uint32_t tpar = 1u;                  // parity to wait for on this issuer's `tempty` barrier
             bool first = true;
-            // common head of a group: accumulator buffer free, the other issuer not too far behind
-            auto head = [&]() -> bool {
-                const int buf = g & (kTmemBufs - 1);
-                if (!wt.mbar(bar_tempty + 8 * buf, (uint32_t)((g >> 3) & 1) ^ 1u, 24)) return false;
-                const int q = g - (S >> 1);
-                const int thr = ((q & 1) != who) ? q + 1 : q;
-                if (other_seen < thr) {
-                    volatile uint32_t* other = misc + 4 + (who ^ 1);
-                    for (uint32_t i = 1; (other_seen = (int)*other) < thr; ++i)
-                        if ((i & 255u) == 0 && wt.expired(25)) return false;
+            // one group: tile(s) at stage st (and st + 1), activation operand at b_addr (0: next to the first tile)
+            auto group = [&](int ntiles, uint32_t b_addr) -> bool {
+                const int st0 = st, st1 = (st + 1 == S) ? 0 : st + 1;
+                const bool mine = (turn == iss);
+                const bool release = (j + S < Ntot);              // a later tile will take this stage
+                st += ntiles; if (st >= S) st -= S;
+                j += ntiles;
+                if (++turn == NI) turn = 0;
+                const uint32_t fp = (fpar >> st0) & 1u;
+                fpar ^= 1u << st0;
+                if (!mine) return true;
+                if (!wt.mbar(bar_tempty + 8 * iss, tpar, 24)) return false;
+                tpar ^= 1u;
+                if (!wt.mbar(bar_full + 8 * st0, fp, 26)) return false;
+                if (first && iss == 0) { MOE_STAMP(7); first = false; }
+                const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)kFusedStage;
+                const uint64_t b_desc = make_smem_desc(b_addr ? b_addr : a0 + kATileBytes);
+                const uint32_t d = tmem_base + (uint32_t)(iss * kBufCols);
+                tc_fence_after();
+                {
+                    const uint64_t a_desc = make_smem_desc(a0);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) umma_f8(d, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc, kk > 0 ? 1u : 0u);
                 }
+                if (ntiles == 2) {
+                    const uint64_t a_desc = make_smem_desc(ring + (uint32_t)st1 * (uint32_t)kFusedStage);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) umma_f8(d + N, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc, kk > 0 ? 1u : 0u);
+                }
+                if (release) umma_commit(bar_empty + 8 * st0);
+                umma_commit(bar_tfull + 8 * iss);
                 return true;
             };
             for (int s = 0; s <= n && !wt.dead; ++s) {
-                if (s < n) {
-                    for (int k = 0; k < nk && !wt.dead; ++k, ++g) {
-                        if ((g & 1) != who) { advance(2); continue; }
-                        if (!head()) break;
-                        const int buf = g & (kTmemBufs - 1);
-                        const int st0 = st;
-                        const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)kFusedStage;
-                        if (!wt.mbar(bar_full + 8 * st0, ph, 26) || !wt.mbar(bar_fullb + 8 * st0, ph, 26)) break;
-                        const uint64_t b_desc = make_smem_desc(a0 + kATileBytes);
-                        const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
-                        if (first && who == 0) { MOE_STAMP(7); first = false; }
-                        tc_fence_after();
-                        {
-                            const uint64_t a_desc = make_smem_desc(a0);
-#pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) umma_f8(d, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc, kk > 0 ? 1u : 0u);
-                        }
-                        advance(1);
-                        const int st1 = st;
-                        if (!wt.mbar(bar_full + 8 * st1, ph, 26) || !wt.mbar(bar_fullb + 8 * st1, ph, 26)) break;
-                        tc_fence_after();
-                        {
-                            const uint64_t a_desc = make_smem_desc(ring + (uint32_t)st1 * (uint32_t)kFusedStage);
-#pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) umma_f8(d + N, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc, kk > 0 ? 1u : 0u);
-                        }
-                        umma_commit(bar_empty + 8 * st0);
-                        umma_commit(bar_empty + 8 * st1);
-                        umma_commit(bar_tfull + 8 * buf);
-                        *(volatile uint32_t*)(misc + 4 + who) = (uint32_t)(g + 1);
-                        advance(1);
-                    }
-                }
+                if (s < n)
+                    for (int k = 0; k < nk; ++k)
+                        if (!group(2, 0u)) break;
                 if (s >= 1 && !wt.dead) {
                     const int slot = (s - 1) & 1;
-                    bool hq_ok = false;
-                    for (int h = 0; h < nh && !wt.dead; ++h, ++g) {
-                        if ((g & 1) != who) { advance(1); continue; }
-                        if (!head()) break;
-                        if (!hq_ok) {                      // the intermediate tile of unit s-1 is in shared memory (written by the accumulator warps)
-                            if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)(((s - 1) >> 1) & 1), 27)) break;
-                            hq_ok = true;
-                        }
-                        const int buf = g & (kTmemBufs - 1);
-                        const int st0 = st;
-                        if (!wt.mbar(bar_full + 8 * st0, ph, 26) || !wt.mbar(bar_fullb + 8 * st0, ph, 26)) break;
-                        const uint64_t a_desc = make_smem_desc(ring + (uint32_t)st0 * (uint32_t)kFusedStage);
-                        const uint64_t b_desc = make_smem_desc(smem_u32(s_hq) + (uint32_t)(slot * N * kBlock));
-                        const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
-                        tc_fence_after();
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) umma_f8(d, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc, kk > 0 ? 1u : 0u);
-                        umma_commit(bar_empty + 8 * st0);
-                        umma_commit(bar_tfull + 8 * buf);
-                        *(volatile uint32_t*)(misc + 4 + who) = (uint32_t)(g + 1);
-                        advance(1);
-                    }
+                    // the intermediate tile of unit s-1 is in shared memory (written by the accumulator warps)
+                    if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)(((s - 1) >> 1) & 1), 27)) break;
+                    for (int h = 0; h < nh; h += 2)
+                        if (!group((h + 1 < nh) ? 2 : 1, smem_u32(s_hq) + (uint32_t)(slot * N * kBlock))) break;
                 }
             }
             if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
-                umma_commit(bar_drain + 8 * (uint32_t)who);
-                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain + 8 * (uint32_t)who, 0); ++i) {}
+                umma_commit(bar_drain + 8 * (uint32_t)iss);
+                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain + 8 * (uint32_t)iss, 0); ++i) {}
             }
         }
         __syncwarp();
     }
     // ------------------------------------------------------------------ role: accumulator / epilogue warps
-    else if (warp >= kEpiWarp0) {
+    else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         bool first_acc = true;
-        if (alive) {
-            // input scales [K block][token]: behind the same counter as the quantised input
-            const bool got = (etid == 0) ? wt.flag(P.ctrl + kQuantCnt + par, (unsigned)G, 28) : true;
-            if (!epi_all(got, kEpiThreads)) { wt.dead = true; }
-            else {
-#pragma unroll 1
-                for (int i = etid; i < T * KBu; i += kEpiThreads) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
-                epi_bar(kEpiThreads);
-            }
-        }
-        int g = 0;                                             // accumulation groups consumed so far
         float sc[TC];                                          // scale of the intermediate tile per token column (unit in its down phase)
 #pragma unroll
         for (int c = 0; c < TC; ++c) sc[c] = 0.f;
+        // wait for group g's accumulators, read the first TC columns of both halves of its buffer, hand the buffer back
+        int buf = 0;
+        uint32_t bpar = 0u;                                    // parity of the next phase of bar_tfull[buf]
+        auto take = [&](float* d0, float* d1) {
+            if (!wt.mbar(bar_tfull + 8 * buf, bpar, 29)) misc[3] = 1u;
+            tc_fence_after();
+            const uint32_t tcol = t_lane + (uint32_t)(buf * kBufCols);
+            tmem_ld<TC>(tcol, d0);
+            tmem_ld<TC>(tcol + N, d1);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+            if (++buf == NI) { buf = 0; bpar ^= 1u; }
+        };
         // Block scales of unit s for this CTA's tiles: lane l holds K block kb_lo + l (and + 32) of the gate and of the up
         // rows, and row block hb_lo + l (and + 32) of the W2 column block.  Fetched one unit ahead of their use.
         float nwg0 = 0.f, nwu0 = 0.f, nwg1 = 0.f, nwu1 = 0.f, nw2a = 0.f, nw2b = 0.f;
@@ -569,35 +565,25 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             nw2a = (lane < nh) ? __ldg(w2 + (size_t)lane * IB) : 0.f;
             nw2b = (lane + 32 < nh) ? __ldg(w2 + (size_t)(lane + 32) * IB) : 0.f;
         };
-        if (alive && !wt.dead && n > 0) {
+        if (alive && n > 0) {
             fetch_scales(0);
             float w2a = 0.f, w2b = 0.f, pw2a = 0.f, pw2b = 0.f;   // W2 scales of the unit in its gate/up phase, and of the one in its down phase
             for (int s = 0; s <= n; ++s) {
                 pw2a = w2a; pw2b = w2b;
-                // ---------------- gate/up k-steps of unit s: accumulate, then park the partial sums for the cluster
+                // ---------------- gate/up groups of unit s: accumulate, then park the partial sums for the cluster
                 if (s < n) {
-                    int e, ib;
-                    unit_of(s, e, ib);
-                    // block scales of this CTA's k-steps (fetched one unit ahead), handed out by shuffle
-                    float wg0 = nwg0, wu0 = nwu0, wg1 = nwg1, wu1 = nwu1;
+                    float wg0 = nwg0, wu0 = nwu0;
+                    const float wg1 = nwg1, wu1 = nwu1;
                     w2a = nw2a; w2b = nw2b;
                     fetch_scales(s + 1);
                     float accg[TC], accu[TC];
 #pragma unroll
                     for (int c = 0; c < TC; ++c) { accg[c] = 0.f; accu[c] = 0.f; }
-                    for (int k = 0; k < nk; ++k, ++g) {
-                        const int buf = g & (kTmemBufs - 1);
-                        if (!wt.mbar(bar_tfull + 8 * buf, (uint32_t)((g >> 3) & 1), 29)) misc[3] = 1u;
-                        tc_fence_after();
-                        if (first_acc) { if (etid == 0) MOE_STAMP(8); first_acc = false; }
+#pragma unroll 1
+                    for (int k = 0; k < nk; ++k) {
                         float dg[TC], du[TC];
-                        const uint32_t tcol = t_lane + (uint32_t)(buf * 2 * N);
-                        tmem_ld<TC>(tcol, dg);
-                        tmem_ld<TC>(tcol + N, du);
-                        tmem_ld_wait();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                        take(dg, du);
+                        if (first_acc) { if (etid == 0) MOE_STAMP(8); first_acc = false; }
                         const int kl = k & 31;
                         if (k == 32) { wg0 = wg1; wu0 = wu1; }
                         const float wsg = __shfl_sync(0xffffffffu, wg0, kl), wsu = __shfl_sync(0xffffffffu, wu0, kl);
@@ -625,17 +611,17 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * slot, (uint32_t)lane));
                     if (s == 0 && etid == 0) MOE_STAMP(9);
                 }
-                // ---------------- unit s-1: gather the cluster's partial sums, SiLU*up, requantise, then its down tiles
+                // ---------------- unit s-1: gather the cluster's partial sums, SiLU*up, requantise, then its down groups
                 if (s >= 1) {
                     const int i = s - 1, slot = i & 1;
                     int e, ib;
                     unit_of(i, e, ib);
-                    const float w2a = pw2a, w2b = pw2b;                     // W2 block scales of this CTA's row blocks (fetched with the unit's gate/up scales)
+                    const float w2a_ = pw2a, w2b_ = pw2b;
                     // token columns of this expert and where their down results go
-                    const unsigned long long mask = s_mask[2 * e];
+                    const unsigned mask = (unsigned)s_mask[2 * e];
                     int yoff_lane = 0;
-                    if (lane < TC && ((mask >> lane) & 1ull)) {
-                        const unsigned pr = s_pair[s_poff[e] + __popcll(mask & ((1ull << lane) - 1ull))];
+                    if (lane < TC && ((mask >> lane) & 1u)) {
+                        const unsigned pr = s_pair[s_poff[e] + __popc(mask & ((1u << lane) - 1u))];
                         yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
                     }
                     {
@@ -644,44 +630,47 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             if ((it & 255u) == 0 && wt.expired(31)) okw = false;
                         if (!okw) misc[3] = 1u;
                     }
-                    float a[TC];
-#pragma unroll
-                    for (int c = 0; c < TC; ++c) a[c] = 0.f;
+                                        float a[TC];
                     {
                         float sg[TC], su[TC];
 #pragma unroll
                         for (int c = 0; c < TC; ++c) { sg[c] = 0.f; su[c] = 0.f; }
                         const uint32_t mine = smem_u32(s_part + slot * 2 * TC * kBlock) + (uint32_t)row * 4u;
+#pragma unroll 1
                         for (int r = 0; r < C; ++r) {                      // rank order: every CTA of the cluster gets the same sums
                             const uint32_t src = map_to_rank(mine, (uint32_t)r);
+                            float vg[TC], vu[TC];
 #pragma unroll
-                            for (int c = 0; c < TC; ++c) {
-                                if ((mask >> c) & 1ull) {                  // only tokens routed to this expert matter (uniform)
-                                    sg[c] += ld_cluster_f32(src + (uint32_t)(c * kBlock * 4));
-                                    su[c] += ld_cluster_f32(src + (uint32_t)((TC + c) * kBlock * 4));
-                                }
+                            for (int c = 0; c < TC; ++c) {                 // (columns of tokens not routed to this expert are dropped below)
+                                vg[c] = ld_cluster_f32(src + (uint32_t)(c * kBlock * 4));
+                                vu[c] = ld_cluster_f32(src + (uint32_t)((TC + c) * kBlock * 4));
                             }
-                        }
-                        // SiLU(gate)*up, 128-wide amax (Section 3.3)
 #pragma unroll
-                        for (int c = 0; c < TC; ++c) {
-                            if ((mask >> c) & 1ull) {
-                                a[c] = __fdiv_rn(sg[c], 1.0f + expf(-sg[c])) * su[c];
-                                const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
-                                if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
-                            }
+                            for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
                         }
+                        // SiLU(gate)*up (Section 3.3).  The intermediate tile is outside the bit-exact set: fast exp and divide.
+#pragma unroll
+                        for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
                     }
-                    __syncwarp();
+                                        __syncwarp();
                     if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
-                    if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
-                    uint8_t* hq = s_hq + slot * N * kBlock;
+                    // 128-wide amax per token column: warp maximum (as an integer: |a| orders like its bits), then across the four warps
 #pragma unroll
                     for (int c = 0; c < TC; ++c) {
-                        if ((mask >> c) & 1ull) {
-                            const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
-                            sc[c] = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
-                            const float2 v = make_float2(__fdiv_rn(a[c], sc[c]), 0.f);
+                        const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
+                        if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
+                    }
+                    if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
+                                        uint8_t* hq = s_hq + slot * N * kBlock;
+#pragma unroll
+                    for (int c = 0; c < TC; ++c) {
+                        const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
+                        sc[c] = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
+                    }
+#pragma unroll
+                    for (int c = 0; c < TC; ++c) {
+                        if ((mask >> c) & 1u) {
+                            const float2 v = make_float2(a[c] * __frcp_rn(sc[c]), 0.f);
                             // K-major, 128-byte swizzled B tile: row = token column, 16-byte chunk (row >> 4) sits at chunk ^ (column & 7)
                             hq[c * kBlock + ((((row >> 4) ^ (c & 7)) << 4) | (row & 15))] = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
                         }
@@ -689,84 +678,83 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     fence_proxy_async();                                   // generic writes -> the tensor core's reads
                     epi_bar(kEpiThreads);
                     if (etid == 0) { mbar_arrive(bar_hq + 8 * slot); if (i == 0) MOE_STAMP(10); }
-                    // ---- down tiles of the unit: one accumulation group each, scaled and stored as the partial of (token, slot, ib)
-                    for (int h = 0; h < nh; ++h, ++g) {
-                        const int buf = g & (kTmemBufs - 1);
-                        if (!wt.mbar(bar_tfull + 8 * buf, (uint32_t)((g >> 3) & 1), 32)) misc[3] = 1u;
-                        tc_fence_after();
-                        float d[TC];
-                        tmem_ld<TC>(t_lane + (uint32_t)(buf * 2 * N), d);
-                        tmem_ld_wait();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-                        const float ws = __shfl_sync(0xffffffffu, (h < 32) ? w2a : w2b, h & 31);
-                        float* yrow = P.yp + (size_t)(hb_lo + h) * kBlock + row;
+                    // ---- down groups of the unit (two row blocks each), scaled and stored as the tagged partials of
+                    // (token, slot, ib): the final reduction polls these words themselves
+                    const unsigned long long tagw = (unsigned long long)tag << 32;
+#pragma unroll 1
+                    for (int h = 0; h < nh; h += 2) {
+                        float d0[TC], d1[TC];
+                        take(d0, d1);
+                                                const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? w2a_ : w2b_, h & 31);
+                        const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? w2a_ : w2b_, (h + 1) & 31);
+                        unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
+                        const bool live = (misc[3] == 0u) && !wt.dead;     // never publish a result that was not computed
+                        const bool two = (h + 1 < nh);
 #pragma unroll
                         for (int c = 0; c < TC; ++c) {
                             const int yo = __shfl_sync(0xffffffffu, yoff_lane, c);
-                            if ((mask >> c) & 1ull) __stcg(yrow + (size_t)yo, d[c] * (ws * sc[c]));
+                            if (((mask >> c) & 1u) && live) {
+                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(d0[c] * (ws0 * sc[c])));
+                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(d1[c] * (ws1 * sc[c])));
+                            }
                         }
                     }
                 }
             }
         }
-        // every partial of this CTA is stored: count it done (all CTAs count, with or without units)
-        epi_bar(kEpiThreads);
-        if (etid == 0) { if (alive && !wt.dead && misc[3] == 0u) red_release_add(P.ctrl + kDoneCnt + par, 1u); MOE_STAMP(11); }
-        // ---------------- final weighted reduction (Section 3.2: only this remains in the drain); deterministic.
-        // Task = (token, 128-row block), task = cta + i * G.  Warp q takes the partials p = q, q + 4, ... of the
-        // K * I/128 (slot, ib) partials, four rows per lane; the four warps' sums are combined in fixed order.
-        if (alive) {
-            const bool got = (etid == 0) ? wt.flag(P.ctrl + kDoneCnt + par, (unsigned)G, 33) : true;
-            if (!epi_all(got && !wt.dead && misc[3] == 0u, kEpiThreads)) wt.dead = true;
-            if (etid == 0) MOE_STAMP(12);
-            const int n_tasks = T * HB, NP = K * IB;
-            float4* s_sum = reinterpret_cast<float4*>(s_part);             // [4 warps][32 lanes] (the partial buffers are idle now)
-#pragma unroll 1
-            for (int task = cta; task < n_tasks && !wt.dead; task += G) {
-                const int t = div_small(task, HB), hb = task - t * HB;
-                const float* base = P.yp + (size_t)t * K * IB * H + (size_t)hb * kBlock + lane * 4;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
-                for (int p0 = q; p0 < NP; p0 += 4 * 8) {                   // eight 16-byte loads in flight per thread
-                    float4 v[8];
-                    float wv[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int p = p0 + 4 * j;
-                        const bool on = p < NP;
-                        v[j] = on ? __ldcg(reinterpret_cast<const float4*>(base + (size_t)p * H)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        wv[j] = on ? s_w[t * K + div_small(p, IB)] : 0.f;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        acc.x = fmaf(wv[j], v[j].x, acc.x); acc.y = fmaf(wv[j], v[j].y, acc.y);
-                        acc.z = fmaf(wv[j], v[j].z, acc.z); acc.w = fmaf(wv[j], v[j].w, acc.w);
-                    }
-                }
-                s_sum[q * 32 + lane] = acc;
-                epi_bar(kEpiThreads);
-                if (q == 0) {
-                    const float4 a0 = s_sum[lane], a1 = s_sum[32 + lane], a2 = s_sum[64 + lane], a3 = s_sum[96 + lane];
-                    const float r0 = (a0.x + a1.x) + (a2.x + a3.x), r1 = (a0.y + a1.y) + (a2.y + a3.y);
-                    const float r2 = (a0.z + a1.z) + (a2.z + a3.z), r3 = (a0.w + a1.w) + (a2.w + a3.w);
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
-                    uint2 o;
-                    o.x = *reinterpret_cast<uint32_t*>(&lo);
-                    o.y = *reinterpret_cast<uint32_t*>(&hi);
-                    *reinterpret_cast<uint2*>(P.out + (size_t)t * H + hb * kBlock + lane * 4) = o;
-                }
-                epi_bar(kEpiThreads);
-            }
-            if (etid == 0) MOE_STAMP(13);
-        }
+        if (etid == 0) MOE_STAMP(11);
     }
 
-    // ------------------------------------------------------------------ teardown
+    // ------------------------------------------------------------------ final weighted reduction (Section 3.2: only this
+    // remains in the drain); deterministic.  Task = (token, 32 rows), task = cta + i * G.  Warp w of warps 0..7 takes the
+    // partials p = w, w + 8, ... of the top_k * I/128 (slot, ib) partials of its task, lane = row; it polls the tagged
+    // words until they carry this launch's tag (their producers' stores need no flag, no fence and no counter), and the
+    // eight warps' sums are combined in fixed order.
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (alive && warp < kMainWarps) {
+        const int QB = H / 32, n_tasks = T * QB, NP = K * IB;
+        float* s_sum = s_part;                                             // [8 warps][32 rows] (the partial buffers are idle now)
+        bool ok = !wt.dead;
+#pragma unroll 1
+        for (int task = cta; task < n_tasks; task += G) {
+            const int t = div_small(task, QB), rb = task - t * QB;
+            const unsigned long long* base = P.ypl + (size_t)t * NP * H + (size_t)rb * 32 + lane;
+            float acc = 0.f;
+#pragma unroll 1
+            for (int p0 = warp; p0 < NP && ok; p0 += 8 * 8) {              // eight words in flight per thread
+                unsigned long long v[8];
+                unsigned pending = 0u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) if (p0 + 8 * j < NP) pending |= 1u << j;
+                for (uint32_t it = 1; pending; ++it) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(base + (size_t)(p0 + 8 * j) * H);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) if ((pending & (1u << j)) && (unsigned)(v[j] >> 32) == tag) pending &= ~(1u << j);
+                    if (pending && (it & 63u) == 0 && wt.expired(33)) { ok = false; break; }
+                }
+                if (!ok) break;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (p0 + 8 * j < NP) acc = fmaf(s_w[t * K + div_small(p0 + 8 * j, IB)], __uint_as_float((unsigned)v[j]), acc);
+            }
+            s_sum[warp * 32 + lane] = acc;
+            ok = named_bar_and(2, kMain, ok);
+            if (!ok) break;
+            if (warp == 0) {
+                const float r = ((s_sum[lane] + s_sum[32 + lane]) + (s_sum[64 + lane] + s_sum[96 + lane])) +
+                                ((s_sum[128 + lane] + s_sum[160 + lane]) + (s_sum[192 + lane] + s_sum[224 + lane]));
+                P.out[(size_t)t * H + rb * 32 + lane] = __float2bfloat16_rn(r);
+            }
+            named_bar_sync(2, kMain);
+        }
+        if (tid == 0) MOE_STAMP(13);
+    }
+
+    // ------------------------------------------------------------------ teardown
+    __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, kFusedTmemCols);
     // no CTA of the cluster leaves while a peer may still read its shared memory or arrive on its barriers
     cluster_arrive();
@@ -774,13 +762,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     if (tid == 0) {
         if (P.stamps) { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); P.stamps[(size_t)blockIdx.x * kStampsPerCta + 14] = smid; }
         MOE_STAMP(15);
-        __threadfence();
-        const unsigned old = atomicAdd(P.ctrl + kExitCnt, 1u);
-        if (old == (unsigned)G - 1u) {          // last CTA out: open the next epoch
-            P.ctrl[kExitCnt] = 0u;
-            __threadfence();
-            st_release(P.ctrl + kEpoch, tag);
-        }
+        // Open the next epoch.  CTA 0 alone does it: it got here only after every CTA of the grid had counted its share
+        // of the quantised input, that is after every CTA had read this launch's tag.  (Unconditionally: a launch that
+        // gave up must not leave its tag to the next one.)
+        if (cta == 0) st_release(P.ctrl + kEpoch, tag);
     }
 }
 

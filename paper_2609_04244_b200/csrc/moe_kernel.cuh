@@ -45,7 +45,7 @@ constexpr int kMaxTokens = 128;       // per launch when tokens are compacted pe
 constexpr int kMaxPasses = 8;         // kMaxTokens / 16
 constexpr int kMaxUnits = kMaxExperts + kMaxTokens * kMaxTopK / 16;   // virtual experts (expert, pass) of one launch
 constexpr int kMaxTmemBufs = 8;      // accumulator buffers in TMEM (one K block each): 8 for N=16, 4 for N=32/64
-constexpr int kStampsPerCta = 16;
+constexpr int kStampsPerCta = 32;
 constexpr int kMaxGrid = 255;         // CTAs the weighted range tables of the compacted variants can hold
 
 // control words at the head of the workspace
@@ -87,8 +87,10 @@ struct Params {
     unsigned* pd_flag;  // [grid]
     float* y;           // [T,K,H]
     unsigned long long* ll;         // [T,E] fused variants: router logits as {launch tag, fp32 bits} words
-    float* yp;          // [T,K,I/128,H] fused variants: down-projection partial of every (token, slot, intermediate block)
-    unsigned long long* stamps;     // [grid][16] globaltimer stamps of the phases of the last launch; NULL = none taken
+    unsigned long long* ypl;        // [T,K,I/128,H] fused variants: down-projection partial of every (token, slot, intermediate block), {launch tag, fp32 bits}
+    int fC, fnCl;                   // fused variants: CTAs per cluster, clusters in the grid
+    int fkb[9], fhb[9];             // fused variants: rank r of a cluster takes K blocks [fkb[r], fkb[r+1]) and W2 row blocks [fhb[r], fhb[r+1])
+    unsigned long long* stamps;     // [grid][32] globaltimer stamps of the phases of the last launch; NULL = none taken
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -233,6 +235,7 @@ __device__ __forceinline__ bool epi_all(bool ok, int nthreads) {
 }
 
 #define MOE_STAMP(i) do { if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
+
 
 // K-major, 128-byte swizzled operand tile (rows of 128 bytes, 8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
