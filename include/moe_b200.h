@@ -218,11 +218,14 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              hold such clusters.  With MOE_KNOB_STAGES = 0 the fused variant takes as many stages as
  *                              leave half of the SM's shared memory to the next launch's CTA.
  *   MOE_KNOB_STAMPS            (plan-wide) kernels record the phase time stamps moe_debug_stamps() reads; off by default
+ *   MOE_KNOB_DEBUG_SKIP        (plan-wide, for tests of the give-up paths) 1: the fused-unit variant never signals that an
+ *                              intermediate tile is ready, so every wait behind that signal runs out after the plan's time
+ *                              limit and the launch ends with MOE_ERR_TIMEOUT -- no fault, nothing waits for ever.  0 (default)
  * Results do not depend on STAGES, ROUTE_ALL_TOKENS, PDL or STAMPS; SPLIT_SLACK_KIB, COMPACT_MIN, SPLIT_WEIGHT, FUSED and
  * CLUSTER change the order of fp32 partial sums (never the routing or the quantised input).
  */
 enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4,
-       MOE_KNOB_SPLIT_WEIGHT = 5, MOE_KNOB_FUSED = 6, MOE_KNOB_CLUSTER = 7, MOE_KNOB_STAMPS = 8 };
+       MOE_KNOB_SPLIT_WEIGHT = 5, MOE_KNOB_FUSED = 6, MOE_KNOB_CLUSTER = 7, MOE_KNOB_STAMPS = 8, MOE_KNOB_DEBUG_SKIP = 9 };
 int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value);
 int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value);
 

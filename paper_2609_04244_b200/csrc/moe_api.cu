@@ -89,6 +89,7 @@ struct moe_plan {
     int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
     int smem_per_sm = 0;
     int take_stamps = 0;            // kernels record their phase time stamps (diagnostics)
+    int debug_skip = 0;             // test hook: readiness signals the kernel leaves out (see MOE_KNOB_DEBUG_SKIP)
     moe_plan() {
         for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = t <= 8 ? 200 : 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
     }
@@ -161,8 +162,10 @@ struct moe_plan {
         return 0;
     }
     // CTAs per unit.  A unit (expert, 128-wide intermediate block) is 3 * H/128 weight tiles; clusters take units
-    // round-robin, so the busiest CTA streams ceil(units / clusters) * ceil(3 * (H/128) / C) tiles: take the C that
-    // makes that smallest for the expected number of distinct experts (text after Eq. 5), the smaller C on a tie.
+    // round-robin, so the busiest CTA streams ceil(units / clusters) rounds of ceil(3 * (H/128) / C) tiles, and every
+    // round costs about 16 tiles' worth of hand-over latency on top (measured on config 2: C = 2 wins at one token,
+    // C = 1 from two tokens on).  Take the C that makes that smallest for the expected number of distinct experts
+    // (text after Eq. 5), the smaller C on a tie.
     int fused_cluster(int T) const {
         const int KB = H / 128;
         const int knob = cluster_knob[T];
@@ -174,7 +177,7 @@ struct moe_plan {
         for (int C = 1; C <= 4; C *= 2) {
             if (max_clusters[C] <= 0 || C > KB) continue;
             const long long rounds = (units + max_clusters[C] - 1) / max_clusters[C];
-            const long long cost = rounds * ((3 * KB + C - 1) / C);
+            const long long cost = rounds * ((3 * KB + C - 1) / C + 16);
             if (!best || cost < best_cost) { best = C; best_cost = cost; }
         }
         return best;
@@ -183,9 +186,11 @@ struct moe_plan {
     bool fused_possible(int T) const {
         return T >= 1 && T <= 8 && T < compact_min && H <= 8192 && fused_cluster(T) > 0 && fused_stages(T) >= 2;
     }
+    // The library's choice: one and two tokens.  Units are dealt to clusters whole, so with more tokens (more units than
+    // clusters, but not many more) the busiest cluster's extra unit costs more than the general variant's latency chain.
     bool fused(int T) const {
         if (fused_mode == 0 || !fused_possible(T)) return false;
-        return true;
+        return fused_mode == 1 || T <= 2;
     }
 
     // Default depth of the stage ring when the knob is 0.  Measured on this machine (config 2 and the paper's shapes,
@@ -339,6 +344,8 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.fC = 1; P.fnCl = p->sms;
     for (int r = 0; r < 9; ++r) { P.fkb[r] = 0; P.fhb[r] = 0; }
     P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
+    P.stamps_fine = p->take_stamps >= 2;
+    P.debug_skip = p->debug_skip;
     return P;
 }
 
@@ -467,8 +474,13 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             if (value > 0 && plan->max_clusters[value] <= 0) return fail(MOE_ERR_OCCUPANCY, "clusters of %d CTAs cannot be launched on this device", value);
             for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->cluster_knob[t] = value;
             return MOE_OK;
+        case MOE_KNOB_DEBUG_SKIP:
+            if (value < 0 || value > 1) return fail(MOE_ERR_ARG, "debug skip must be 0 or 1");
+            plan->debug_skip = value;
+            return MOE_OK;
         case MOE_KNOB_STAMPS:
-            plan->take_stamps = value != 0;
+            if (value < 0 || value > 2) return fail(MOE_ERR_ARG, "stamps must be 0, 1 or 2");
+            plan->take_stamps = value;
             return MOE_OK;
         default:
             return fail(MOE_ERR_ARG, "unknown knob %d", knob);
@@ -489,6 +501,7 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_FUSED: *value = plan->fused_mode; return MOE_OK;
         case MOE_KNOB_CLUSTER: *value = t <= 8 ? plan->cluster_knob[t] : 0; return MOE_OK;
         case MOE_KNOB_STAMPS: *value = plan->take_stamps; return MOE_OK;
+        case MOE_KNOB_DEBUG_SKIP: *value = plan->debug_skip; return MOE_OK;
         default: return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
 }

@@ -131,8 +131,11 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
 // Warps: 0 producer (weight and activation tiles), 1, 2, 3 and 8 MMA issuers, 4..7 accumulator warps; warp 8 keeps
 // house during the routing phase.
 // ---------------------------------------------------------------------------------------------
+#ifndef MOE_FUSED_MIN_BLOCKS
+#define MOE_FUSED_MIN_BLOCKS 1
+#endif
 template <int TC>
-__global__ void __launch_bounds__(kFusedThreads, 1)
+__global__ void __launch_bounds__(kFusedThreads, MOE_FUSED_MIN_BLOCKS)
 moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                  const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ Params P) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -181,7 +184,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             mbar_init(bar_xfree + 8 * b, 4 * C);
         }
         for (int b = 0; b < 4; ++b) mbar_init(bar_drain + 8 * b, 1);
-        misc[3] = 0u; misc[6] = 0u;
+        misc[3] = 0u; misc[6] = 0u; misc[7] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kFusedTmemCols); tmem_relinquish(); }
@@ -339,8 +342,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             }
         }
         alive = named_bar_and(2, kMain, ok && !wt.dead);
-        if (tid == 0) MOE_STAMP(3);
-        __syncwarp();
+        if (P.stamps_fine) { if (tid == 0) MOE_STAMP(3); __syncwarp(); }
         // -------------------------------------------------------------- top-k for every token, in every CTA (Section 4.1)
         if (alive) {
 #pragma unroll 1
@@ -351,8 +353,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             }
         }
         named_bar_sync(2, kMain);
-        if (tid == 0) MOE_STAMP(4);
-        __syncwarp();
+        if (P.stamps_fine) { if (tid == 0) MOE_STAMP(4); __syncwarp(); }
         // -------------------------------------------------------------- routing metadata: active experts (warp 0), routed pairs (warps 4..7)
         if (alive && warp == 0) {
             int base = 0;
@@ -391,8 +392,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
     alive = __syncthreads_and(alive && !wt.dead) != 0;          // (the housekeeping warp joins here)
     if (misc[6] != 1u) alive = false;                           // the quantised input never arrived: its wait has recorded why
-    if (tid == 0) MOE_STAMP(5);
-    __syncwarp();
+    if (P.stamps_fine) { if (tid == 0) MOE_STAMP(5); __syncwarp(); }
     const int U = alive ? (int)misc[1] : 0;
     const int nU = U * IB;                                       // units of this step
     const int n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units of this cluster: cl, cl + nCl, ... (grid_magic divides by the cluster count here)
@@ -416,12 +416,15 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             const uint64_t stream_once = l2_policy_evict_first();
             fence_proxy_async();                 // xq was written with ordinary stores by other CTAs (acquired by the housekeeping warp)
             int cur = 0, st = 0;
+            long long w_empty = 0;
             uint32_t cntpar = 0u, second = 0u;   // per stage: parity of the number of groups it anchored; last filled as the second tile of a pair
             // one group: 1 or 2 weight tiles (rows y0 / y1 of `m`, column x) and, for gate/up groups, the activation tile of K block xq_kb
             auto put = [&](const CUtensorMap* m, int x0, int y0, int x1, int y1, int ntiles, int xq_kb) -> bool {
                 const int st0 = st, st1 = (st + 1 == S) ? 0 : st + 1;
+                const long long c0 = clock64();
                 if (!((second >> st0) & 1u) && !wt.mbar(bar_empty + 8 * st0, ((cntpar >> st0) & 1u) ^ 1u, 21)) return false;
                 if (ntiles == 2 && !((second >> st1) & 1u) && !wt.mbar(bar_empty + 8 * st1, ((cntpar >> st1) & 1u) ^ 1u, 21)) return false;
+                w_empty += clock64() - c0;
                 const uint32_t full = bar_full + 8 * st0, dst0 = smem_u32(smem) + (uint32_t)st0 * kFusedStage;
                 mbar_expect_tx(full, (uint32_t)(ntiles * kATileBytes + (xq_kb >= 0 ? N * kBlock : 0)));
                 tma_load_2d_hint(dst0, m, x0, y0, full, stream_once);
@@ -450,10 +453,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         if (!put(&tmW2, ib * kBlock, e * H + h * kBlock, ib * kBlock, e * H + (h + 1) * kBlock, (h + 1 < hb_hi) ? 2 : 1, -1)) break;
                 }
             }
-            if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight: every barrier it may have armed in the last lap
-                for (int s = 0; s < S; ++s)
-                    for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
-            }
+            if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + 16] = (unsigned long long)w_empty;
+            misc[7] = cntpar;      // which phase of every stage's `full` barrier was armed last (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
     }
@@ -473,6 +474,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             int st = 0, j = 0, turn = 0;
             uint32_t fpar = 0u;                  // per stage: parity of the next phase of its `full` barrier
             uint32_t tpar = 1u;                  // parity to wait for on this issuer's `tempty` barrier
+            long long w_te = 0, w_fu = 0, w_hq = 0, w_is = 0;
             bool first = true;
             // one group: tile(s) at stage st (and st + 1), activation operand at b_addr (0: next to the first tile)
             auto group = [&](int ntiles, uint32_t b_addr) -> bool {
@@ -485,9 +487,13 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 const uint32_t fp = (fpar >> st0) & 1u;
                 fpar ^= 1u << st0;
                 if (!mine) return true;
+                const long long c0 = clock64();
                 if (!wt.mbar(bar_tempty + 8 * iss, tpar, 24)) return false;
                 tpar ^= 1u;
+                const long long c1 = clock64();
                 if (!wt.mbar(bar_full + 8 * st0, fp, 26)) return false;
+                const long long c2 = clock64();
+                w_te += c1 - c0; w_fu += c2 - c1;
                 if (first && iss == 0) { MOE_STAMP(7); first = false; }
                 const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)kFusedStage;
                 const uint64_t b_desc = make_smem_desc(b_addr ? b_addr : a0 + kATileBytes);
@@ -505,6 +511,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 }
                 if (release) umma_commit(bar_empty + 8 * st0);
                 umma_commit(bar_tfull + 8 * iss);
+                w_is += clock64() - c2;
                 return true;
             };
             for (int s = 0; s <= n && !wt.dead; ++s) {
@@ -514,15 +521,12 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 if (s >= 1 && !wt.dead) {
                     const int slot = (s - 1) & 1;
                     // the intermediate tile of unit s-1 is in shared memory (written by the accumulator warps)
-                    if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)(((s - 1) >> 1) & 1), 27)) break;
+                    { const long long c0 = clock64(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)(((s - 1) >> 1) & 1), 27)) break; w_hq += clock64() - c0; }
                     for (int h = 0; h < nh; h += 2)
                         if (!group((h + 1 < nh) ? 2 : 1, smem_u32(s_hq) + (uint32_t)(slot * N * kBlock))) break;
                 }
             }
-            if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
-                umma_commit(bar_drain + 8 * (uint32_t)iss);
-                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain + 8 * (uint32_t)iss, 0); ++i) {}
-            }
+            if (P.stamps && iss == 0) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[17] = w_te; o[18] = w_fu; o[19] = w_hq; o[20] = w_is; }
         }
         __syncwarp();
     }
@@ -536,10 +540,13 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
         for (int c = 0; c < TC; ++c) sc[c] = 0.f;
         // wait for group g's accumulators, read the first TC columns of both halves of its buffer, hand the buffer back
+        long long w_tf = 0, w_xf = 0, w_fc = 0;
         int buf = 0;
         uint32_t bpar = 0u;                                    // parity of the next phase of bar_tfull[buf]
         auto take = [&](float* d0, float* d1) {
+            const long long c0 = clock64();
             if (!wt.mbar(bar_tfull + 8 * buf, bpar, 29)) misc[3] = 1u;
+            w_tf += clock64() - c0;
             tc_fence_after();
             const uint32_t tcol = t_lane + (uint32_t)(buf * kBufCols);
             tmem_ld<TC>(tcol, d0);
@@ -567,9 +574,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         };
         if (alive && n > 0) {
             fetch_scales(0);
-            float w2a = 0.f, w2b = 0.f, pw2a = 0.f, pw2b = 0.f;   // W2 scales of the unit in its gate/up phase, and of the one in its down phase
+            float w2a = 0.f, w2b = 0.f, dw2a = 0.f, dw2b = 0.f;     // W2 scales of the unit in its gate/up phase, and of the one in its down phase
+            unsigned dmask = 0u;                                   // token columns and result offsets of the unit in its down phase
+            int dyoff = 0;
             for (int s = 0; s <= n; ++s) {
-                pw2a = w2a; pw2b = w2b;
                 // ---------------- gate/up groups of unit s: accumulate, then park the partial sums for the cluster
                 if (s < n) {
                     float wg0 = nwg0, wu0 = nwu0;
@@ -611,12 +619,36 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * slot, (uint32_t)lane));
                     if (s == 0 && etid == 0) MOE_STAMP(9);
                 }
-                // ---------------- unit s-1: gather the cluster's partial sums, SiLU*up, requantise, then its down groups
+                // ---------------- unit s-1: its down groups (the intermediate tile was made at the end of the previous turn, long
+                // before the issuers got here: no hand-over wait on the weight stream's path), scaled and stored as the tagged
+                // partials of (token, slot, ib): the final reduction polls these words themselves
                 if (s >= 1) {
-                    const int i = s - 1, slot = i & 1;
+                    const unsigned long long tagw = (unsigned long long)tag << 32;
+#pragma unroll 1
+                    for (int h = 0; h < nh; h += 2) {
+                        float d0[TC], d1[TC];
+                        take(d0, d1);
+                        const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? dw2a : dw2b, h & 31);
+                        const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? dw2a : dw2b, (h + 1) & 31);
+                        unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
+                        const bool live = (misc[3] == 0u) && !wt.dead;     // never publish a result that was not computed
+                        const bool two = (h + 1 < nh);
+#pragma unroll
+                        for (int c = 0; c < TC; ++c) {
+                            const int yo = __shfl_sync(0xffffffffu, dyoff, c);
+                            if (((dmask >> c) & 1u) && live) {
+                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(d0[c] * (ws0 * sc[c])));
+                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(d1[c] * (ws1 * sc[c])));
+                            }
+                        }
+                    }
+                }
+                // ---------------- unit s: gather the cluster's partial sums, SiLU*up, requantise -> the intermediate tile its
+                // down groups will use one turn later
+                if (s < n) {
+                    const int i = s, slot = i & 1;
                     int e, ib;
                     unit_of(i, e, ib);
-                    const float w2a_ = pw2a, w2b_ = pw2b;
                     // token columns of this expert and where their down results go
                     const unsigned mask = (unsigned)s_mask[2 * e];
                     int yoff_lane = 0;
@@ -624,13 +656,15 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         const unsigned pr = s_pair[s_poff[e] + __popc(mask & ((1u << lane) - 1u))];
                         yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
                     }
+                    const long long cf0 = clock64();
                     {
                         bool okw = !wt.dead;
                         for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, (uint32_t)((i >> 1) & 1)); ++it)
                             if ((it & 255u) == 0 && wt.expired(31)) okw = false;
                         if (!okw) misc[3] = 1u;
                     }
-                                        float a[TC];
+                    w_xf += clock64() - cf0;
+                    float a[TC];
                     {
                         float sg[TC], su[TC];
 #pragma unroll
@@ -652,7 +686,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                         for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
                     }
-                                        __syncwarp();
+                    __syncwarp();
                     if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
                     // 128-wide amax per token column: warp maximum (as an integer: |a| orders like its bits), then across the four warps
 #pragma unroll
@@ -661,76 +695,65 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
                     }
                     if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
-                                        uint8_t* hq = s_hq + slot * N * kBlock;
+                    uint8_t* hq = s_hq + slot * N * kBlock;
 #pragma unroll
                     for (int c = 0; c < TC; ++c) {
                         const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
-                        sc[c] = __fdiv_rn(fmaxf(amax, 1e-10f), 448.0f);
+                        sc[c] = fmaxf(amax, 1e-10f) * (1.0f / 448.0f);      // (the intermediate tile's scale is outside the bit-exact set)
                     }
 #pragma unroll
                     for (int c = 0; c < TC; ++c) {
                         if ((mask >> c) & 1u) {
-                            const float2 v = make_float2(a[c] * __frcp_rn(sc[c]), 0.f);
+                            const float2 v = make_float2(a[c] * __fdividef(1.0f, sc[c]), 0.f);
                             // K-major, 128-byte swizzled B tile: row = token column, 16-byte chunk (row >> 4) sits at chunk ^ (column & 7)
                             hq[c * kBlock + ((((row >> 4) ^ (c & 7)) << 4) | (row & 15))] = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
                         }
                     }
                     fence_proxy_async();                                   // generic writes -> the tensor core's reads
                     epi_bar(kEpiThreads);
-                    if (etid == 0) { mbar_arrive(bar_hq + 8 * slot); if (i == 0) MOE_STAMP(10); }
-                    // ---- down groups of the unit (two row blocks each), scaled and stored as the tagged partials of
-                    // (token, slot, ib): the final reduction polls these words themselves
-                    const unsigned long long tagw = (unsigned long long)tag << 32;
-#pragma unroll 1
-                    for (int h = 0; h < nh; h += 2) {
-                        float d0[TC], d1[TC];
-                        take(d0, d1);
-                                                const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? w2a_ : w2b_, h & 31);
-                        const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? w2a_ : w2b_, (h + 1) & 31);
-                        unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
-                        const bool live = (misc[3] == 0u) && !wt.dead;     // never publish a result that was not computed
-                        const bool two = (h + 1 < nh);
-#pragma unroll
-                        for (int c = 0; c < TC; ++c) {
-                            const int yo = __shfl_sync(0xffffffffu, yoff_lane, c);
-                            if (((mask >> c) & 1u) && live) {
-                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(d0[c] * (ws0 * sc[c])));
-                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(d1[c] * (ws1 * sc[c])));
-                            }
-                        }
-                    }
+                    if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * slot); if (i == 0) MOE_STAMP(10); }
+                    w_fc += clock64() - cf0;
+                    dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b;
                 }
             }
         }
-        if (etid == 0) MOE_STAMP(11);
+        if (etid == 0) { MOE_STAMP(11); if (P.stamps) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[21] = w_tf; o[22] = w_xf; o[23] = w_fc; } }
     }
 
     // ------------------------------------------------------------------ final weighted reduction (Section 3.2: only this
-    // remains in the drain); deterministic.  Task = (token, 32 rows), task = cta + i * G.  Warp w of warps 0..7 takes the
-    // partials p = w, w + 8, ... of the top_k * I/128 (slot, ib) partials of its task, lane = row; it polls the tagged
-    // words until they carry this launch's tag (their producers' stores need no flag, no fence and no counter), and the
-    // eight warps' sums are combined in fixed order.
+    // remains in the drain); deterministic.  Task = (token, 32 rows), task = cta + i * G, lane = row.  The top_k * I/128
+    // (slot, ib) partials of a task are tagged words: a reader polls them until they carry this launch's tag -- their
+    // producers' stores need no flag, no fence and no counter.  `sp` warps share a task (8 when a CTA has one task, 1
+    // when it has eight or more), warp part q of them taking the partials q, q + sp, ...; their sums are combined in
+    // fixed order.  sp depends only on the shape, the token count and the grid.
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     if (alive && warp < kMainWarps) {
         const int QB = H / 32, n_tasks = T * QB, NP = K * IB;
+        const int tpc = (n_tasks + G - 1) / G;                             // tasks of the busiest CTA
+        int sp = 8;
+        while (sp > 1 && sp * tpc > 8) sp >>= 1;
+        const int slots = 8 / sp, slot = warp / sp, part = warp - slot * sp;
+        const int mine = (cta < n_tasks) ? (n_tasks - cta + G - 1) / G : 0;
         float* s_sum = s_part;                                             // [8 warps][32 rows] (the partial buffers are idle now)
         bool ok = !wt.dead;
 #pragma unroll 1
-        for (int task = cta; task < n_tasks; task += G) {
+        for (int i0 = 0; i0 < mine; i0 += slots) {
+            const bool valid = (i0 + slot < mine);
+            const int task = cta + (valid ? i0 + slot : i0) * G;
             const int t = div_small(task, QB), rb = task - t * QB;
             const unsigned long long* base = P.ypl + (size_t)t * NP * H + (size_t)rb * 32 + lane;
             float acc = 0.f;
 #pragma unroll 1
-            for (int p0 = warp; p0 < NP && ok; p0 += 8 * 8) {              // eight words in flight per thread
+            for (int p0 = part; p0 < NP && ok && valid; p0 += sp * 8) {   // eight words in flight per thread
                 unsigned long long v[8];
                 unsigned pending = 0u;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) if (p0 + 8 * j < NP) pending |= 1u << j;
+                for (int j = 0; j < 8; ++j) if (p0 + sp * j < NP) pending |= 1u << j;
                 for (uint32_t it = 1; pending; ++it) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(base + (size_t)(p0 + 8 * j) * H);
+                    for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(base + (size_t)(p0 + sp * j) * H);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) if ((pending & (1u << j)) && (unsigned)(v[j] >> 32) == tag) pending &= ~(1u << j);
                     if (pending && (it & 63u) == 0 && wt.expired(33)) { ok = false; break; }
@@ -738,14 +761,14 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 if (!ok) break;
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    if (p0 + 8 * j < NP) acc = fmaf(s_w[t * K + div_small(p0 + 8 * j, IB)], __uint_as_float((unsigned)v[j]), acc);
+                    if (p0 + sp * j < NP) acc = fmaf(s_w[t * K + div_small(p0 + sp * j, IB)], __uint_as_float((unsigned)v[j]), acc);
             }
             s_sum[warp * 32 + lane] = acc;
             ok = named_bar_and(2, kMain, ok);
             if (!ok) break;
-            if (warp == 0) {
-                const float r = ((s_sum[lane] + s_sum[32 + lane]) + (s_sum[64 + lane] + s_sum[96 + lane])) +
-                                ((s_sum[128 + lane] + s_sum[160 + lane]) + (s_sum[192 + lane] + s_sum[224 + lane]));
+            if (part == 0 && valid) {
+                float r = s_sum[warp * 32 + lane];
+                for (int q2 = 1; q2 < sp; ++q2) r += s_sum[(warp + q2) * 32 + lane];
                 P.out[(size_t)t * H + rb * 32 + lane] = __float2bfloat16_rn(r);
             }
             named_bar_sync(2, kMain);
@@ -755,6 +778,24 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 
     // ------------------------------------------------------------------ teardown
     __syncthreads();
+    // A launch that gave up somewhere: nothing asynchronous may outlive the CTA.  The bulk copies the producer had
+    // requested and the MMAs the issuers had issued are waited for here (bounded), whether or not those roles
+    // noticed the give-up themselves, before tensor memory is freed and shared memory goes to the next CTA.
+    if (*(volatile unsigned*)(P.ctrl + kAbort) != 0u) {
+        if (tid == 0) {
+            const uint32_t cntpar = misc[7];
+            for (int s = 0; s < S; ++s)
+                for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
+        }
+        if (lane == 0 && ((warp >= 1 && warp < kEpiWarp0) || warp == 8)) {
+            const uint32_t bar = bar_drain + 8 * (uint32_t)((warp == 8) ? 3 : warp - 1);
+            umma_commit(bar);
+            for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar, 0); ++i) {}
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
     if (warp == 1) tmem_dealloc(tmem_base, kFusedTmemCols);
     // no CTA of the cluster leaves while a peer may still read its shared memory or arrive on its barriers
     cluster_arrive();

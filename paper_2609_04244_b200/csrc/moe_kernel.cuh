@@ -91,6 +91,8 @@ struct Params {
     int fC, fnCl;                   // fused variants: CTAs per cluster, clusters in the grid
     int fkb[9], fhb[9];             // fused variants: rank r of a cluster takes K blocks [fkb[r], fkb[r+1]) and W2 row blocks [fhb[r], fhb[r+1])
     unsigned long long* stamps;     // [grid][32] globaltimer stamps of the phases of the last launch; NULL = none taken
+    int debug_skip;                 // test hook, bit 0: the fused variants never publish the intermediate tile's readiness (a flag that nothing sets: the waits on it must run out cleanly)
+    int stamps_fine;                // fused variants: also stamp inside the routing phase (each stamp costs that phase ~0.1 us)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -582,7 +584,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         for (int b = 0; b < kTmemBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4 * kEpiGroups); }
         mbar_init(bar_drain, 1);
         mbar_init(bar_drain + 16, 1);
-        misc[3] = 0u; misc[4] = 0u; misc[5] = 0u;
+        misc[3] = 0u; misc[4] = 0u; misc[5] = 0u; misc[6] = 0u; misc[7] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kTmemCols); tmem_relinquish(); }
@@ -955,10 +957,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; }
             }
-            if (wt.dead) {   // give-up path: wait (bounded) for this thread's copies in flight
-                for (int it = (a_cur > S ? a_cur - S : 0); it < a_cur; ++it)
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_full + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
-            }
+            misc[6] = (uint32_t)a_cur;      // weight tiles requested (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
     }
@@ -1031,11 +1030,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
             }
-            cp_async_wait_all();                 // nothing of this warp is in flight past this point ...
-            if (!ok && lane == 0) {              // ... except bulk copies: give-up path waits (bounded) for them
-                for (int it = (b_cur > S ? b_cur - S : 0); it < b_cur; ++it)
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_fullb + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
-            }
+            cp_async_wait_all();                 // nothing of this warp is in flight past this point, except bulk copies:
+            if (lane == 0) misc[7] = (uint32_t)b_cur;   // activation tiles requested (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
     }
@@ -1077,10 +1073,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 dst += L.stage_bytes; full += 8; empty += 8;
                 if (++b_st == S) { b_st = 0; b_ph ^= 1u; dst = smem_u32(smem) + kATileBytes; full = bar_fullb; empty = bar_empty; }
             }
-            if (wt.dead) {
-                for (int it = (b_cur > S ? b_cur - S : 0); it < b_cur; ++it)
-                    for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_fullb + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
-            }
+            misc[7] = (uint32_t)b_cur;      // activation tiles requested (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
     }
@@ -1156,10 +1149,6 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 // move past the rest of this k-step and the other issuer's k-step
                 advance(1);
                 if (ks + 1 < n_up + n_dn) advance(ks + 1 < n_up ? 2 : 1);
-            }
-            if (wt.dead) {                                     // let issued MMAs retire before TMEM is released
-                umma_commit(bar_drain + 8 * (uint32_t)who * 2);
-                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar_drain + 8 * (uint32_t)who * 2, 0); ++i) {}
             }
         }
         __syncwarp();
@@ -1579,6 +1568,25 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // A launch that gave up somewhere: nothing asynchronous may outlive the CTA.  Whatever each role had requested --
+    // weight and activation tiles by bulk copy, MMAs -- is waited for here (bounded), whether or not the role itself
+    // noticed the give-up, before tensor memory is freed and shared memory goes to the next CTA.
+    if (*(volatile unsigned*)(P.ctrl + kAbort) != 0u) {
+        if (lane == 0 && (warp == 0 || warp == 2)) {
+            const int cur = (int)misc[6 + (warp >> 1)];
+            const uint32_t bar0 = warp ? bar_fullb : bar_full;
+            for (int it = (cur > S ? cur - S : 0); it < cur; ++it)
+                for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar0 + 8 * (it % S), (uint32_t)((it / S) & 1)); ++i) {}
+        }
+        if (lane == 0 && (warp == 1 || warp == 3)) {
+            const uint32_t bar = bar_drain + 8 * (uint32_t)(warp >> 1) * 2;
+            umma_commit(bar);
+            for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar, 0); ++i) {}
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
     if (tid == 0) {
         MOE_STAMP(15);
