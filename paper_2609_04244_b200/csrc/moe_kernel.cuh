@@ -722,7 +722,8 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // tokens (one each, up to the grid size), publish ids and weights, and everybody reads all of them after a second
         // arrival counter (two more L2 round trips).  The idle weight ring holds the keys and score values.
         constexpr bool kAlwaysAll = (TC <= 8);             // the token-column variants serve at most 8 tokens: no shared routing code in them
-        const bool route_all = kAlwaysAll || ((T <= P.route_all_tokens) && (T * E <= 8192));
+        // (keys and score values of all tokens go into the idle weight ring: they have to fit what the stage count leaves)
+        const bool route_all = kAlwaysAll || ((T <= P.route_all_tokens) && (T * E <= 8192) && (2 * T * E * 4 <= S * L.stage_bytes));
         const int tpc = (T + G - 1) / G;                   // tokens per selecting CTA when the grid shares them (1 up to G tokens)
         const int n_route_ctas = (T + tpc - 1) / tpc;
         const int rt0 = route_all ? 0 : min(T, cta * tpc), rnt = route_all ? T : min(T - rt0, tpc);

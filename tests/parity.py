@@ -17,6 +17,11 @@ from paper_2609_04244_b200 import workloads as wl
 REL_L2_TOL = 5e-3
 
 
+def max_ambiguous(T):
+    """Tokens of a launch that may fall inside the near-tie band of the routing comparison."""
+    return max(1, -(-T // 100))
+
+
 def _u16(t):
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
@@ -48,12 +53,15 @@ def check_against_oracle(shape, T, d, dbg, routed_scale=1.0, max_oracle_tokens=N
         assert all(abs(key[e] - kK) <= 2 * tau for e in diff), f"token {t}: swapped experts outside the near-tie band"
         assert len(set(g_ids[t])) == K
         ambiguous.append(t)
+    # near-ties are rare (about one token in a thousand with 256 experts): a launch with more than one token in a
+    # hundred of them -- or any, where the caller says the seed has none -- is a logit regression, not a tie
+    assert len(ambiguous) <= max_ambiguous(T), f"{len(ambiguous)} of {T} tokens inside the near-tie band"
     exact = [t for t in range(T) if t not in ambiguous]
     np.testing.assert_allclose(g_w[exact], rt["w"][exact], rtol=2e-5, atol=1e-7)
     # --- expert path: oracle needs only the experts actually used
     # the oracle runs on all tokens, or on a sample spread evenly over them (first and last included)
     tok = list(range(T)) if max_oracle_tokens is None or max_oracle_tokens >= T else \
-        sorted(set(int(x) for x in np.linspace(0, T - 1, max_oracle_tokens).round()))
+        structured_sample(g_ids, T, max_oracle_tokens)
     ids_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_ids, rt["ids"])[tok]
     w_use = np.where(np.isin(np.arange(T), ambiguous)[:, None], g_w, rt["w"])[tok]
     used = np.unique(ids_use)
@@ -73,6 +81,29 @@ def check_against_oracle(shape, T, d, dbg, routed_scale=1.0, max_oracle_tokens=N
     assert worst <= 2e-2 * rms + 1e-3, f"max |diff| {worst:.3e} vs rms {rms:.3e}"
     return {"rel_l2": float(rel), "max_abs": float(worst), "rms": float(rms), "ambiguous": len(ambiguous),
             "unique_experts": int(len(np.unique(g_ids)))}
+
+
+def structured_sample(ids, T, count):
+    """Tokens for the oracle when it cannot afford all of them: the first and the last token, and tokens of the most
+    crowded expert chosen by their rank among that expert's tokens -- ranks 0, 7, 8, 15, 16, 31, 32, ... -- so that the
+    sample sees every pass of 16 or 32 compacted columns, both 8-column blocks of a pass and both accumulator groups."""
+    ids = np.asarray(ids)
+    experts, counts = np.unique(ids, return_counts=True)
+    crowded = experts[np.argmax(counts)]
+    members = [t for t in range(T) if crowded in ids[t]]
+    ranks = sorted({r for base in range(0, len(members), 16) for r in (base, base + 7, base + 8, base + 15) if r < len(members)}
+                   | {len(members) - 1})
+    picked = [0, T - 1]
+    for r in ranks:
+        if len(set(picked)) >= count:
+            break
+        picked.append(members[r])
+    rest = [int(x) for x in np.linspace(0, T - 1, count).round()]
+    for t in rest:                                   # fill up evenly if the crowded expert had few tokens
+        if len(set(picked)) >= count:
+            break
+        picked.append(t)
+    return sorted(set(picked))
 
 
 def _only_order_within_band(a, b, key, tau):
