@@ -41,6 +41,19 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
+# (config, tokens, regime) cells measured after the headline in the default run
+CELLS = [("c1_tiny", 1, "natural"), ("c2_qwen3_30b_a3b", 2, "natural"), ("c2_qwen3_30b_a3b", 4, "natural"),
+         ("c2_qwen3_30b_a3b", 8, "natural"), ("c2_qwen3_30b_a3b", 8, "same"), ("c4_mixtral_8x7b", 1, "natural"),
+         ("c5_deepseek_v3", 1, "natural"), ("c5_deepseek_v3", 8, "natural")]
+
+
+def kernel_name(info, T):
+    """Name of the kernel instantiation a plan launches for T tokens."""
+    if info.get("fused"):
+        return f"moe_fused_kernel<{1 if T <= 1 else 2 if T <= 2 else 4 if T <= 4 else 8}>"
+    return f"moe_decode_kernel<N={info['n_hw']}>"
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -57,6 +70,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps directly instead of from CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cells", action="store_true", help="skip the extra (config, tokens) cells measured after the headline")
     return ap.parse_args()
 
 
@@ -244,106 +258,123 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     T, K, W = args.tokens, args.steps, max(args.warmup, 3)
-    # enough distinct layer copies that the bytes streamed between two uses of a copy exceed 2x L2 (126 MB)
-    per_step = wl.algorithmic_bytes(shape, T, min(shape.E, int(round(wl.expected_unique_experts(shape.E, shape.top_k, T)))))
-    free_b, _ = torch.cuda.mem_get_info()
-    layer_bytes = shape.E * shape.bytes_per_expert
-    L = args.layers or max(2, min(16, -(-2 * 126 * 2**20 // per_step) + 1))
-    L = max(1, min(L, int(0.6 * free_b // layer_bytes)))
-    layers = [wl.make_layer(shape, T, regime=args.regime, layer=rank * 64 + l, device=dev) for l in range(L)]
     schedule = None
     if args.schedule:
         import json as _json
         with open(args.schedule) as f:
             schedule = _json.load(f)
-    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T, schedule=schedule)
-    info = plan.info(T)
-    outs = [torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev) for _ in range(L)]
 
-    def step(i):
-        d = layers[i % L]
-        plan.forward(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], out=outs[i % L])
+    def measure(shape, T, regime, K, W, keep=False):
+        """Device-resident timing of K layer-steps of `shape` at T tokens: CUDA-graph replay over distinct layer copies."""
+        # enough distinct layer copies that the bytes streamed between two uses of a copy exceed 2x L2 (126 MB)
+        per_step = wl.algorithmic_bytes(shape, T, min(shape.E, int(round(wl.expected_unique_experts(shape.E, shape.top_k, T)))))
+        free_b, _ = torch.cuda.mem_get_info()
+        layer_bytes = shape.E * shape.bytes_per_expert
+        L = args.layers or max(2, min(16, -(-2 * 126 * 2**20 // per_step) + 1))
+        L = max(1, min(L, int(0.6 * free_b // layer_bytes)))
+        layers = [wl.make_layer(shape, T, regime=regime, layer=rank * 64 + l, device=dev) for l in range(L)]
+        plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T, schedule=schedule)
+        info = plan.info(T)
+        outs = [torch.empty((T, shape.H), dtype=torch.bfloat16, device=dev) for _ in range(L)]
 
-    # unique experts per layer copy (from the kernel's own routing) -> algorithmic bytes per step
-    uniq = []
-    tpl = plan.tokens_per_launch()
-    for l in range(L):
-        d = layers[l]
-        ids_all = []
-        for lo in range(0, T, tpl):              # the debug entry point takes one launch's worth of tokens
-            dbg = plan.forward_debug(d["hidden"][lo:lo + tpl].contiguous(), d["Wr"], d["bias"], d["W13q"], d["W13s"],
-                                     d["W2q"], d["W2s"])
-            plan.sync_status()
-            ids_all.append(dbg["ids"])
-        ids_last = torch.cat(ids_all)
-        uniq.append(int(torch.unique(ids_last).numel()))
-    bytes_per_step = float(np.mean([wl.algorithmic_bytes(shape, T, u) for u in uniq]))
-    launches_per_step = -(-T // tpl)
+        def step(i):
+            d = layers[i % L]
+            plan.forward(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], out=outs[i % L])
 
-    # The timed steps are replayed from CUDA graphs (Section 4.1 of the paper times graph replays): a graph holds
-    # up to 1000 consecutive steps, so the host's per-call cost (Python, ctypes, launch) is not what is measured.
+        # unique experts per layer copy (from the kernel's own routing) -> algorithmic bytes per step
+        uniq = []
+        tpl = plan.tokens_per_launch()
+        ids_last = None
+        for l in range(L):
+            d = layers[l]
+            ids_all = []
+            for lo in range(0, T, tpl):              # the debug entry point takes one launch's worth of tokens
+                dbg = plan.forward_debug(d["hidden"][lo:lo + tpl].contiguous(), d["Wr"], d["bias"], d["W13q"], d["W13s"],
+                                         d["W2q"], d["W2s"])
+                plan.sync_status()
+                ids_all.append(dbg["ids"])
+            ids_last = torch.cat(ids_all)
+            uniq.append(int(torch.unique(ids_last).numel()))
+        bytes_per_step = float(np.mean([wl.algorithmic_bytes(shape, T, u) for u in uniq]))
+        launches_per_step = -(-T // tpl)
+
+        # The timed steps are replayed from CUDA graphs (Section 4.1 of the paper times graph replays): a graph holds
+        # up to 1000 consecutive steps, so the host's per-call cost (Python, ctypes, launch) is not what is measured.
+        for i in range(W):
+            step(i)
+        torch.cuda.synchronize()
+
+        def capture(first, n):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(n):
+                    step(first + i)
+            return g
+
+        class _Direct:                                      # --no-graph: same interface, plain launches
+            def __init__(self, first, n):
+                self.first, self.n = first, n
+
+            def replay(self):
+                for i in range(self.n):
+                    step(self.first + i)
+
+        if args.no_graph:
+            capture = _Direct
+        CH = 1000
+        graphs, done = [], 0
+        full = capture(W, CH) if K >= CH else None          # replayed K // CH times; the layer rotation inside it is
+        while done + CH <= K:                               # what keeps L2 cold, not the seam between two replays
+            graphs.append(full)
+            done += CH
+        if K - done:
+            graphs.append(capture(W + done, K - done))
+        for g in {id(g): g for g in graphs}.values():       # one untimed replay of each graph (first-launch upload)
+            g.replay()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t_wall0 = time.perf_counter()
+        torch.cuda.nvtx.range_push("timed_region")      # lets a profiler restrict itself to the timed steps
+        ev0.record(stream)
+        for g in graphs:
+            g.replay()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        torch.cuda.nvtx.range_pop()
+        t_wall1 = time.perf_counter()
+        if world > 1:
+            dist.barrier()
+        ms = ev0.elapsed_time(ev1)
+        if t_wall1 - t_wall0 < 0.25:        # timed region too short for a clock sample: keep the same load running briefly
+            t_end = time.perf_counter() + 0.3
+            while time.perf_counter() < t_end:
+                graphs[0].replay()
+                torch.cuda.synchronize()
+            clocks = sampler.finish()
+            clocks["window"] = "timed region + 0.3 s of the same load"
+        else:
+            clocks = sampler.finish(t_wall0, t_wall1)
+        plan.sync_status()
+        res = {"ms": ms, "K": K, "L": L, "info": info, "uniq": uniq, "bytes_per_step": bytes_per_step,
+               "launches_per_step": launches_per_step, "clocks": clocks}
+        if keep:
+            res.update(plan=plan, layers=layers, ids_last=ids_last)
+        else:
+            plan.close()
+            del layers, outs, graphs, full
+            torch.cuda.empty_cache()
+        return res
+
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
-    for i in range(W):
-        step(i)
-    torch.cuda.synchronize()
-
-    def capture(first, n):
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=stream):
-            for i in range(n):
-                step(first + i)
-        return g
-
-    class _Direct:                                      # --no-graph: same interface, plain launches
-        def __init__(self, first, n):
-            self.first, self.n = first, n
-
-        def replay(self):
-            for i in range(self.n):
-                step(self.first + i)
-
-    if args.no_graph:
-        capture = _Direct
-    CH = 1000
-    graphs, done = [], 0
-    full = capture(W, CH) if K >= CH else None          # replayed K // CH times; the layer rotation inside it is
-    while done + CH <= K:                               # what keeps L2 cold, not the seam between two replays
-        graphs.append(full)
-        done += CH
-    if K - done:
-        graphs.append(capture(W + done, K - done))
-    for g in {id(g): g for g in graphs}.values():       # one untimed replay of each graph (first-launch upload)
-        g.replay()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    t_wall0 = time.perf_counter()
-    torch.cuda.nvtx.range_push("timed_region")      # lets a profiler restrict itself to the timed steps
-    ev0.record(stream)
-    for g in graphs:
-        g.replay()
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    torch.cuda.nvtx.range_pop()
-    t_wall1 = time.perf_counter()
-    if world > 1:
-        dist.barrier()
-    ms = ev0.elapsed_time(ev1)
-    if t_wall1 - t_wall0 < 0.25:        # timed region too short for a clock sample: keep the same load running briefly
-        t_end = time.perf_counter() + 0.3
-        while time.perf_counter() < t_end:
-            graphs[0].replay()
-            torch.cuda.synchronize()
-        clocks = sampler.finish()
-        clocks["window"] = "timed region + 0.3 s of the same load"
-    else:
-        clocks = sampler.finish(t_wall0, t_wall1)
-    plan.sync_status()
+    head = measure(shape, T, args.regime, K, W, keep=True)
+    plan, layers, ids_last, L = head["plan"], head["layers"], head["ids_last"], head["L"]
+    info, uniq, bytes_per_step, launches_per_step, clocks, ms = (head[k] for k in ("info", "uniq", "bytes_per_step", "launches_per_step", "clocks", "ms"))
 
     # end to end: the step's input comes from pinned host memory, the result goes back to the host
     e2e = None
@@ -375,6 +406,24 @@ def main():
         e2e = {"ms": e2e_ms, "steps": Ke}
         plan.sync_status()
 
+    # More cells of the (config, tokens) table, measured in this same run with the same protocol (graph replay, layer
+    # rotation, clocks sampled per cell): the headline stays the line's `value`.
+    cells = None
+    if world == 1 and not args.no_cells and args.config == "c2_qwen3_30b_a3b" and T == 1 and args.regime == "natural" and not args.experts:
+        peak_c, _ = peak_hbm()
+        cells = []
+        Kc = max(200, min(K, 1000))
+        for name, Tc, regime in CELLS:
+            shp = wl.SHAPES[name]
+            r = measure(shp, Tc, regime, Kc, W)
+            us = r["ms"] * 1e3 / Kc
+            gbs = r["bytes_per_step"] / (us * 1e-6) / 1e9
+            cells.append({"workload": f"{name} T={Tc} regime={regime}", "us": us, "steps": Kc,
+                          "algorithmic_bytes_per_step": r["bytes_per_step"], "achieved_gbs": gbs, "frac": gbs / peak_c,
+                          "unique_experts_mean": float(np.mean(r["uniq"])), "layer_copies": r["L"],
+                          "variant": kernel_name(r["info"], Tc), "cluster": r["info"]["cluster"], "stages": r["info"]["stages"],
+                          "clocks": {k: r["clocks"].get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")}})
+
     ms, e2e_ms_max = max_over_ranks([ms, e2e["ms"] if e2e else 0.0], dev)
     if e2e:
         e2e["ms"] = e2e_ms_max
@@ -395,10 +444,11 @@ def main():
                        f"({L * bytes_per_step / 2**20:.0f} MiB streamed between reuses, L2 is 126 MiB)",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "grid": info["grid"], "stages": info["stages"], "n_hw": info["n_hw"],
+                       "variant": kernel_name(info, T), "cluster": info["cluster"],
                        "launch": "direct launches" if args.no_graph else "CUDA graph replay, one kernel node per step"},
             "achieved_gbs": achieved, "algorithmic_bytes_per_step": bytes_per_step,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}", "kernel": "moe_decode_kernel", "kernel_us": kernel_us,
+                         "peak_kind": f"of {peak_kind}", "kernel": kernel_name(info, T), "kernel_us": kernel_us,
                          "traffic": NCU_TRAFFIC_BYTES.get((shape.name, T))},
             "gpu_launches": K * launches_per_step,
             "clocks": clocks,
@@ -413,6 +463,8 @@ def main():
             us_cpu, reps, thr = time_oracle(shape, host)
             line["cpu_baseline"] = {"value": us_cpu, "unit": "us", "cores": thr, "kind": "oracle",
                                     "sample": f"{reps} full layer-steps of the same workload (T={T}), mean"}
+        if cells is not None:
+            line["cells"] = cells
         print(json.dumps(line), flush=True)
     plan.close()
     if world > 1:
