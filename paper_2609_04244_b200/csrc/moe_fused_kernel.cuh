@@ -39,6 +39,7 @@ namespace moe {
 constexpr int kFusedN = 16;                                   // MMA N of the fused variants (tokens 0..7 are columns 0..7)
 constexpr int kFusedStage = kATileBytes + kFusedN * kBlock;    // weight tile + activation tile
 constexpr int kFusedTmemBufs = 4;                              // accumulator buffers of 2 x 16 columns, one per MMA issuer
+constexpr int kFusedIssuers = 3;                               // warps 1..3
 constexpr int kFusedTmemCols = 128;
 constexpr int kFusedThreads = 288;                             // 9 warps
 constexpr int kFusedMaxRows = 4;                               // router rows per CTA: ceil(kMaxExperts / 128)
@@ -128,8 +129,8 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
 
 // ---------------------------------------------------------------------------------------------
 // the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8 >= T).
-// Warps: 0 producer (weight and activation tiles), 1, 2, 3 and 8 MMA issuers, 4..7 accumulator warps; warp 8 keeps
-// house during the routing phase.
+// Warps: 0 producer (weight and activation tiles), 1..3 MMA issuers, 4..7 accumulator warps; warp 8 keeps house
+// during the routing phase (everything that costs L2 round trips but is not needed before the first activation tile).
 // ---------------------------------------------------------------------------------------------
 #ifndef MOE_FUSED_MIN_BLOCKS
 #define MOE_FUSED_MIN_BLOCKS 1
@@ -158,13 +159,12 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kBufs);
     const uint32_t bar_x = smem_u32(bars + 2 * kMaxStages + 2 * kBufs);
-    const uint32_t bar_hq = bar_x, bar_xfull = bar_x + 16, bar_xfree = bar_x + 32, bar_drain = bar_x + 48;   // 2 + 2 + 2 + 4
+    const uint32_t bar_hq = bar_x, bar_xfull = bar_x + 16, bar_xfree = bar_x + 32, bar_drain = bar_x + 48, bar_hk = bar_x + 80;   // 2 + 2 + 2 + 4 + 1
     uint32_t* misc = (uint32_t*)(smem + L.misc_off);   // [0] tmem base, [1] U, [3] accumulator give-up, [6] quantised input published (1) or given up (2)
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
     int* s_act = (int*)(smem + L.act_off);
-    int* s_uidx = (int*)(smem + L.uidx_off);
     float* s_xs = (float*)(smem + L.xs_off);
     float* s_red = (float*)(smem + L.red_off);
     int* s_poff = (int*)(smem + L.poff_off);
@@ -184,6 +184,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             mbar_init(bar_xfree + 8 * b, 4 * C);
         }
         for (int b = 0; b < 4; ++b) mbar_init(bar_drain + 8 * b, 1);
+        mbar_init(bar_hk, 1);
         misc[3] = 0u; misc[6] = 0u; misc[7] = 0u;
         fence_barrier_init();
     }
@@ -297,8 +298,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll 1
             for (int i = lane; i < T * KBu; i += 32) { const int tt = div_small(i, KBu); s_xs[(i - tt * KBu) * TS + tt] = __ldcg(P.xs + i); }
         }
+        fence_proxy_async();                 // what the counter's acquire made visible -> the producer's bulk-tensor reads of xq
         __syncwarp();
-        if (lane == 0) misc[6] = okq ? 1u : 2u;
+        if (lane == 0 && okq) mbar_arrive(bar_hk);      // the quantised input and its scales are there (never, if the wait gave up)
     }
     const uint32_t tmem_base = misc[0];
 
@@ -352,22 +354,26 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 else route_select<16>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
             }
         }
-        named_bar_sync(2, kMain);
+        named_bar_sync(2, kMain);            // the selected experts and token masks of every token are in shared memory
         if (P.stamps_fine) { if (tid == 0) MOE_STAMP(4); __syncwarp(); }
-        // -------------------------------------------------------------- routing metadata: active experts (warp 0), routed pairs (warps 4..7)
-        if (alive && warp == 0) {
-            int base = 0;
+    } else {
+        alive = false;                       // (the housekeeping warp takes no further part)
+    }
+    // Routing metadata without another CTA-wide barrier: every warp that needs the list of active experts (ascending)
+    // builds it itself -- a ballot per 32 experts; all of them write the same values -- and the accumulator warps build
+    // the table of routed (token, slot) pairs among themselves.
+    int U = 0;
+    if (alive) {
 #pragma unroll 1
-            for (int e0 = 0; e0 < E; e0 += 32) {
-                const int e = e0 + lane;
-                const bool on = (e < E) && (s_mask[2 * e] != 0ull);
-                const unsigned b = __ballot_sync(0xffffffffu, on);
-                if (on) { const int u = base + __popc(b & ((1u << lane) - 1u)); s_act[u] = e; s_uidx[e] = u; }
-                base += __popc(b);
-            }
-            if (lane == 0) { misc[1] = (uint32_t)base; s_act[base] = 0; }
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const bool on = (e < E) && (s_mask[2 * e] != 0ull);
+            const unsigned bsel = __ballot_sync(0xffffffffu, on);
+            if (on) s_act[U + __popc(bsel & ((1u << lane) - 1u))] = e;
+            U += __popc(bsel);
         }
-        if (alive && warp >= kEpiWarp0) {
+        __syncwarp();
+        if (warp >= kEpiWarp0) {
             // (token, slot) pairs grouped by expert, tokens ascending: entry r of expert e = its r-th token and the slot e holds for it
             const int etid = tid - kEpiWarp0 * 32;
             if (warp == kEpiWarp0) {
@@ -388,12 +394,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 const int t = div_small(pi, K), ex = s_ids[pi];
                 s_pair[s_poff[ex] + __popcll(s_mask[2 * ex] & ((1ull << t) - 1ull))] = (unsigned short)(t | ((pi - t * K) << 8));
             }
+            epi_bar(kEpiThreads);
         }
     }
-    alive = __syncthreads_and(alive && !wt.dead) != 0;          // (the housekeeping warp joins here)
-    if (misc[6] != 1u) alive = false;                           // the quantised input never arrived: its wait has recorded why
     if (P.stamps_fine) { if (tid == 0) MOE_STAMP(5); __syncwarp(); }
-    const int U = alive ? (int)misc[1] : 0;
     const int nU = U * IB;                                       // units of this step
     const int n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units of this cluster: cl, cl + nCl, ... (grid_magic divides by the cluster count here)
     // this CTA's share of every unit: K blocks [kb_lo, kb_hi) of the gate/up rows, row blocks [hb_lo, hb_hi) of W2
@@ -408,13 +412,13 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // single last W2 tile.  One mbarrier per group in each direction: the group's tiles land on the `full` barrier of
     // its first stage and are released through that stage's `empty` barrier, so a stage that was the second of a pair
     // needs no wait of its own (the ring is refilled in order: its pair-mate's release came first).
-    const int NI = (S >> 1) < kBufs ? (S >> 1) : kBufs;           // MMA issuers = accumulator buffers in use
+    const int NI = (S >> 1) < kFusedIssuers ? (S >> 1) : kFusedIssuers;   // MMA issuers = accumulator buffers in use
     const int Ntot = n * (2 * nk + nh);                          // weight tiles of this CTA
     // ------------------------------------------------------------------ role: producer (weight tiles and activation tiles)
     if (warp == 0) {
         if (lane == 0 && alive && n > 0) {
             const uint64_t stream_once = l2_policy_evict_first();
-            fence_proxy_async();                 // xq was written with ordinary stores by other CTAs (acquired by the housekeeping warp)
+            wt.mbar(bar_hk, 0u, 22);             // the quantised input of every CTA is published and fenced for bulk copies (housekeeping warp); long done by now
             int cur = 0, st = 0;
             long long w_empty = 0;
             uint32_t cntpar = 0u, second = 0u;   // per stage: parity of the number of groups it anchored; last filled as the second tile of a pair
@@ -466,8 +470,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // no `empty` for stages that are never refilled.  With NI issuers and NI buffers nobody runs more than NI groups
     // ahead of the slowest (a buffer is handed back only after every earlier group was read), and NI <= S/2 groups is
     // less than a lap of the ring: a parity wait on a stage can never be a phase off.
-    else if (warp < kEpiWarp0 || warp == 8) {
-        const int iss = (warp == 8) ? 3 : warp - 1;
+    else if (warp < kEpiWarp0) {
+        const int iss = warp - 1;
         if (lane == 0 && alive && n > 0 && iss < NI) {
             constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBlock >> 4) << 24);
             const uint32_t ring = smem_u32(smem);
@@ -574,6 +578,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         };
         if (alive && n > 0) {
             fetch_scales(0);
+            if (!wt.mbar(bar_hk, 0u, 28)) misc[3] = 1u;          // the input scales are in shared memory (housekeeping warp)
             float w2a = 0.f, w2b = 0.f, dw2a = 0.f, dw2b = 0.f;     // W2 scales of the unit in its gate/up phase, and of the one in its down phase
             unsigned dmask = 0u;                                   // token columns and result offsets of the unit in its down phase
             int dyoff = 0;
@@ -721,7 +726,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
 
     // ------------------------------------------------------------------ final weighted reduction (Section 3.2: only this
-    // remains in the drain); deterministic.  Task = (token, 32 rows), task = cta + i * G, lane = row.  The top_k * I/128
+    // remains in the drain); deterministic.  Task = (token, 32 rows), task = (G - 1 - cta) + i * G, lane = row.  The top_k * I/128
     // (slot, ib) partials of a task are tagged words: a reader polls them until they carry this launch's tag -- their
     // producers' stores need no flag, no fence and no counter.  `sp` warps share a task (8 when a CTA has one task, 1
     // when it has eight or more), warp part q of them taking the partials q, q + sp, ...; their sums are combined in
@@ -735,13 +740,17 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         int sp = 8;
         while (sp > 1 && sp * tpc > 8) sp >>= 1;
         const int slots = 8 / sp, slot = warp / sp, part = warp - slot * sp;
-        const int mine = (cta < n_tasks) ? (n_tasks - cta + G - 1) / G : 0;
+        // tasks go to the CTAs from the LAST one down: the first CTAs hold the router rows and the units, and with them
+        // the next launch's critical path -- they should be the first to leave (the next launch's CTAs are placed in
+        // index order as SMs free up)
+        const int rc = G - 1 - cta;
+        const int mine = (rc < n_tasks) ? (n_tasks - rc + G - 1) / G : 0;
         float* s_sum = s_part;                                             // [8 warps][32 rows] (the partial buffers are idle now)
         bool ok = !wt.dead;
 #pragma unroll 1
         for (int i0 = 0; i0 < mine; i0 += slots) {
             const bool valid = (i0 + slot < mine);
-            const int task = cta + (valid ? i0 + slot : i0) * G;
+            const int task = rc + (valid ? i0 + slot : i0) * G;
             const int t = div_small(task, QB), rb = task - t * QB;
             const unsigned long long* base = P.ypl + (size_t)t * NP * H + (size_t)rb * 32 + lane;
             float acc = 0.f;
@@ -787,8 +796,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             for (int s = 0; s < S; ++s)
                 for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
         }
-        if (lane == 0 && ((warp >= 1 && warp < kEpiWarp0) || warp == 8)) {
-            const uint32_t bar = bar_drain + 8 * (uint32_t)((warp == 8) ? 3 : warp - 1);
+        if (lane == 0 && warp >= 1 && warp < kEpiWarp0) {
+            const uint32_t bar = bar_drain + 8 * (uint32_t)(warp - 1);
             umma_commit(bar);
             for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar, 0); ++i) {}
         }

@@ -463,30 +463,13 @@ __device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, in
     else route_scores_t<2, 8>(P, t0, nt, ksplit, tid, nthreads, s_key, s_val, write_global);
 }
 
-template <int NPER>
-__device__ __forceinline__ void route_select(const Params& P, int t, int lane, const uint32_t* s_key, const float* s_val,
+// Second half of the routing of one token (one warp; lane j < K holds the expert of slot j in `my_id`): the routing
+// weights -- softmax over all experts or the plain sigmoid score, optionally renormalised over the selected experts,
+// times the routed scaling factor (Section 4.1) -- and the token's entries in the id / weight / token-mask tables.
+__device__ __forceinline__ void route_finish(const Params& P, int t, int lane, int my_id, const float* s_val,
                                              int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global, bool build_mask) {
     const int E = P.E, K = P.K;
     const bool softmax = (P.scoring == 0);
-    uint32_t key[NPER];
-#pragma unroll
-    for (int i = 0; i < NPER; ++i) key[i] = (i * 32 + lane < E) ? s_key[i * 32 + lane] : 0u;    // 0 is below every real key
-    int my_id = 0;
-#pragma unroll 1
-    for (int j = 0; j < K; ++j) {                              // (a serial chain: unrolling buys nothing, and code fetched once per launch is dear)
-        uint32_t m = key[0];
-#pragma unroll
-        for (int i = 1; i < NPER; ++i) m = max(m, key[i]);
-        const uint32_t wm = __reduce_max_sync(0xffffffffu, m);
-        int cand = 0x7fffffff;
-#pragma unroll
-        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 : cand;
-        const int we = __reduce_min_sync(0xffffffffu, cand == 0x7fffffff ? cand : cand + lane);
-        const int mine = we - lane;                            // i * 32 if this lane holds the winner
-#pragma unroll
-        for (int i = 0; i < NPER; ++i) key[i] = (mine == i * 32) ? 0u : key[i];
-        if (lane == j) my_id = we;
-    }
     float v = (lane < K) ? s_val[my_id] : 0.f;
     float total = 1.0f;
     if (softmax) {
@@ -509,6 +492,32 @@ __device__ __forceinline__ void route_select(const Params& P, int t, int lane, c
         if (build_mask) mask_add(s_mask, my_id, t);
         if (write_global) { P.ids[t * K + lane] = my_id; P.wts[t * K + lane] = w; }
     }
+}
+
+template <int NPER>
+__device__ __forceinline__ void route_select(const Params& P, int t, int lane, const uint32_t* s_key, const float* s_val,
+                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global, bool build_mask) {
+    const int E = P.E, K = P.K;
+    uint32_t key[NPER];
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) key[i] = (i * 32 + lane < E) ? s_key[i * 32 + lane] : 0u;    // 0 is below every real key
+    int my_id = 0;
+#pragma unroll 1
+    for (int j = 0; j < K; ++j) {                              // (a serial chain: unrolling buys nothing, and code fetched once per launch is dear)
+        uint32_t m = key[0];
+#pragma unroll
+        for (int i = 1; i < NPER; ++i) m = max(m, key[i]);
+        const uint32_t wm = __reduce_max_sync(0xffffffffu, m);
+        int cand = 0x7fffffff;
+#pragma unroll
+        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 : cand;
+        const int we = __reduce_min_sync(0xffffffffu, cand == 0x7fffffff ? cand : cand + lane);
+        const int mine = we - lane;                            // i * 32 if this lane holds the winner
+#pragma unroll
+        for (int i = 0; i < NPER; ++i) key[i] = (mine == i * 32) ? 0u : key[i];
+        if (lane == j) my_id = we;
+    }
+    route_finish(P, t, lane, my_id, s_val, s_ids, s_w, s_mask, write_global, build_mask);
 }
 
 // quantise 4 floats with scale s into 4 E4M3 bytes (memory order x0..x3)
