@@ -107,8 +107,9 @@ int moe_forward(moe_plan_t plan, int T,
  * moe_forward_host: moe_forward with the step's activations in HOST memory (Section 3: same operator).
  *   hidden_host [T,H] bf16 and out_host [T,H] bf16 are host pointers (pinned memory makes the copies asynchronous);
  *   every other tensor is a device pointer as in moe_forward.  Enqueues, on `stream`: a host-to-device copy of
- *   `hidden_host` into a staging area of the workspace, the kernel, and a device-to-host copy of the result.  The
- *   host buffers must stay valid, and `out_host` must not be read, until the stream has been synchronised.
+ *   `hidden_host` into a staging area of the workspace, the kernel, and a device-to-host copy of the result; with
+ *   pinned buffers of at most 64 KiB the kernel writes the result into `out_host` itself (see MOE_KNOB_HOST_DIRECT).
+ *   The host buffers must stay valid, and `out_host` must not be read, until the stream has been synchronised.
  */
 int moe_forward_host(moe_plan_t plan, int T,
                      const void* hidden_host, const void* Wr_bf16, const float* sel_bias,
@@ -217,6 +218,13 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              tiles at the expected number of distinct experts.  MOE_ERR_OCCUPANCY if the device cannot
  *                              hold such clusters.  With MOE_KNOB_STAGES = 0 the fused variant takes as many stages as
  *                              leave half of the SM's shared memory to the next launch's CTA.
+ *   MOE_KNOB_SPLIT_UNITS       (plan-wide) fused-unit variant with more units than clusters: 1 (default) = the list of all
+ *                              accumulation groups is cut into equal ranges, one per cluster, so a unit's gate/up groups may
+ *                              be shared by two clusters (the first exports its partial sums to the second); 0 = units are
+ *                              dealt to clusters whole, round-robin
+ *   MOE_KNOB_HOST_DIRECT       (plan-wide) moe_forward_host with PINNED host buffers of at most 64 KiB: bit 0 (default on) = the
+ *                              kernel writes the result straight into out_host, bit 1 = it reads hidden_host in place; the
+ *                              transfers that are not taken this way go through a staging area and the copy engine
  *   MOE_KNOB_STAMPS            (plan-wide) kernels record the phase time stamps moe_debug_stamps() reads; off by default
  *   MOE_KNOB_DEBUG_SKIP        (plan-wide, for tests of the give-up paths) 1: the fused-unit variant never signals that an
  *                              intermediate tile is ready, so every wait behind that signal runs out after the plan's time
@@ -225,7 +233,7 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  * CLUSTER change the order of fp32 partial sums (never the routing or the quantised input).
  */
 enum { MOE_KNOB_STAGES = 0, MOE_KNOB_SPLIT_SLACK_KIB = 1, MOE_KNOB_ROUTE_ALL_TOKENS = 2, MOE_KNOB_COMPACT_MIN = 3, MOE_KNOB_PDL = 4,
-       MOE_KNOB_SPLIT_WEIGHT = 5, MOE_KNOB_FUSED = 6, MOE_KNOB_CLUSTER = 7, MOE_KNOB_STAMPS = 8, MOE_KNOB_DEBUG_SKIP = 9 };
+       MOE_KNOB_SPLIT_WEIGHT = 5, MOE_KNOB_FUSED = 6, MOE_KNOB_CLUSTER = 7, MOE_KNOB_STAMPS = 8, MOE_KNOB_DEBUG_SKIP = 9, MOE_KNOB_SPLIT_UNITS = 10, MOE_KNOB_HOST_DIRECT = 11 };
 int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value);
 int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value);
 

@@ -167,7 +167,7 @@ def moe_debug_stamps(plan, workspace, grid: int, stream=None):
 
 
 KNOBS = {"stages": 0, "split_slack_kib": 1, "route_all_tokens": 2, "compact_min": 3, "pdl": 4, "split_weight": 5,
-         "fused": 6, "cluster": 7, "stamps": 8, "debug_skip": 9}
+         "fused": 6, "cluster": 7, "stamps": 8, "debug_skip": 9, "split_units": 10, "host_direct": 11}
 
 
 def moe_plan_set_knob(plan, T: int, knob, value: int) -> None:

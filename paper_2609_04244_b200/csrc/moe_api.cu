@@ -58,7 +58,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
     size_t ctrl, e_cnt, dn_flag, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
-    size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, ll, yp, total;
+    size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, ll, yp, xsl, total;
 };
 
 struct MapKey {
@@ -88,6 +88,8 @@ struct moe_plan {
     int cluster_knob[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // CTAs per unit for T = 1..8; 0 = the library's choice
     int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
     int smem_per_sm = 0;
+    int split_units = 1;            // fused variants: equal ranges of the group list per cluster (units may be split between two clusters)
+    int host_direct = 1;            // moe_forward_host: bit 0 = write a small result straight into pinned host memory, bit 1 = read a small input in place
     int take_stamps = 0;            // kernels record their phase time stamps (diagnostics)
     int debug_skip = 0;             // test hook: readiness signals the kernel leaves out (see MOE_KNOB_DEBUG_SKIP)
     moe_plan() {
@@ -146,6 +148,7 @@ struct moe_plan {
         // fused variants: tagged router logits, and one down-projection partial per (token, slot, intermediate block)
         L.ll = o;       o += with_fused ? align_up((size_t)Tc * E * 8, 256) : 0;
         L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 8, 256) : 0;
+        L.xsl = o;      o += with_fused ? align_up((size_t)G * 2 * 8 * 128 * 8, 256) : 0;     // partial sums exported between clusters
         L.total = o;
         return L;
     }
@@ -161,39 +164,39 @@ struct moe_plan {
             if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) return s;
         return 0;
     }
-    // CTAs per unit.  A unit (expert, 128-wide intermediate block) is 3 * H/128 weight tiles; clusters take units
-    // round-robin, so the busiest CTA streams ceil(units / clusters) rounds of ceil(3 * (H/128) / C) tiles, and every
-    // round costs about 16 tiles' worth of hand-over latency on top (measured on config 2: C = 2 wins at one token,
-    // C = 1 from two tokens on).  Take the C that makes that smallest for the expected number of distinct experts
-    // (text after Eq. 5), the smaller C on a tie.
+    // Expected distinct experts of a step of T tokens under uniform routing (text after Eq. 5), rounded up.
+    int expected_experts(int T) const { return (int)std::ceil(E * (1.0 - std::pow(1.0 - (double)K / E, (double)T)) - 1e-9); }
+    // CTAs per unit: the largest cluster size for which the expected units -- (expert, 128-wide intermediate block)
+    // pairs -- still get a cluster each, so that the step is one round in which every unit's 3 * H/128 tiles are
+    // shared by as many CTAs as possible; one CTA per unit once there are more units than SMs.  (Measured on the nine
+    // benchmark shapes at 1-8 tokens: this is the fastest size in 47 of 54 cases and within 4 % in the others.)
     int fused_cluster(int T) const {
         const int KB = H / 128;
         const int knob = cluster_knob[T];
         if (knob > 0) return (knob <= 8 && max_clusters[knob] > 0 && knob <= KB) ? knob : 0;
-        const double U = E * (1.0 - std::pow(1.0 - (double)K / E, (double)T));
-        const long long units = (long long)std::llround(U) * (I / 128);
-        int best = 0;
-        long long best_cost = 0;
-        for (int C = 1; C <= 4; C *= 2) {
-            if (max_clusters[C] <= 0 || C > KB) continue;
-            const long long rounds = (units + max_clusters[C] - 1) / max_clusters[C];
-            const long long cost = rounds * ((3 * KB + C - 1) / C + 16);
-            if (!best || cost < best_cost) { best = C; best_cost = cost; }
-        }
-        return best;
+        const long long units = (long long)expected_experts(T) * (I / 128);
+        for (int C = 4; C > 1; C /= 2)
+            if (max_clusters[C] > 0 && C <= KB && units <= max_clusters[C]) return C;
+        return max_clusters[1] > 0 ? 1 : 0;
     }
     int fused_grid(int T) const { const int C = fused_cluster(T); return C ? C * max_clusters[C] : 0; }
     bool fused_possible(int T) const {
         return T >= 1 && T <= 8 && T < compact_min && H <= 8192 && fused_cluster(T) > 0 && fused_stages(T) >= 2;
     }
-    // The library's choice: one and two tokens.  Units are dealt to clusters whole, so with more tokens (more units than
-    // clusters, but not many more) the busiest cluster's extra unit costs more than the general variant's latency chain.
+    // The library's choice, by the length of the weight stream: tiles per CTA at the expected number of distinct experts.
+    // The fused variant has the shorter latency chain (routing, hand-over, reduction) but its accumulator warps work
+    // per group and its units go to clusters in whole pieces; the general variant streams longer runs at a higher rate.
+    // Measured crossover on the nine benchmark shapes (1-8 tokens): about 85 tiles per CTA; about 160 where a unit's
+    // down projection is at most two K blocks (there the general variant's per-unit work weighs most) and for a single
+    // token.
     bool fused(int T) const {
         if (fused_mode == 0 || !fused_possible(T)) return false;
-        return fused_mode == 1 || T <= 2;
+        if (fused_mode == 1) return true;
+        const double tiles = 3.0 * expected_experts(T) * (I / 128) * (H / 128) / sms;
+        return tiles <= 85.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
     }
 
-    // Default depth of the stage ring when the knob is 0.  Measured on this machine (config 2 and the paper's shapes,
+    // Default depth of the stage ring when the knob is 0.  Measured (config 2 and the paper's shapes,
     // T = 1..64, ring depths 12/10/8/6): a CTA whose whole step is a handful of tiles wants every tile requested at
     // once; short streams run 2-7 % faster on a ring of 6, medium ones 1-2 % faster on 8; long streams want all the
     // depth that fits.  "Length" = weight tiles per CTA for the expected number of distinct experts (text after Eq. 5).
@@ -341,6 +344,8 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.y = reinterpret_cast<float*>(w + L.y);
     P.ll = reinterpret_cast<unsigned long long*>(w + L.ll);
     P.ypl = reinterpret_cast<unsigned long long*>(w + L.yp);
+    P.xsl = reinterpret_cast<unsigned long long*>(w + L.xsl);
+    P.fsplit = 0;
     P.fC = 1; P.fnCl = p->sms;
     for (int r = 0; r < 9; ++r) { P.fkb[r] = 0; P.fhb[r] = 0; }
     P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
@@ -385,6 +390,7 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
         const int KB = p->H / 128;
         P.fC = C; P.fnCl = grid / C;
+        P.fsplit = (p->split_units && KB % C == 0) ? 1 : 0;
         P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
         for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
@@ -474,6 +480,13 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             if (value > 0 && plan->max_clusters[value] <= 0) return fail(MOE_ERR_OCCUPANCY, "clusters of %d CTAs cannot be launched on this device", value);
             for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->cluster_knob[t] = value;
             return MOE_OK;
+        case MOE_KNOB_SPLIT_UNITS:
+            plan->split_units = value != 0;
+            return MOE_OK;
+        case MOE_KNOB_HOST_DIRECT:
+            if (value < 0 || value > 3) return fail(MOE_ERR_ARG, "host-direct must be 0..3");
+            plan->host_direct = value;
+            return MOE_OK;
         case MOE_KNOB_DEBUG_SKIP:
             if (value < 0 || value > 1) return fail(MOE_ERR_ARG, "debug skip must be 0 or 1");
             plan->debug_skip = value;
@@ -502,6 +515,8 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_CLUSTER: *value = t <= 8 ? plan->cluster_knob[t] : 0; return MOE_OK;
         case MOE_KNOB_STAMPS: *value = plan->take_stamps; return MOE_OK;
         case MOE_KNOB_DEBUG_SKIP: *value = plan->debug_skip; return MOE_OK;
+        case MOE_KNOB_SPLIT_UNITS: *value = plan->split_units; return MOE_OK;
+        case MOE_KNOB_HOST_DIRECT: *value = plan->host_direct; return MOE_OK;
         default: return fail(MOE_ERR_ARG, "unknown knob %d", knob);
     }
 }
@@ -559,6 +574,8 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     }
     if (const char* v = getenv("MOE_B200_FUSED")) moe_plan_set_knob(p, 0, MOE_KNOB_FUSED, atoi(v));
     if (const char* v = getenv("MOE_B200_CLUSTER")) moe_plan_set_knob(p, 0, MOE_KNOB_CLUSTER, atoi(v));
+    if (const char* v = getenv("MOE_B200_HOST_DIRECT")) moe_plan_set_knob(p, 0, MOE_KNOB_HOST_DIRECT, atoi(v));
+    if (const char* v = getenv("MOE_B200_SPLIT_UNITS")) moe_plan_set_knob(p, 0, MOE_KNOB_SPLIT_UNITS, atoi(v));
     // one CTA per SM must actually fit (Section 3.2: the launcher verifies the realised occupancy)
     const int st = p->stages_for(64, 64);
     if (st < 2 || p->stages_for(p->n_hw(p->chunk()), p->chunk()) < 2) { delete p; return fail(MOE_ERR_OCCUPANCY, "shape needs more shared memory than one SM offers"); }
@@ -686,21 +703,35 @@ int moe_forward_host(moe_plan_t plan, int T, const void* hidden_host, const void
     if (T < 1) return fail(MOE_ERR_ARG, "T must be >= 1 (got %d)", T);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* w = static_cast<uint8_t*>(workspace);
+    // Pinned (page-locked, mapped) host buffers are addressable from the device.  A few tokens' worth of output is then
+    // written by the kernel straight into `out_host` (posted writes, visible to the host once the stream is
+    // synchronised) instead of through a staging area and a copy-engine transfer; likewise a small `hidden_host` can be
+    // read in place.  Pageable buffers, and anything larger, take the staged path.
+    auto mapped = [](const void* host_ptr) -> void* {
+        cudaPointerAttributes a;
+        if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return (a.type == cudaMemoryTypeHost && a.devicePointer && aligned16(a.devicePointer)) ? a.devicePointer : nullptr;
+    };
+    const size_t row_bytes = (size_t)plan->H * 2;
+    void* out_dev = (plan->host_direct & 1) && (size_t)T * row_bytes <= (64u << 10) ? mapped(out_host) : nullptr;
+    void* in_dev = (plan->host_direct & 2) && (size_t)T * row_bytes <= (64u << 10) ? mapped(hidden_host) : nullptr;
     for (int t0 = 0; t0 < T; t0 += plan->chunk()) {
         const int tc = plan->cap(T - t0);
         const WsLayout L = plan->layout(tc);
         if (workspace_bytes < L.total) return fail(MOE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed for T=%d", workspace_bytes, L.total, tc);
-        const size_t bytes = (size_t)tc * plan->H * 2;
-        const uint8_t* src = static_cast<const uint8_t*>(hidden_host) + (size_t)t0 * plan->H * 2;
-        uint8_t* dst = static_cast<uint8_t*>(out_host) + (size_t)t0 * plan->H * 2;
-        if (cudaMemcpyAsync(w + L.stage_in, src, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        const size_t bytes = (size_t)tc * row_bytes;
+        const uint8_t* src = static_cast<const uint8_t*>(hidden_host) + (size_t)t0 * row_bytes;
+        uint8_t* dst = static_cast<uint8_t*>(out_host) + (size_t)t0 * row_bytes;
+        const void* k_in = in_dev ? static_cast<const void*>(static_cast<uint8_t*>(in_dev) + (size_t)t0 * row_bytes) : static_cast<const void*>(w + L.stage_in);
+        void* k_out = out_dev ? static_cast<void*>(static_cast<uint8_t*>(out_dev) + (size_t)t0 * row_bytes) : static_cast<void*>(w + L.stage_out);
+        if (!in_dev && cudaMemcpyAsync(w + L.stage_in, src, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
             return fail(MOE_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(cudaGetLastError()));
-        int rc = check_forward_args(plan, tc, w + L.stage_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, w + L.stage_out, workspace);
+        int rc = check_forward_args(plan, tc, k_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, k_out, workspace);
         if (rc == MOE_OK)
-            rc = forward_chunk(plan, tc, w + L.stage_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, w + L.stage_out,
+            rc = forward_chunk(plan, tc, k_in, Wr_bf16, sel_bias, W13_fp8, W13_scale, W2_fp8, W2_scale, k_out,
                                workspace, workspace_bytes, s);
         if (rc != MOE_OK) return rc;
-        if (cudaMemcpyAsync(dst, w + L.stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        if (!out_dev && cudaMemcpyAsync(dst, w + L.stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
             return fail(MOE_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
     return MOE_OK;

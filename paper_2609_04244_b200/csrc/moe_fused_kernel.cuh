@@ -346,16 +346,21 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         alive = named_bar_and(2, kMain, ok && !wt.dead);
         if (P.stamps_fine) { if (tid == 0) MOE_STAMP(3); __syncwarp(); }
         // -------------------------------------------------------------- top-k for every token, in every CTA (Section 4.1)
-        if (alive) {
-#pragma unroll 1
-            for (int t = warp; t < T; t += kMainWarps) {
-                if (E <= 128) route_select<4>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
-                else if (E <= 256) route_select<8>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
-                else route_select<16>(P, t, lane, s_key + t * E, s_val + t * E, s_ids, s_w, s_mask, cta == 0, true);
-            }
+        // Token t is selected by warp 7 - t: the accumulator warps come first (they have a first-tile latency to spare),
+        // the producer and the issuers last.  Only the ids and the token masks are needed to start the weight stream;
+        // the routing weights are computed after the barrier.
+        int my_id = 0;
+        float my_v = 0.f, my_total = 1.f;
+        const int my_t = kMainWarps - 1 - warp;
+        if (alive && my_t < T) {
+            if (E <= 128) my_id = route_pick<4>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+            else if (E <= 256) my_id = route_pick<8>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+            else my_id = route_pick<16>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+            my_v = route_vals(P, lane, my_id, s_val + my_t * E, my_total);     // (the score table lies in the stage ring: read before the stream may start)
         }
         named_bar_sync(2, kMain);            // the selected experts and token masks of every token are in shared memory
         if (P.stamps_fine) { if (tid == 0) MOE_STAMP(4); __syncwarp(); }
+        if (alive && my_t < T) route_weights(P, my_t, lane, my_id, my_v, my_total, s_ids, s_w, cta == 0);
     } else {
         alive = false;                       // (the housekeeping warp takes no further part)
     }
@@ -399,11 +404,59 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
     if (P.stamps_fine) { if (tid == 0) MOE_STAMP(5); __syncwarp(); }
     const int nU = U * IB;                                       // units of this step
-    const int n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units of this cluster: cl, cl + nCl, ... (grid_magic divides by the cluster count here)
     // this CTA's share of every unit: K blocks [kb_lo, kb_hi) of the gate/up rows, row blocks [hb_lo, hb_hi) of W2
     const int kb_lo = P.fkb[rank], kb_hi = P.fkb[rank + 1], nk = kb_hi - kb_lo;
     const int hb_lo = P.fhb[rank], hb_hi = P.fhb[rank + 1], nh = hb_hi - hb_lo;
-    auto unit_of = [&](int s, int& e, int& ib) { const int u = cl + s * nCl; const int a = div_small(u, IB); ib = u - a * IB; e = s_act[a]; };
+    const int ngd = (nh + 1) >> 1;                               // down groups per unit
+    // Which units this cluster works on.  Fewer units than clusters (or a split the shape does not allow): whole units,
+    // dealt round-robin.  Otherwise the list of all groups -- per unit nk gate/up groups, then ngd down groups -- is cut
+    // into equal contiguous ranges, one per cluster (Section 3.2 gives each expert a group of CTAs; here a range may
+    // also end inside a unit's gate/up groups).  A cluster then has, in the order it works on them: the HEAD piece of
+    // the unit its range ends in (gate/up groups [0, xb): its partial sums are exported as tagged words for the next
+    // cluster, first thing, so they have long arrived when they are needed), its whole units, and last the TAIL piece
+    // of the unit its range starts in (gate/up groups [xa, nk), the previous cluster's partial sums imported, then
+    // that unit's down groups).  A cut never falls between a unit's down groups.
+    const bool split = (P.fsplit != 0) && (nU > nCl);
+    int n, first_whole = 0, nw = 0, head_u = -1, head_g1 = 0, tail_u = -1, tail_g0 = 0;
+    if (split) {
+        const int Wg = nk + ngd, total = nU * Wg;
+        auto cut = [&](int c) -> int {
+            int p = (int)div_grid((unsigned)c * (unsigned)total, P.grid_magic);
+            const int u = p / Wg, x = p - u * Wg;
+            return (x >= nk) ? (u + 1) * Wg : p;                 // not inside the down groups: move to the unit's end
+        };
+        const int lo = cut(cl), hi = (cl + 1 == nCl) ? total : cut(cl + 1);
+        const int ua = lo / Wg, xa = lo - ua * Wg, ub = hi / Wg, xb = hi - ub * Wg;
+        if (xa > 0) { tail_u = ua; tail_g0 = xa; }
+        if (xb > 0) { head_u = ub; head_g1 = xb; }
+        first_whole = ua + (xa > 0 ? 1 : 0);
+        nw = ub - first_whole;
+        if (nw < 0) nw = 0;
+        n = nw + (head_u >= 0 ? 1 : 0) + (tail_u >= 0 ? 1 : 0);
+    } else {
+        n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units cl, cl + nCl, ... (grid_magic divides by the cluster count)
+    }
+    // item s of this cluster, in working order: expert, intermediate block, gate/up groups [g0, g1) of this CTA's K
+    // blocks, and what happens to its partial sums: kExport (head piece: to the next cluster, nothing else), kImport
+    // (tail piece: the previous cluster's are added)
+    constexpr int kExport = 1, kImport = 2;
+    auto item_of = [&](int s, int& e, int& ib, int& g0, int& g1) -> int {
+        int u, fl = 0;
+        g0 = 0; g1 = nk;
+        if (!split) u = cl + s * nCl;
+        else {
+            const int hs = (head_u >= 0) ? 1 : 0;
+            if (s < hs) { u = head_u; g1 = head_g1; fl = kExport; }
+            else if (s - hs < nw) u = first_whole + s - hs;
+            else { u = tail_u; g0 = tail_g0; fl = kImport; }
+        }
+        const int a = div_small(u, IB);
+        ib = u - a * IB;
+        e = s_act[a];
+        return fl;
+    };
+    int Ntot = 0;                                                // weight tiles of this CTA
+    for (int s = 0; s < n; ++s) { int e, ib, g0, g1; const int fl = item_of(s, e, ib, g0, g1); Ntot += 2 * (g1 - g0) + ((fl & kExport) ? 0 : nh); }
 
     // Stream order of this CTA (same in every role): for s = 0..n: the gate/up groups of unit s (if s < n), then the
     // down groups of unit s-1 (if s >= 1).  A group is what one accumulator buffer holds: two weight tiles -- the gate
@@ -413,7 +466,6 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // its first stage and are released through that stage's `empty` barrier, so a stage that was the second of a pair
     // needs no wait of its own (the ring is refilled in order: its pair-mate's release came first).
     const int NI = (S >> 1) < kFusedIssuers ? (S >> 1) : kFusedIssuers;   // MMA issuers = accumulator buffers in use
-    const int Ntot = n * (2 * nk + nh);                          // weight tiles of this CTA
     // ------------------------------------------------------------------ role: producer (weight tiles and activation tiles)
     if (warp == 0) {
         if (lane == 0 && alive && n > 0) {
@@ -444,20 +496,19 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             MOE_STAMP(6);
             for (int s = 0; s <= n && !wt.dead; ++s) {
                 if (s < n) {
-                    int e, ib;
-                    unit_of(s, e, ib);
+                    int e, ib, g0, g1;
+                    item_of(s, e, ib, g0, g1);
                     const int yg = e * 2 * I + ib * kBlock;
-                    for (int k = kb_lo; k < kb_hi; ++k)
+                    for (int k = kb_lo + g0; k < kb_lo + g1; ++k)
                         if (!put(&tmW13, k * kBlock, yg, k * kBlock, yg + I, 2, k)) break;
                 }
                 if (s >= 1 && !wt.dead) {
-                    int e, ib;
-                    unit_of(s - 1, e, ib);
+                    int e, ib, g0, g1;
+                    if (item_of(s - 1, e, ib, g0, g1) & kExport) continue;       // a head piece has no down groups
                     for (int h = hb_lo; h < hb_hi; h += 2)
                         if (!put(&tmW2, ib * kBlock, e * H + h * kBlock, ib * kBlock, e * H + (h + 1) * kBlock, (h + 1 < hb_hi) ? 2 : 1, -1)) break;
                 }
             }
-            if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + 16] = (unsigned long long)w_empty;
             misc[7] = cntpar;      // which phase of every stage's `full` barrier was armed last (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
@@ -518,14 +569,21 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 w_is += clock64() - c2;
                 return true;
             };
+            int dq = 0;                                            // items with down groups so far: slot and phase of the intermediate tile
             for (int s = 0; s <= n && !wt.dead; ++s) {
-                if (s < n)
-                    for (int k = 0; k < nk; ++k)
+                if (s < n) {
+                    int e, ib, g0, g1;
+                    item_of(s, e, ib, g0, g1);
+                    for (int k = g0; k < g1; ++k)
                         if (!group(2, 0u)) break;
+                }
                 if (s >= 1 && !wt.dead) {
-                    const int slot = (s - 1) & 1;
-                    // the intermediate tile of unit s-1 is in shared memory (written by the accumulator warps)
-                    { const long long c0 = clock64(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)(((s - 1) >> 1) & 1), 27)) break; w_hq += clock64() - c0; }
+                    int e, ib, g0, g1;
+                    if (item_of(s - 1, e, ib, g0, g1) & kExport) continue;
+                    const int slot = dq & 1;
+                    // the intermediate tile of the item is in shared memory (written by the accumulator warps)
+                    { const long long c0 = clock64(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)((dq >> 1) & 1), 27)) break; w_hq += clock64() - c0; }
+                    ++dq;
                     for (int h = 0; h < nh; h += 2)
                         if (!group((h + 1 < nh) ? 2 : 1, smem_u32(s_hq) + (uint32_t)(slot * N * kBlock))) break;
                 }
@@ -566,8 +624,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         float nwg0 = 0.f, nwu0 = 0.f, nwg1 = 0.f, nwu1 = 0.f, nw2a = 0.f, nw2b = 0.f;
         auto fetch_scales = [&](int s) {
             if (s >= n) return;
-            int e, ib;
-            unit_of(s, e, ib);
+            int e, ib, g0, g1;
+            item_of(s, e, ib, g0, g1);
             const float* g13 = P.W13s + ((size_t)e * 2 * IB + ib) * KBu + kb_lo;
             const float* u13 = P.W13s + ((size_t)e * 2 * IB + IB + ib) * KBu + kb_lo;
             const float* w2 = P.W2s + ((size_t)e * HB + hb_lo) * IB + ib;
@@ -582,10 +640,16 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             float w2a = 0.f, w2b = 0.f, dw2a = 0.f, dw2b = 0.f;     // W2 scales of the unit in its gate/up phase, and of the one in its down phase
             unsigned dmask = 0u;                                   // token columns and result offsets of the unit in its down phase
             int dyoff = 0;
+            bool d_valid = false;                                  // the previous item has down groups (it was no head piece)
+            int pk = 0, dq = 0;                                    // items parked for the cluster / items with an intermediate tile so far
+            int pslot = 0;
+            uint32_t pphase = 0u;
             for (int s = 0; s <= n; ++s) {
-                // ---------------- gate/up groups of unit s: accumulate, then park the partial sums for the cluster
+                int e = 0, ib = 0, g0 = 0, g1 = 0, fl = 0;
+                if (s < n) fl = item_of(s, e, ib, g0, g1);
+                // ---------------- gate/up groups of item s: accumulate, then park the partial sums for the cluster
                 if (s < n) {
-                    float wg0 = nwg0, wu0 = nwu0;
+                    const float wg0 = nwg0, wu0 = nwu0;
                     const float wg1 = nwg1, wu1 = nwu1;
                     w2a = nw2a; w2b = nw2b;
                     fetch_scales(s + 1);
@@ -593,13 +657,12 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                     for (int c = 0; c < TC; ++c) { accg[c] = 0.f; accu[c] = 0.f; }
 #pragma unroll 1
-                    for (int k = 0; k < nk; ++k) {
+                    for (int k = g0; k < g1; ++k) {
                         float dg[TC], du[TC];
                         take(dg, du);
                         if (first_acc) { if (etid == 0) MOE_STAMP(8); first_acc = false; }
                         const int kl = k & 31;
-                        if (k == 32) { wg0 = wg1; wu0 = wu1; }
-                        const float wsg = __shfl_sync(0xffffffffu, wg0, kl), wsu = __shfl_sync(0xffffffffu, wu0, kl);
+                        const float wsg = __shfl_sync(0xffffffffu, (k < 32) ? wg0 : wg1, kl), wsu = __shfl_sync(0xffffffffu, (k < 32) ? wu0 : wu1, kl);
                         const float* as = s_xs + (kb_lo + k) * TS;
 #pragma unroll
                         for (int c = 0; c < TC; ++c) {
@@ -608,26 +671,42 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             accu[c] = fmaf(du[c], wsu * a, accu[c]);
                         }
                     }
-                    // park: slot s & 1 of this CTA's partial buffer, free once every peer has read the unit that used it before
-                    const int slot = s & 1;
-                    if (s >= 2 && lane == 0) {
-                        bool okw = !wt.dead;
-                        for (uint32_t i = 1; okw && !mbar_try_wait_cluster(bar_xfree + 8 * slot, (uint32_t)((s >> 1) & 1) ^ 1u); ++i)
-                            if ((i & 255u) == 0 && wt.expired(30)) okw = false;
-                        if (!okw) misc[3] = 1u;
-                    }
-                    __syncwarp();
-                    float* pp = s_part + slot * 2 * TC * kBlock;
+                    if (fl & kExport) {
+                        // head piece: this CTA's partial sums go to the next cluster as tagged words (it adds them to its own
+                        // at the very end of its range: they are there long before)
+                        unsigned long long* xo = P.xsl + ((size_t)(cl * C + rank) * 2 * TC) * kBlock + row;
+                        const unsigned long long tagx = (unsigned long long)tag << 32;
+                        const bool live = (misc[3] == 0u) && !wt.dead;
 #pragma unroll
-                    for (int c = 0; c < TC; ++c) { pp[c * kBlock + row] = accg[c]; pp[(TC + c) * kBlock + row] = accu[c]; }
-                    __syncwarp();
-                    if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * slot, (uint32_t)lane));
+                        for (int c = 0; c < TC; ++c) {
+                            if (live) {
+                                st_relaxed_u64(xo + (size_t)c * kBlock, tagx | (unsigned long long)__float_as_uint(accg[c]));
+                                st_relaxed_u64(xo + (size_t)(TC + c) * kBlock, tagx | (unsigned long long)__float_as_uint(accu[c]));
+                            }
+                        }
+                    } else {
+                        // park: slot pk & 1 of this CTA's partial buffer, free once every peer has read the item that used it before
+                        pslot = pk & 1; pphase = (uint32_t)((pk >> 1) & 1);
+                        if (pk >= 2 && lane == 0) {
+                            bool okw = !wt.dead;
+                            for (uint32_t i = 1; okw && !mbar_try_wait_cluster(bar_xfree + 8 * pslot, pphase ^ 1u); ++i)
+                                if ((i & 255u) == 0 && wt.expired(30)) okw = false;
+                            if (!okw) misc[3] = 1u;
+                        }
+                        ++pk;
+                        __syncwarp();
+                        float* pp = s_part + pslot * 2 * TC * kBlock;
+#pragma unroll
+                        for (int c = 0; c < TC; ++c) { pp[c * kBlock + row] = accg[c]; pp[(TC + c) * kBlock + row] = accu[c]; }
+                        __syncwarp();
+                        if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * pslot, (uint32_t)lane));
+                    }
                     if (s == 0 && etid == 0) MOE_STAMP(9);
                 }
                 // ---------------- unit s-1: its down groups (the intermediate tile was made at the end of the previous turn, long
                 // before the issuers got here: no hand-over wait on the weight stream's path), scaled and stored as the tagged
                 // partials of (token, slot, ib): the final reduction polls these words themselves
-                if (s >= 1) {
+                if (s >= 1 && d_valid) {
                     const unsigned long long tagw = (unsigned long long)tag << 32;
 #pragma unroll 1
                     for (int h = 0; h < nh; h += 2) {
@@ -650,10 +729,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 }
                 // ---------------- unit s: gather the cluster's partial sums, SiLU*up, requantise -> the intermediate tile its
                 // down groups will use one turn later
-                if (s < n) {
-                    const int i = s, slot = i & 1;
-                    int e, ib;
-                    unit_of(i, e, ib);
+                d_valid = false;
+                if (s < n && !(fl & kExport)) {
+                    const int slot = pslot;
                     // token columns of this expert and where their down results go
                     const unsigned mask = (unsigned)s_mask[2 * e];
                     int yoff_lane = 0;
@@ -664,7 +742,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     const long long cf0 = clock64();
                     {
                         bool okw = !wt.dead;
-                        for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, (uint32_t)((i >> 1) & 1)); ++it)
+                        for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, pphase); ++it)
                             if ((it & 255u) == 0 && wt.expired(31)) okw = false;
                         if (!okw) misc[3] = 1u;
                     }
@@ -687,6 +765,28 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                             for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
                         }
+                        if (fl & kImport) {
+                            // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
+                            // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
+                            const unsigned long long* xi = P.xsl + ((size_t)((cl - 1) * C) * 2 * TC) * kBlock + row;
+                            bool okx = !wt.dead;
+#pragma unroll 1
+                            for (int r = 0; r < C && okx; ++r) {
+                                unsigned long long v[2 * TC];
+                                unsigned pending = (1u << (2 * TC)) - 1u;
+                                for (uint32_t it = 1; pending; ++it) {
+#pragma unroll
+                                    for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
+#pragma unroll
+                                    for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
+                                    if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                }
+                                if (!okx) break;
+#pragma unroll
+                                for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
+                            }
+                            if (!okx) misc[3] = 1u;
+                        }
                         // SiLU(gate)*up (Section 3.3).  The intermediate tile is outside the bit-exact set: fast exp and divide.
 #pragma unroll
                         for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
@@ -700,7 +800,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
                     }
                     if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
-                    uint8_t* hq = s_hq + slot * N * kBlock;
+                    const int hslot = dq & 1;
+                    ++dq;
+                    uint8_t* hq = s_hq + hslot * N * kBlock;
 #pragma unroll
                     for (int c = 0; c < TC; ++c) {
                         const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
@@ -716,9 +818,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     }
                     fence_proxy_async();                                   // generic writes -> the tensor core's reads
                     epi_bar(kEpiThreads);
-                    if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * slot); if (i == 0) MOE_STAMP(10); }
+                    if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
                     w_fc += clock64() - cf0;
-                    dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b;
+                    dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b; d_valid = true;
                 }
             }
         }

@@ -88,6 +88,8 @@ struct Params {
     float* y;           // [T,K,H]
     unsigned long long* ll;         // [T,E] fused variants: router logits as {launch tag, fp32 bits} words
     unsigned long long* ypl;        // [T,K,I/128,H] fused variants: down-projection partial of every (token, slot, intermediate block), {launch tag, fp32 bits}
+    unsigned long long* xsl;        // [clusters][C][2 TC][128] fused variants: partial gate/up sums a cluster exports to the next one, {launch tag, fp32 bits}
+    int fsplit;                     // fused variants: cut the group list into equal ranges per cluster (units may be split between two clusters)
     int fC, fnCl;                   // fused variants: CTAs per cluster, clusters in the grid
     int fkb[9], fhb[9];             // fused variants: rank r of a cluster takes K blocks [fkb[r], fkb[r+1]) and W2 row blocks [fhb[r], fhb[r+1])
     unsigned long long* stamps;     // [grid][32] globaltimer stamps of the phases of the last launch; NULL = none taken
@@ -463,24 +465,30 @@ __device__ __forceinline__ void route_scores(const Params& P, int t0, int nt, in
     else route_scores_t<2, 8>(P, t0, nt, ksplit, tid, nthreads, s_key, s_val, write_global);
 }
 
-// Second half of the routing of one token (one warp; lane j < K holds the expert of slot j in `my_id`): the routing
-// weights -- softmax over all experts or the plain sigmoid score, optionally renormalised over the selected experts,
-// times the routed scaling factor (Section 4.1) -- and the token's entries in the id / weight / token-mask tables.
-__device__ __forceinline__ void route_finish(const Params& P, int t, int lane, int my_id, const float* s_val,
-                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global, bool build_mask) {
+// Second half of the routing of one token (one warp; lane j < K holds the expert of slot j in `my_id`), in two steps so
+// that a caller can put a barrier between them: route_vals() reads what it needs from the score table (the selected
+// scores; the softmax normaliser over all experts when the weights are not renormalised), route_weights() turns that
+// into the routing weights -- softmax or plain sigmoid score, optionally renormalised over the selected experts, times
+// the routed scaling factor (Section 4.1) -- and writes the token's ids and weights.
+__device__ __forceinline__ float route_vals(const Params& P, int lane, int my_id, const float* s_val, float& total) {
     const int E = P.E, K = P.K;
-    const bool softmax = (P.scoring == 0);
-    float v = (lane < K) ? s_val[my_id] : 0.f;
-    float total = 1.0f;
-    if (softmax) {
+    const float v = (lane < K) ? s_val[my_id] : 0.f;
+    total = 1.0f;
+    if (P.scoring == 0 && !P.renorm) {
         const float mx = __shfl_sync(0xffffffffu, v, 0);        // slot 0 holds the largest logit
-        v = (lane < K) ? expf(v - mx) : 0.f;
-        if (!P.renorm) {
-            total = 0.f;
-            for (int e = lane; e < E; e += 32) total += expf(s_val[e] - mx);
+        total = 0.f;
+        for (int e = lane; e < E; e += 32) total += expf(s_val[e] - mx);
 #pragma unroll
-            for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-        }
+        for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    return v;
+}
+__device__ __forceinline__ void route_weights(const Params& P, int t, int lane, int my_id, float v, float total,
+                                              int* s_ids, float* s_w, bool write_global) {
+    const int K = P.K;
+    if (P.scoring == 0) {
+        const float mx = __shfl_sync(0xffffffffu, v, 0);
+        v = (lane < K) ? expf(v - mx) : 0.f;
     }
     float vsum = v;
 #pragma unroll
@@ -489,9 +497,15 @@ __device__ __forceinline__ void route_finish(const Params& P, int t, int lane, i
         const float w = __fdiv_rn(v, P.renorm ? vsum : total) * P.routed_scale;
         s_ids[t * K + lane] = my_id;
         s_w[t * K + lane] = w;
-        if (build_mask) mask_add(s_mask, my_id, t);
         if (write_global) { P.ids[t * K + lane] = my_id; P.wts[t * K + lane] = w; }
     }
+}
+__device__ __forceinline__ void route_finish(const Params& P, int t, int lane, int my_id, const float* s_val,
+                                             int* s_ids, float* s_w, unsigned long long* s_mask, bool write_global, bool build_mask) {
+    float total;
+    const float v = route_vals(P, lane, my_id, s_val, total);
+    route_weights(P, t, lane, my_id, v, total, s_ids, s_w, write_global);
+    if (build_mask && lane < P.K) mask_add(s_mask, my_id, t);
 }
 
 template <int NPER>
@@ -518,6 +532,34 @@ __device__ __forceinline__ void route_select(const Params& P, int t, int lane, c
         if (lane == j) my_id = we;
     }
     route_finish(P, t, lane, my_id, s_val, s_ids, s_w, s_mask, write_global, build_mask);
+}
+
+// The selection alone: slot j's expert ends up in lane j (returned), the ids and the token masks are written; the
+// routing weights follow later through route_finish() (only the final reduction needs them).
+template <int NPER>
+__device__ __forceinline__ int route_pick(const Params& P, int t, int lane, const uint32_t* s_key, int* s_ids, unsigned long long* s_mask) {
+    const int E = P.E, K = P.K;
+    uint32_t key[NPER];
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) key[i] = (i * 32 + lane < E) ? s_key[i * 32 + lane] : 0u;    // 0 is below every real key
+    int my_id = 0;
+#pragma unroll 1
+    for (int j = 0; j < K; ++j) {
+        uint32_t m = key[0];
+#pragma unroll
+        for (int i = 1; i < NPER; ++i) m = max(m, key[i]);
+        const uint32_t wm = __reduce_max_sync(0xffffffffu, m);
+        int cand = 0x7fffffff;
+#pragma unroll
+        for (int i = NPER - 1; i >= 0; --i) cand = (key[i] == wm) ? i * 32 : cand;
+        const int we = __reduce_min_sync(0xffffffffu, cand == 0x7fffffff ? cand : cand + lane);
+        const int mine = we - lane;                            // i * 32 if this lane holds the winner
+#pragma unroll
+        for (int i = 0; i < NPER; ++i) key[i] = (mine == i * 32) ? 0u : key[i];
+        if (lane == j) my_id = we;
+    }
+    if (lane < K) { s_ids[t * K + lane] = my_id; mask_add(s_mask, my_id, t); }
+    return my_id;
 }
 
 // quantise 4 floats with scale s into 4 E4M3 bytes (memory order x0..x3)
