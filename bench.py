@@ -30,13 +30,19 @@ if ROOT not in sys.path:
 METRIC = "us_per_moe_layer_step"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the fused kernel from the ncu
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the step's kernel from the ncu
 # captures summarised under profiles/; keyed by (config, tokens).  None where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("c2_qwen3_30b_a3b", 1): 38.700e6 + 0.036e6,     # profiles/moe_decode_kernel_c2_qwen3_t1.md
+    ("c1_tiny", 1): 3.496e6,                         # profiles/moe_fused_kernel_c1_tiny_t1.md
+    ("c2_qwen3_30b_a3b", 1): 39.208e6 + 0.190e6,     # profiles/moe_fused_kernel_c2_qwen3_t1.md
+    ("c2_qwen3_30b_a3b", 2): 76.977e6 + 1.894e6,     # profiles/moe_fused_kernel_c2_qwen3_t2.md
+    ("c2_qwen3_30b_a3b", 4): 150.04e6 + 4.18e6,      # profiles/moe_fused_kernel_c2_qwen3_t4.md
+    ("c2_qwen3_30b_a3b", 8): 249.25e6 + 4.28e6,      # profiles/moe_decode_kernel_c2_qwen3_t8.md
     ("c2_qwen3_30b_a3b", 64): 601.9e6 + 5.6e6,       # profiles/moe_decode_kernel_c2_qwen3_t64.md
+    ("c4_mixtral_8x7b", 1): 366.13e6 + 4.69e6,       # profiles/moe_fused_kernel_c4_mixtral_t1.md
     ("c4_mixtral_8x7b", 64): 1416.3e6 + 6.8e6,       # profiles/moe_decode_kernel_c4_mixtral_t64.md
     ("c5_deepseek_v3[E=16]", 1): 356.76e6 + 4.67e6,  # profiles/moe_decode_kernel_c5like_e16_t1.md
+    ("c5_deepseek_v3[E=32]", 1): 353.61e6 + 5.08e6,  # profiles/moe_fused_kernel_c5like_e32_t1.md
     ("c5_deepseek_v3[E=64]", 8): 1680.1e6 + 4.8e6,   # profiles/moe_decode_kernel_c5like_e64_t8.md
 }
 
@@ -385,10 +391,13 @@ def main():
         h_in = [layers[l]["hidden"].cpu().pin_memory() for l in range(L)]
         h_out = torch.empty((T, shape.H), dtype=torch.bfloat16).pin_memory()
 
+        bound = [plan.bind_forward_host(h_in[l], layers[l]["Wr"], layers[l]["bias"], layers[l]["W13q"], layers[l]["W13s"],
+                                        layers[l]["W2q"], layers[l]["W2s"], h_out, stream) for l in range(L)]
+        sync = stream.synchronize
+
         def e2e_step(i):
-            d = layers[i % L]
-            plan.forward_host(h_in[i % L], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"], h_out, stream)
-            stream.synchronize()
+            bound[i % L]()          # moe_forward_host: H2D copy of the step's input, the kernel (writes h_out itself)
+            sync()                  # the caller consumes the result before the next step
 
         Ke = min(K, 2000)
         for i in range(W):
@@ -420,6 +429,7 @@ def main():
             gbs = r["bytes_per_step"] / (us * 1e-6) / 1e9
             cells.append({"workload": f"{name} T={Tc} regime={regime}", "us": us, "steps": Kc,
                           "algorithmic_bytes_per_step": r["bytes_per_step"], "achieved_gbs": gbs, "frac": gbs / peak_c,
+                          "traffic": NCU_TRAFFIC_BYTES.get((name, Tc)) if regime == "natural" else None,
                           "unique_experts_mean": float(np.mean(r["uniq"])), "layer_copies": r["L"],
                           "variant": kernel_name(r["info"], Tc), "cluster": r["info"]["cluster"], "stages": r["info"]["stages"],
                           "clocks": {k: r["clocks"].get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")}})

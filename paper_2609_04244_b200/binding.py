@@ -248,6 +248,24 @@ class MoEPlan:
                          self.workspace, stream)
         return out_host
 
+    def bind_forward_host(self, hidden_host, Wr, sel_bias, W13q, W13s, W2q, W2s, out_host, stream=None):
+        """moe_forward_host with its arguments marshalled once: returns a zero-argument callable that enqueues the step on
+        `stream`.  For callers that repeat a step on the same buffers (a decode loop re-filling `hidden_host` in place):
+        only the C call remains per step."""
+        if hidden_host.is_cuda or out_host.is_cuda or not hidden_host.is_contiguous() or not out_host.is_contiguous():
+            raise MoEError(-1, "hidden_host and out_host must be contiguous host tensors")
+        fn = load_library().moe_forward_host
+        args = (self.handle, hidden_host.shape[0], ctypes.c_void_p(hidden_host.data_ptr()), _p(Wr), _p(sel_bias), _p(W13q),
+                _p(W13s), _p(W2q), _p(W2s), ctypes.c_void_p(out_host.data_ptr()), _p(self.workspace),
+                self.workspace.numel() * self.workspace.element_size(), _stream(stream))
+        keep = (hidden_host, Wr, sel_bias, W13q, W13s, W2q, W2s, out_host)      # the tensors must outlive the callable
+
+        def step(_keep=keep):
+            rc = fn(*args)
+            if rc != 0:
+                _check(rc)
+        return step
+
     def forward_debug(self, hidden, Wr, sel_bias, W13q, W13s, W2q, W2s, stream=None):
         T, dev = hidden.shape[0], hidden.device
         out = torch.empty((T, self.H), dtype=torch.bfloat16, device=dev)
