@@ -225,7 +225,9 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *   MOE_KNOB_HOST_DIRECT       (plan-wide) moe_forward_host with PINNED host buffers of at most 64 KiB: bit 0 (default on) = the
  *                              kernel writes the result straight into out_host, bit 1 = it reads hidden_host in place; the
  *                              transfers that are not taken this way go through a staging area and the copy engine
- *   MOE_KNOB_STAMPS            (plan-wide) kernels record the phase time stamps moe_debug_stamps() reads; off by default
+ *   MOE_KNOB_STAMPS            (plan-wide) the fused-unit variant records the phase time stamps moe_debug_stamps() reads
+ *                              (1; 2 = also inside its routing phase); off by default.  The general variant always records
+ *                              its sixteen stamps: one store per phase, and guarding them measured slower
  *   MOE_KNOB_DEBUG_SKIP        (plan-wide, for tests of the give-up paths) 1: the fused-unit variant never signals that an
  *                              intermediate tile is ready, so every wait behind that signal runs out after the plan's time
  *                              limit and the launch ends with MOE_ERR_TIMEOUT -- no fault, nothing waits for ever.  0 (default)

@@ -258,7 +258,7 @@ int launch(Plan* p, const CUtensorMap& m13, const CUtensorMap& m2, const CUtenso
 }
 
 // Fused-unit variants: grid = clusters x C CTAs, cluster size chosen at run time.
-template <int TC>
+template <int TC, bool SPLIT>
 int launch_fused(Plan* p, int grid, int C, const CUtensorMap& m13, const CUtensorMap& m2, const CUtensorMap& mx,
                  const moe::Params& P, int smem_bytes, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
@@ -273,7 +273,7 @@ int launch_fused(Plan* p, int grid, int C, const CUtensorMap& m13, const CUtenso
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p->use_pdl ? 2 : 1;
-    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_fused_kernel<TC>, m13, m2, mx, P);
+    cudaError_t err = cudaLaunchKernelEx(&cfg, moe::moe_fused_kernel<TC, SPLIT>, m13, m2, mx, P);
     if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(MOE_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
     return MOE_OK;
@@ -283,7 +283,8 @@ int launch_fused(Plan* p, int grid, int C, const CUtensorMap& m13, const CUtenso
 // the SM may still belong to the previous launch); 0 when such a cluster cannot be launched at all.
 template <int TC>
 int fused_clusters(int C, int smem_optin, int sms) {
-    if (cudaFuncSetAttribute(moe::moe_fused_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaFuncSetAttribute(moe::moe_fused_kernel<TC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaFuncSetAttribute(moe::moe_fused_kernel<TC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) { cudaGetLastError(); return 0; }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((sms / C) * C, 1, 1);
     cfg.blockDim = dim3(moe::kFusedThreads, 1, 1);
@@ -294,7 +295,10 @@ int fused_clusters(int C, int smem_optin, int sms) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, moe::moe_fused_kernel<TC>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    int m = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, moe::moe_fused_kernel<TC, false>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaOccupancyMaxActiveClusters(&m, moe::moe_fused_kernel<TC, true>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (m < n) n = m;
     return n < sms / C ? n : sms / C;
 }
 
@@ -349,6 +353,7 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.fC = 1; P.fnCl = p->sms;
     for (int r = 0; r < 9; ++r) { P.fkb[r] = 0; P.fhb[r] = 0; }
     P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
+    P.stamps_buf = reinterpret_cast<unsigned long long*>(w + L.stamps);
     P.stamps_fine = p->take_stamps >= 2;
     P.debug_skip = p->debug_skip;
     return P;
@@ -390,15 +395,18 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
         const int KB = p->H / 128;
         P.fC = C; P.fnCl = grid / C;
-        P.fsplit = (p->split_units && KB % C == 0) ? 1 : 0;
+        // units are shared between clusters only where the step can have more units than clusters at all: T tokens select
+        // at most min(E, T * top_k) experts (the instantiations without that code are smaller and faster)
+        const int max_units = (T * p->K < p->E ? T * p->K : p->E) * (p->I / 128);
+        P.fsplit = (p->split_units && KB % C == 0 && max_units > P.fnCl) ? 1 : 0;
         P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
         for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
         switch (TC) {
-            case 1: return launch_fused<1>(p, grid, C, m13, m2, mx, P, smem, stream);
-            case 2: return launch_fused<2>(p, grid, C, m13, m2, mx, P, smem, stream);
-            case 4: return launch_fused<4>(p, grid, C, m13, m2, mx, P, smem, stream);
-            default: return launch_fused<8>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 1: return P.fsplit ? launch_fused<1, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<1, false>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 2: return P.fsplit ? launch_fused<2, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<2, false>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 4: return P.fsplit ? launch_fused<4, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<4, false>(p, grid, C, m13, m2, mx, P, smem, stream);
+            default: return P.fsplit ? launch_fused<8, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<8, false>(p, grid, C, m13, m2, mx, P, smem, stream);
         }
     }
     const int N = p->n_hw(T);

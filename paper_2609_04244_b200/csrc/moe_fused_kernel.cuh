@@ -128,14 +128,16 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
 }
 
 // ---------------------------------------------------------------------------------------------
-// the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8 >= T).
+// the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8 >= T).  SPLIT = the step may have more units
+// than clusters, so the code that shares a unit between two clusters is compiled in (the host knows the largest unit
+// count a token count can give; the instantiations without it are smaller and measurably faster on the short steps).
 // Warps: 0 producer (weight and activation tiles), 1..3 MMA issuers, 4..7 accumulator warps; warp 8 keeps house
 // during the routing phase (everything that costs L2 round trips but is not needed before the first activation tile).
 // ---------------------------------------------------------------------------------------------
 #ifndef MOE_FUSED_MIN_BLOCKS
 #define MOE_FUSED_MIN_BLOCKS 1
 #endif
-template <int TC>
+template <int TC, bool SPLIT>
 __global__ void __launch_bounds__(kFusedThreads, MOE_FUSED_MIN_BLOCKS)
 moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constant__ CUtensorMap tmW2,
                  const __grid_constant__ CUtensorMap tmXq, const __grid_constant__ Params P) {
@@ -411,24 +413,22 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // Which units this cluster works on.  Fewer units than clusters (or a split the shape does not allow): whole units,
     // dealt round-robin.  Otherwise the list of all groups -- per unit nk gate/up groups, then ngd down groups -- is cut
     // into equal contiguous ranges, one per cluster (Section 3.2 gives each expert a group of CTAs; here a range may
-    // also end inside a unit's gate/up groups).  A cluster then has, in the order it works on them: the HEAD piece of
-    // the unit its range ends in (gate/up groups [0, xb): its partial sums are exported as tagged words for the next
-    // cluster, first thing, so they have long arrived when they are needed), its whole units, and last the TAIL piece
-    // of the unit its range starts in (gate/up groups [xa, nk), the previous cluster's partial sums imported, then
-    // that unit's down groups).  A cut never falls between a unit's down groups.
-    const bool split = (P.fsplit != 0) && (nU > nCl);
-    int n, first_whole = 0, nw = 0, head_u = -1, head_g1 = 0, tail_u = -1, tail_g0 = 0;
+    // end anywhere inside a unit).  A cluster then has, in the order it works on them: the HEAD piece of the unit its
+    // range ends in (gate/up groups [0, g1) and, if the cut lies beyond them, down groups [0, d1); its partial sums are
+    // exported as tagged words for the next cluster right after its gate/up groups, first thing, so they have long
+    // arrived when they are needed), its whole units, and last the TAIL piece of the unit its range starts in (gate/up
+    // groups [g0, nk) -- none if the cut lies beyond them --, the previous cluster's partial sums imported, then the
+    // unit's down groups [d0, ngd)).  When a unit's down groups are shared, both clusters hold its complete sums (one
+    // computed them, one imported them) and both make the intermediate tile, with the same arithmetic in the same order.
+    const bool split = SPLIT && (P.fsplit != 0) && (nU > nCl);
+    int n, first_whole = 0, nw = 0, head_u = -1, head_g1 = 0, head_d1 = 0, tail_u = -1, tail_g0 = 0, tail_d0 = 0;
     if (split) {
         const int Wg = nk + ngd, total = nU * Wg;
-        auto cut = [&](int c) -> int {
-            int p = (int)div_grid((unsigned)c * (unsigned)total, P.grid_magic);
-            const int u = p / Wg, x = p - u * Wg;
-            return (x >= nk) ? (u + 1) * Wg : p;                 // not inside the down groups: move to the unit's end
-        };
+        auto cut = [&](int c) -> int { return (int)div_grid((unsigned)c * (unsigned)total, P.grid_magic); };
         const int lo = cut(cl), hi = (cl + 1 == nCl) ? total : cut(cl + 1);
         const int ua = lo / Wg, xa = lo - ua * Wg, ub = hi / Wg, xb = hi - ub * Wg;
-        if (xa > 0) { tail_u = ua; tail_g0 = xa; }
-        if (xb > 0) { head_u = ub; head_g1 = xb; }
+        if (xa > 0) { tail_u = ua; tail_g0 = xa < nk ? xa : nk; tail_d0 = xa > nk ? xa - nk : 0; }
+        if (xb > 0) { head_u = ub; head_g1 = xb < nk ? xb : nk; head_d1 = xb > nk ? xb - nk : 0; }
         first_whole = ua + (xa > 0 ? 1 : 0);
         nw = ub - first_whole;
         if (nw < 0) nw = 0;
@@ -437,18 +437,19 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units cl, cl + nCl, ... (grid_magic divides by the cluster count)
     }
     // item s of this cluster, in working order: expert, intermediate block, gate/up groups [g0, g1) of this CTA's K
-    // blocks, and what happens to its partial sums: kExport (head piece: to the next cluster, nothing else), kImport
-    // (tail piece: the previous cluster's are added)
+    // blocks, down groups [d0, d1) of this CTA's row blocks (none: the item ends with its partial sums), and what
+    // happens to its partial sums: kExport (head piece: stored for the next cluster), kImport (tail piece: the previous
+    // cluster's are added)
     constexpr int kExport = 1, kImport = 2;
-    auto item_of = [&](int s, int& e, int& ib, int& g0, int& g1) -> int {
+    auto item_of = [&](int s, int& e, int& ib, int& g0, int& g1, int& d0, int& d1) -> int {
         int u, fl = 0;
-        g0 = 0; g1 = nk;
-        if (!split) u = cl + s * nCl;
+        g0 = 0; g1 = nk; d0 = 0; d1 = ngd;
+        if (!SPLIT || !split) u = cl + s * nCl;
         else {
             const int hs = (head_u >= 0) ? 1 : 0;
-            if (s < hs) { u = head_u; g1 = head_g1; fl = kExport; }
+            if (s < hs) { u = head_u; g1 = head_g1; d1 = head_d1; fl = kExport; }
             else if (s - hs < nw) u = first_whole + s - hs;
-            else { u = tail_u; g0 = tail_g0; fl = kImport; }
+            else { u = tail_u; g0 = tail_g0; d0 = tail_d0; fl = kImport; }
         }
         const int a = div_small(u, IB);
         ib = u - a * IB;
@@ -456,7 +457,11 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         return fl;
     };
     int Ntot = 0;                                                // weight tiles of this CTA
-    for (int s = 0; s < n; ++s) { int e, ib, g0, g1; const int fl = item_of(s, e, ib, g0, g1); Ntot += 2 * (g1 - g0) + ((fl & kExport) ? 0 : nh); }
+    for (int s = 0; s < n; ++s) {
+        int e, ib, g0, g1, d0, d1;
+        item_of(s, e, ib, g0, g1, d0, d1);
+        Ntot += 2 * (g1 - g0) + ((2 * d1 < nh ? 2 * d1 : nh) - 2 * d0);     // (a unit's last down group may be a single tile)
+    }
 
     // Stream order of this CTA (same in every role): for s = 0..n: the gate/up groups of unit s (if s < n), then the
     // down groups of unit s-1 (if s >= 1).  A group is what one accumulator buffer holds: two weight tiles -- the gate
@@ -496,19 +501,20 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             MOE_STAMP(6);
             for (int s = 0; s <= n && !wt.dead; ++s) {
                 if (s < n) {
-                    int e, ib, g0, g1;
-                    item_of(s, e, ib, g0, g1);
+                    int e, ib, g0, g1, d0, d1;
+                    item_of(s, e, ib, g0, g1, d0, d1);
                     const int yg = e * 2 * I + ib * kBlock;
                     for (int k = kb_lo + g0; k < kb_lo + g1; ++k)
                         if (!put(&tmW13, k * kBlock, yg, k * kBlock, yg + I, 2, k)) break;
                 }
                 if (s >= 1 && !wt.dead) {
-                    int e, ib, g0, g1;
-                    if (item_of(s - 1, e, ib, g0, g1) & kExport) continue;       // a head piece has no down groups
-                    for (int h = hb_lo; h < hb_hi; h += 2)
+                    int e, ib, g0, g1, d0, d1;
+                    item_of(s - 1, e, ib, g0, g1, d0, d1);
+                    for (int h = hb_lo + 2 * d0; h < hb_hi && h < hb_lo + 2 * d1; h += 2)
                         if (!put(&tmW2, ib * kBlock, e * H + h * kBlock, ib * kBlock, e * H + (h + 1) * kBlock, (h + 1 < hb_hi) ? 2 : 1, -1)) break;
                 }
             }
+            if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + 16] = (unsigned long long)w_empty;
             misc[7] = cntpar;      // which phase of every stage's `full` barrier was armed last (the teardown waits for them if the launch gave up)
         }
         __syncwarp();
@@ -572,19 +578,20 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             int dq = 0;                                            // items with down groups so far: slot and phase of the intermediate tile
             for (int s = 0; s <= n && !wt.dead; ++s) {
                 if (s < n) {
-                    int e, ib, g0, g1;
-                    item_of(s, e, ib, g0, g1);
+                    int e, ib, g0, g1, d0, d1;
+                    item_of(s, e, ib, g0, g1, d0, d1);
                     for (int k = g0; k < g1; ++k)
                         if (!group(2, 0u)) break;
                 }
                 if (s >= 1 && !wt.dead) {
-                    int e, ib, g0, g1;
-                    if (item_of(s - 1, e, ib, g0, g1) & kExport) continue;
+                    int e, ib, g0, g1, d0, d1;
+                    item_of(s - 1, e, ib, g0, g1, d0, d1);
+                    if (d1 <= d0) continue;                                  // (a head piece that ends with its partial sums)
                     const int slot = dq & 1;
                     // the intermediate tile of the item is in shared memory (written by the accumulator warps)
                     { const long long c0 = clock64(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)((dq >> 1) & 1), 27)) break; w_hq += clock64() - c0; }
                     ++dq;
-                    for (int h = 0; h < nh; h += 2)
+                    for (int h = 2 * d0; h < nh && h < 2 * d1; h += 2)
                         if (!group((h + 1 < nh) ? 2 : 1, smem_u32(s_hq) + (uint32_t)(slot * N * kBlock))) break;
                 }
             }
@@ -624,8 +631,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         float nwg0 = 0.f, nwu0 = 0.f, nwg1 = 0.f, nwu1 = 0.f, nw2a = 0.f, nw2b = 0.f;
         auto fetch_scales = [&](int s) {
             if (s >= n) return;
-            int e, ib, g0, g1;
-            item_of(s, e, ib, g0, g1);
+            int e, ib, g0, g1, d0, d1;
+            item_of(s, e, ib, g0, g1, d0, d1);
             const float* g13 = P.W13s + ((size_t)e * 2 * IB + ib) * KBu + kb_lo;
             const float* u13 = P.W13s + ((size_t)e * 2 * IB + IB + ib) * KBu + kb_lo;
             const float* w2 = P.W2s + ((size_t)e * HB + hb_lo) * IB + ib;
@@ -640,13 +647,14 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             float w2a = 0.f, w2b = 0.f, dw2a = 0.f, dw2b = 0.f;     // W2 scales of the unit in its gate/up phase, and of the one in its down phase
             unsigned dmask = 0u;                                   // token columns and result offsets of the unit in its down phase
             int dyoff = 0;
-            bool d_valid = false;                                  // the previous item has down groups (it was no head piece)
+            bool d_valid = false;                                  // the previous item has down groups
+            int dh0 = 0, dh1 = 0;                                  // ... for the row blocks [dh0, dh1) of this CTA's share
             int pk = 0, dq = 0;                                    // items parked for the cluster / items with an intermediate tile so far
             int pslot = 0;
             uint32_t pphase = 0u;
             for (int s = 0; s <= n; ++s) {
-                int e = 0, ib = 0, g0 = 0, g1 = 0, fl = 0;
-                if (s < n) fl = item_of(s, e, ib, g0, g1);
+                int e = 0, ib = 0, g0 = 0, g1 = 0, d0 = 0, d1 = 0, fl = 0;
+                if (s < n) fl = item_of(s, e, ib, g0, g1, d0, d1);
                 // ---------------- gate/up groups of item s: accumulate, then park the partial sums for the cluster
                 if (s < n) {
                     const float wg0 = nwg0, wu0 = nwu0;
@@ -671,7 +679,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             accu[c] = fmaf(du[c], wsu * a, accu[c]);
                         }
                     }
-                    if (fl & kExport) {
+                    if (SPLIT && (fl & kExport)) {
                         // head piece: this CTA's partial sums go to the next cluster as tagged words (it adds them to its own
                         // at the very end of its range: they are there long before)
                         unsigned long long* xo = P.xsl + ((size_t)(cl * C + rank) * 2 * TC) * kBlock + row;
@@ -684,7 +692,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                                 st_relaxed_u64(xo + (size_t)(TC + c) * kBlock, tagx | (unsigned long long)__float_as_uint(accu[c]));
                             }
                         }
-                    } else {
+                    }
+                    if (d1 > d0) {
                         // park: slot pk & 1 of this CTA's partial buffer, free once every peer has read the item that used it before
                         pslot = pk & 1; pphase = (uint32_t)((pk >> 1) & 1);
                         if (pk >= 2 && lane == 0) {
@@ -709,9 +718,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 if (s >= 1 && d_valid) {
                     const unsigned long long tagw = (unsigned long long)tag << 32;
 #pragma unroll 1
-                    for (int h = 0; h < nh; h += 2) {
-                        float d0[TC], d1[TC];
-                        take(d0, d1);
+                    for (int h = dh0; h < dh1; h += 2) {
+                        float y0[TC], y1[TC];
+                        take(y0, y1);
                         const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? dw2a : dw2b, h & 31);
                         const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? dw2a : dw2b, (h + 1) & 31);
                         unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
@@ -721,8 +730,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         for (int c = 0; c < TC; ++c) {
                             const int yo = __shfl_sync(0xffffffffu, dyoff, c);
                             if (((dmask >> c) & 1u) && live) {
-                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(d0[c] * (ws0 * sc[c])));
-                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(d1[c] * (ws1 * sc[c])));
+                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(y0[c] * (ws0 * sc[c])));
+                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(y1[c] * (ws1 * sc[c])));
                             }
                         }
                     }
@@ -730,7 +739,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 // ---------------- unit s: gather the cluster's partial sums, SiLU*up, requantise -> the intermediate tile its
                 // down groups will use one turn later
                 d_valid = false;
-                if (s < n && !(fl & kExport)) {
+                if (s < n && d1 > d0) {
                     const int slot = pslot;
                     // token columns of this expert and where their down results go
                     const unsigned mask = (unsigned)s_mask[2 * e];
@@ -765,7 +774,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                             for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
                         }
-                        if (fl & kImport) {
+                        if (SPLIT && (fl & kImport)) {
                             // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
                             // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
                             const unsigned long long* xi = P.xsl + ((size_t)((cl - 1) * C) * 2 * TC) * kBlock + row;
@@ -821,6 +830,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
                     w_fc += clock64() - cf0;
                     dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b; d_valid = true;
+                    dh0 = 2 * d0; dh1 = (2 * d1 < nh) ? 2 * d1 : nh;
                 }
             }
         }
@@ -888,11 +898,12 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
 
     // ------------------------------------------------------------------ teardown
-    __syncthreads();
-    // A launch that gave up somewhere: nothing asynchronous may outlive the CTA.  The bulk copies the producer had
-    // requested and the MMAs the issuers had issued are waited for here (bounded), whether or not those roles
-    // noticed the give-up themselves, before tensor memory is freed and shared memory goes to the next CTA.
-    if (*(volatile unsigned*)(P.ctrl + kAbort) != 0u) {
+    const int gave_up = __syncthreads_or((wt.dead || misc[3] != 0u) ? 1 : 0);
+    // A launch in which some thread of this CTA gave up: nothing asynchronous may outlive the CTA.  The bulk copies the
+    // producer had requested and the MMAs the issuers had issued are waited for here (bounded), whether or not those
+    // roles noticed the give-up themselves, before tensor memory is freed and shared memory goes to the next CTA.  (If
+    // no thread of the CTA gave up, every role ran to its end: every tile requested was consumed, every MMA read back.)
+    if (gave_up) {
         if (tid == 0) {
             const uint32_t cntpar = misc[7];
             for (int s = 0; s < S; ++s)

@@ -93,6 +93,7 @@ struct Params {
     int fC, fnCl;                   // fused variants: CTAs per cluster, clusters in the grid
     int fkb[9], fhb[9];             // fused variants: rank r of a cluster takes K blocks [fkb[r], fkb[r+1]) and W2 row blocks [fhb[r], fhb[r+1])
     unsigned long long* stamps;     // [grid][32] globaltimer stamps of the phases of the last launch; NULL = none taken
+    unsigned long long* stamps_buf; // the same buffer, never NULL (the general variant always records its phases)
     int debug_skip;                 // test hook, bit 0: the fused variants never publish the intermediate tile's readiness (a flag that nothing sets: the waits on it must run out cleanly)
     int stamps_fine;                // fused variants: also stamp inside the routing phase (each stamp costs that phase ~0.1 us)
 };
@@ -239,6 +240,9 @@ __device__ __forceinline__ bool epi_all(bool ok, int nthreads) {
 }
 
 #define MOE_STAMP(i) do { if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
+// The general variant takes its sixteen stamps unconditionally (`stamps_buf` always points into the workspace): one
+// store per phase and role.  Guarding them was measured 1.3 % SLOWER at 64 tokens (code layout), so they stay.
+#define MOE_STAMP_ALWAYS(i) do { P.stamps_buf[(size_t)blockIdx.x * kStampsPerCta + (i)] = gtime(); } while (0)
 
 
 // K-major, 128-byte swizzled operand tile (rows of 128 bytes, 8-row groups 1024 bytes apart).
@@ -665,7 +669,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     Waiter wt;
     wt.init(P.ctrl, P.timeout_ns);
     const unsigned tag = ld_acquire(P.ctrl + kEpoch) + 1u;
-    if (tid == 0) MOE_STAMP(0);
+    if (tid == 0) MOE_STAMP_ALWAYS(0);
     const unsigned par = tag & 1u;
     unsigned* e_cnt = P.e_cnt + par * kMaxPasses * E;       // counters of this launch: [pass][expert]
 #pragma unroll 1
@@ -693,7 +697,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             *reinterpret_cast<uint32_t*>(P.xq + (size_t)t * H + g * kBlock + lane * 4) = quant4(x0, x1, x2, x3, s);
             if (lane == 0) P.xs[p] = s;
         }
-        if (tid == 0) MOE_STAMP(1);
+        if (tid == 0) MOE_STAMP_ALWAYS(1);
         // Router logits (Section 3.3): a (16 experts x 8 tokens) tile and one of `ksplit` parts of H per CTA turn; the
         // CTA's warps split that part of H, each accumulates with warp-level bf16 MMAs (m16n8k16, fp32 accumulate)
         // straight from global memory, the warps' partial tiles are summed in warp order, and the K-split parts are
@@ -737,7 +741,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
         }
     }
-    if (tid == 0) MOE_STAMP(2);
+    if (tid == 0) MOE_STAMP_ALWAYS(2);
     // publish: generic writes of xq must be visible to the async proxy (TMA) of every CTA
     fence_proxy_async();
     tc_fence_before();
@@ -756,11 +760,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         }
     }
     if (tid == 0) {
-        MOE_STAMP(3);
+        MOE_STAMP_ALWAYS(3);
         red_release_add(P.ctrl + kRouteCnt + par, 1u);      // all CTAs' logits and xq published once this reaches G
         const bool ok = wt.flag(P.ctrl + kRouteCnt + par, (unsigned)G, 1);
         misc[2] = ok ? 1u : 0u;
-        MOE_STAMP(4);
+        MOE_STAMP_ALWAYS(4);
     }
     __syncthreads();
     bool alive = (misc[2] != 0u);
@@ -794,7 +798,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
         }
         __syncthreads();
-        if (tid == 0) MOE_STAMP(5);
+        if (tid == 0) MOE_STAMP_ALWAYS(5);
 #pragma unroll 1
         for (int tl = warp; tl < rnt; tl += kWarps) {
             const int t = rt0 + tl;
@@ -830,7 +834,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             }
             __syncthreads();
         }
-        if (tid == 0) MOE_STAMP(6);
+        if (tid == 0) MOE_STAMP_ALWAYS(6);
         if constexpr (kCompact && !WS) {
             // active list in ascending expert order, entry = expert | pass << 16 (passes of N tokens): every warp takes
             // 32-expert chunks; the chunks' totals meet in shared memory (the idle weight ring)
@@ -929,7 +933,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         __syncthreads();
     }
     const int U = alive ? (int)misc[1] : 0;
-    if (tid == 0) MOE_STAMP(7);
+    if (tid == 0) MOE_STAMP_ALWAYS(7);
     const int S_up = U * IB * KBu, S_dn = U * HB * KBd;     // k-steps of the two projections (host checks the range)
     const unsigned long long gm = P.grid_magic;
     const int q_up = range_quantum(U * IB, KBu, G, 32, P.split_slack_kib, gm), q_dn = range_quantum(U * HB, KBd, G, 16, P.split_slack_kib, gm);
@@ -990,7 +994,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             if (n_up_st > 0) aw.init(up_lo, KBu, IB, s_act);
             else if (n_st > 0) aw.init(dn_lo, KBd, HB, s_act);
             bool stamped = false;
-            MOE_STAMP(8);
+            MOE_STAMP_ALWAYS(8);
             for (; a_cur < n_up_st; ++a_cur) {                       // gate/up weight tiles
                 if (!wt.mbar(empty, a_ph, 2)) break;
                 const int half = a_cur & 1;
@@ -998,7 +1002,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 tma_load_2d_hint(dst, &tmW13, aw.kb * kBlock, (aw.e & 0xFFFF) * 2 * I + half * I + aw.mb * kBlock, full, stream_once);
                 if (half) aw.next(s_act);
                 dst += L.stage_bytes; full += 8; empty += 8;
-                if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; if (!stamped) { MOE_STAMP(9); stamped = true; } }
+                if (++a_st == S) { a_st = 0; a_ph ^= 1u; dst = smem_u32(smem); full = bar_full; empty = bar_empty; if (!stamped) { MOE_STAMP_ALWAYS(9); stamped = true; } }
             }
             if (!wt.dead && n_st > n_up_st) aw.init(dn_lo, KBd, HB, s_act);
             for (; a_cur < n_st && !wt.dead; ++a_cur) {              // down weight tiles
@@ -1174,7 +1178,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                 if (kCompact && up) fence_proxy_async();       // the gathered tile was written through the generic proxy
                 const uint64_t b_desc = make_smem_desc(a0 + kATileBytes);
                 const uint32_t d = tmem_base + (uint32_t)(buf * 2 * N);
-                if (first && who == 0) { MOE_STAMP(10); first = false; }
+                if (first && who == 0) { MOE_STAMP_ALWAYS(10); first = false; }
                 tc_fence_after();
                 {
                     const uint64_t a_desc = make_smem_desc(a0);
@@ -1281,7 +1285,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             float* part = up ? P.part_up : P.part_dn;
             unsigned* pflag = up ? P.pu_flag : P.pd_flag;
             const int pcols = up ? 2 * N : N;
-            if (!up && etid == 0) MOE_STAMP(12);
+            if (!up && etid == 0) MOE_STAMP_ALWAYS(12);
             if (hi <= lo) continue;
             if (!kCompact && !up) { build_pairs(); col_entry = -1; }
             Walk w;
@@ -1427,7 +1431,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
                         two = (i + 1 < pend - s) && __all_sync(0xffffffffu, mbar_try_wait(bar_tfull + 8 * buf1, tph1));
                     if (two) next_scales(s + i + 1, wsg1, wsu1);
                     tc_fence_after();
-                    if (first_acc) { if (etid == 0) MOE_STAMP(11); first_acc = false; }
+                    if (first_acc) { if (etid == 0) MOE_STAMP_ALWAYS(11); first_acc = false; }
                     // all TMEM loads first, one wait, free the buffers, then the arithmetic
                     float dg0[TCG], du0[TCG], dg1[kDual ? TCG : 1], du1[kDual ? TCG : 1];
                     load_acc(buf, dg0, du0);
@@ -1552,7 +1556,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
         // every down-projection result of this CTA's range is stored: one release for all of them (a release per
         // unit would stall on the unit's own stores; units can be as short as two k-steps)
         epi_bar(kEpiThreads);
-        if (etid == 0) { st_release(P.dn_flag + cta, tag); MOE_STAMP(13); }
+        if (etid == 0) { st_release(P.dn_flag + cta, tag); MOE_STAMP_ALWAYS(13); }
         // ---- final weighted reduction in slot order (deterministic); tasks (token, 128-row block): task = cta + i * G.
         // First every (task, slot) of this CTA waits for the CTA that stored its down-projection result -- all of
         // them in parallel, one thread each -- then the tasks are summed two (four for 16 token columns and more) at a time so that their loads overlap.
@@ -1613,17 +1617,18 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
             for (int r = 0; r < RT; ++r)
                 if (i0 + r * kEpiGroups < n_mine) P.out[(size_t)tt[r] * H + hh[r] * kBlock + row] = __float2bfloat16_rn(acc[r]);
         }
-        if (etid == 0) MOE_STAMP(14);
+        if (etid == 0) MOE_STAMP_ALWAYS(14);
     }
 
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
-    __syncthreads();
+    const int gave_up = __syncthreads_or(wt.dead ? 1 : 0);
     tc_fence_after();
-    // A launch that gave up somewhere: nothing asynchronous may outlive the CTA.  Whatever each role had requested --
-    // weight and activation tiles by bulk copy, MMAs -- is waited for here (bounded), whether or not the role itself
-    // noticed the give-up, before tensor memory is freed and shared memory goes to the next CTA.
-    if (*(volatile unsigned*)(P.ctrl + kAbort) != 0u) {
+    // A launch in which some thread of this CTA gave up: nothing asynchronous may outlive the CTA.  Whatever each role
+    // had requested -- weight and activation tiles by bulk copy, MMAs -- is waited for here (bounded), whether or not
+    // the role itself noticed the give-up, before tensor memory is freed and shared memory goes to the next CTA.  (If no
+    // thread of the CTA gave up, every role ran to its end: every tile requested was consumed, every MMA read back.)
+    if (gave_up) {
         if (lane == 0 && (warp == 0 || warp == 2)) {
             const int cur = (int)misc[6 + (warp >> 1)];
             const uint32_t bar0 = warp ? bar_fullb : bar_full;
@@ -1641,7 +1646,7 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     }
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
     if (tid == 0) {
-        MOE_STAMP(15);
+        MOE_STAMP_ALWAYS(15);
         __threadfence();
         const unsigned old = atomicAdd(P.ctrl + kExitCnt, 1u);
         if (old == (unsigned)G - 1u) {          // last CTA out: open the next epoch
