@@ -42,7 +42,7 @@ constexpr int kFusedTmemBufs = 4;                              // accumulator bu
 constexpr int kFusedIssuers = 3;                               // warps 1..3
 constexpr int kFusedTmemCols = 128;
 constexpr int kFusedThreads = 288;                             // 9 warps
-constexpr int kFusedMaxRows = 4;                               // router rows per CTA: ceil(kMaxExperts / 128)
+constexpr int kFusedMaxRows = 4;          // router rows per CTA: ceil(kMaxExperts / 128)
 
 // ---------------------------------------------------------------------------------------------
 // cluster / distributed-shared-memory wrappers
@@ -609,7 +609,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
         for (int c = 0; c < TC; ++c) sc[c] = 0.f;
         // wait for group g's accumulators, read the first TC columns of both halves of its buffer, hand the buffer back
-        long long w_tf = 0, w_xf = 0, w_fc = 0;
+        long long w_tf = 0, w_xf = 0, w_fc = 0, w_f1 = 0, w_f2 = 0, w_f3 = 0, w_imp = 0, n_f = 0;
         int buf = 0;
         uint32_t bpar = 0u;                                    // parity of the next phase of bar_tfull[buf]
         auto take = [&](float* d0, float* d1) {
@@ -696,7 +696,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     if (d1 > d0) {
                         // park: slot pk & 1 of this CTA's partial buffer, free once every peer has read the item that used it before
                         pslot = pk & 1; pphase = (uint32_t)((pk >> 1) & 1);
-                        if (pk >= 2 && lane == 0) {
+                        if (C > 1 && pk >= 2 && lane == 0) {
                             bool okw = !wt.dead;
                             for (uint32_t i = 1; okw && !mbar_try_wait_cluster(bar_xfree + 8 * pslot, pphase ^ 1u); ++i)
                                 if ((i & 255u) == 0 && wt.expired(30)) okw = false;
@@ -708,7 +708,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                         for (int c = 0; c < TC; ++c) { pp[c * kBlock + row] = accg[c]; pp[(TC + c) * kBlock + row] = accu[c]; }
                         __syncwarp();
-                        if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * pslot, (uint32_t)lane));
+                        if (C > 1 && lane < C) mbar_arrive_cluster(map_to_rank(bar_xfull + 8 * pslot, (uint32_t)lane));
                     }
                     if (s == 0 && etid == 0) MOE_STAMP(9);
                 }
@@ -749,7 +749,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
                     }
                     const long long cf0 = clock64();
-                    {
+                    if (C > 1) {
                         bool okw = !wt.dead;
                         for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, pphase); ++it)
                             if ((it & 255u) == 0 && wt.expired(31)) okw = false;
@@ -762,8 +762,14 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                         for (int c = 0; c < TC; ++c) { sg[c] = 0.f; su[c] = 0.f; }
                         const uint32_t mine = smem_u32(s_part + slot * 2 * TC * kBlock) + (uint32_t)row * 4u;
+                        if (C == 1) {
+                            // a cluster of one: every thread reads back what it parked itself (no barrier, no cluster addressing)
+                            const float* pp = s_part + slot * 2 * TC * kBlock + row;
+#pragma unroll
+                            for (int c = 0; c < TC; ++c) { sg[c] = 0.f + pp[c * kBlock]; su[c] = 0.f + pp[(TC + c) * kBlock]; }
+                        }
 #pragma unroll 1
-                        for (int r = 0; r < C; ++r) {                      // rank order: every CTA of the cluster gets the same sums
+                        for (int r = 0; r < C && C > 1; ++r) {             // rank order: every CTA of the cluster gets the same sums
                             const uint32_t src = map_to_rank(mine, (uint32_t)r);
                             float vg[TC], vu[TC];
 #pragma unroll
@@ -774,6 +780,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                             for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
                         }
+                        const long long ci0 = clock64();
                         if (SPLIT && (fl & kImport)) {
                             // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
                             // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
@@ -796,19 +803,23 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             }
                             if (!okx) misc[3] = 1u;
                         }
+                        w_imp += clock64() - ci0;
                         // SiLU(gate)*up (Section 3.3).  The intermediate tile is outside the bit-exact set: fast exp and divide.
 #pragma unroll
                         for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
                     }
                     __syncwarp();
-                    if (lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
+                    if (C > 1 && lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
                     // 128-wide amax per token column: warp maximum (as an integer: |a| orders like its bits), then across the four warps
 #pragma unroll
                     for (int c = 0; c < TC; ++c) {
                         const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
                         if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
                     }
+                    const long long cb0 = clock64();
+                    w_f1 += cb0 - cf0;
                     if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
+                    w_f2 += clock64() - cb0;
                     const int hslot = dq & 1;
                     ++dq;
                     uint8_t* hq = s_hq + hslot * N * kBlock;
@@ -825,16 +836,18 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             hq[c * kBlock + ((((row >> 4) ^ (c & 7)) << 4) | (row & 15))] = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
                         }
                     }
-                    fence_proxy_async();                                   // generic writes -> the tensor core's reads
+                    w_f3 += clock64() - cf0;
+                    fence_proxy_async_smem();                              // generic shared-memory writes -> the tensor core's reads (not the tagged global stores in flight)
                     epi_bar(kEpiThreads);
                     if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
-                    w_fc += clock64() - cf0;
+                    w_fc += clock64() - cf0; ++n_f;
                     dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b; d_valid = true;
                     dh0 = 2 * d0; dh1 = (2 * d1 < nh) ? 2 * d1 : nh;
                 }
             }
         }
         if (etid == 0) { MOE_STAMP(11); if (P.stamps) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[21] = w_tf; o[22] = w_xf; o[23] = w_fc; } }
+        if (lane == 0 && P.stamps) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[24 + q] = w_f1; o[28 + q] = w_f2; }
     }
 
     // ------------------------------------------------------------------ final weighted reduction (Section 3.2: only this
@@ -852,6 +865,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         int sp = 8;
         while (sp > 1 && sp * tpc > 8) sp >>= 1;
         const int slots = 8 / sp, slot = warp / sp, part = warp - slot * sp;
+        constexpr int kRG = (SPLIT || TC >= 4) ? 3 : 1;                   // groups of eight tagged words a thread polls side by side
         // tasks go to the CTAs from the LAST one down: the first CTAs hold the router rows and the units, and with them
         // the next launch's critical path -- they should be the first to leave (the next launch's CTAs are placed in
         // index order as SMs free up)
@@ -866,23 +880,43 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             const int t = div_small(task, QB), rb = task - t * QB;
             const unsigned long long* base = P.ypl + (size_t)t * NP * H + (size_t)rb * 32 + lane;
             float acc = 0.f;
+            // kRG groups of eight tagged words per thread and chunk.  The groups are polled in turn WITHOUT waiting for one
+            // to complete before the next is looked at: by the time the slowest producer's words arrive, every other word
+            // has been taken, and only the groups that still miss something cost another round trip.  (Waiting group by
+            // group cost a round trip per group after the last arrival.)  Values are kept, summed in fixed order.
 #pragma unroll 1
-            for (int p0 = part; p0 < NP && ok && valid; p0 += sp * 8) {   // eight words in flight per thread
-                unsigned long long v[8];
-                unsigned pending = 0u;
+            for (int p0 = part; p0 < NP && ok && valid; p0 += sp * 8 * kRG) {
+                float val[kRG][8];
+                unsigned pend[kRG];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) if (p0 + sp * j < NP) pending |= 1u << j;
-                for (uint32_t it = 1; pending; ++it) {
+                for (int g = 0; g < kRG; ++g) {
+                    pend[g] = 0u;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) if (pending & (1u << j)) v[j] = ld_relaxed_u64(base + (size_t)(p0 + sp * j) * H);
+                    for (int j = 0; j < 8; ++j) { val[g][j] = 0.f; if (p0 + sp * (g * 8 + j) < NP) pend[g] |= 1u << j; }
+                }
+                for (uint32_t it = 1;; ++it) {
+                    unsigned any = 0u;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) if ((pending & (1u << j)) && (unsigned)(v[j] >> 32) == tag) pending &= ~(1u << j);
-                    if (pending && (it & 63u) == 0 && wt.expired(33)) { ok = false; break; }
+                    for (int g = 0; g < kRG; ++g) {
+                        if (pend[g]) {
+                            unsigned long long v[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) if (pend[g] & (1u << j)) v[j] = ld_relaxed_u64(base + (size_t)(p0 + sp * (g * 8 + j)) * H);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if ((pend[g] & (1u << j)) && (unsigned)(v[j] >> 32) == tag) { pend[g] &= ~(1u << j); val[g][j] = __uint_as_float((unsigned)v[j]); }
+                            any |= pend[g];
+                        }
+                    }
+                    if (!any) break;
+                    if ((it & 63u) == 0 && wt.expired(33)) { ok = false; break; }
                 }
                 if (!ok) break;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (p0 + sp * j < NP) acc = fmaf(s_w[t * K + div_small(p0 + sp * j, IB)], __uint_as_float((unsigned)v[j]), acc);
+                for (int g = 0; g < kRG; ++g)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (p0 + sp * (g * 8 + j) < NP) acc = fmaf(s_w[t * K + div_small(p0 + sp * (g * 8 + j), IB)], val[g][j], acc);
             }
             s_sum[warp * 32 + lane] = acc;
             ok = named_bar_and(2, kMain, ok);
