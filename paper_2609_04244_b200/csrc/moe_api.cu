@@ -185,15 +185,15 @@ struct moe_plan {
     }
     // The library's choice, by the length of the weight stream: tiles per CTA at the expected number of distinct experts.
     // The fused variant has the shorter latency chain (routing, hand-over, reduction) but its accumulator warps work
-    // per group and its units go to clusters in whole pieces; the general variant streams longer runs at a higher rate.
-    // Measured crossover on the nine benchmark shapes (1-8 tokens): about 85 tiles per CTA; about 160 where a unit's
+    // per group; the general variant streams longer runs at a higher rate.
+    // Measured crossover on the nine benchmark shapes (1-8 tokens): about 120 tiles per CTA; about 160 where a unit's
     // down projection is at most two K blocks (there the general variant's per-unit work weighs most) and for a single
     // token.
     bool fused(int T) const {
         if (fused_mode == 0 || !fused_possible(T)) return false;
         if (fused_mode == 1) return true;
         const double tiles = 3.0 * expected_experts(T) * (I / 128) * (H / 128) / sms;
-        return tiles <= 85.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
+        return tiles <= 120.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
     }
 
     // Default depth of the stage ring when the knob is 0.  Measured (config 2 and the paper's shapes,

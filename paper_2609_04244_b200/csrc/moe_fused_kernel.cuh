@@ -275,7 +275,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             *reinterpret_cast<uint32_t*>(P.xq + (size_t)t * H + g * kBlock + lane * 4) = quant4(x0, x1, x2, x3, s);
             if (lane == 0) P.xs[p] = s;
         }
-        fence_proxy_async();                                    // generic writes of xq -> the async proxy (bulk-tensor copies) of every CTA
+        // generic writes of xq -> the async proxy (bulk-tensor copies) of every CTA.  By every warp, also those that wrote
+        // nothing of xq: the fence pushes out the thread's stores in flight, the router logits just published among them
+        // (measured: without it the step is 1-1.5 us longer -- the logits reach the other CTAs later).
+        fence_proxy_async();
         named_bar_arrive(3, kFusedThreads);                     // hand over to the housekeeping warp, do not wait for it
     } else {
         // ---------------------------------------------------------- housekeeping warp: everything that costs L2 round
@@ -609,7 +612,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
         for (int c = 0; c < TC; ++c) sc[c] = 0.f;
         // wait for group g's accumulators, read the first TC columns of both halves of its buffer, hand the buffer back
-        long long w_tf = 0, w_xf = 0, w_fc = 0, w_f1 = 0, w_f2 = 0, w_f3 = 0, w_imp = 0, n_f = 0;
+        long long w_tf = 0, w_xf = 0, w_fc = 0;
         int buf = 0;
         uint32_t bpar = 0u;                                    // parity of the next phase of bar_tfull[buf]
         auto take = [&](float* d0, float* d1) {
@@ -712,142 +715,157 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     }
                     if (s == 0 && etid == 0) MOE_STAMP(9);
                 }
-                // ---------------- unit s-1: its down groups (the intermediate tile was made at the end of the previous turn, long
-                // before the issuers got here: no hand-over wait on the weight stream's path), scaled and stored as the tagged
-                // partials of (token, slot, ib): the final reduction polls these words themselves
-                if (s >= 1 && d_valid) {
-                    const unsigned long long tagw = (unsigned long long)tag << 32;
+                // ---------------- two steps, normally in this order:
+                //   down(s-1): the down groups of unit s-1 (its intermediate tile was made at the end of the previous turn, long
+                //     before the issuers got here: no hand-over wait on the weight stream's path), scaled and stored as the
+                //     tagged partials of (token, slot, ib): the final reduction polls these words themselves;
+                //   F(s): gather the cluster's partial sums of unit s, SiLU*up, requantise -> the intermediate tile its down
+                //     groups will use one turn later.
+                // In the LAST turn with gate/up groups nothing follows that could hide F(s) -- the issuers go from the down
+                // groups of s-1 straight to those of s -- so there F(s) comes first, while the down MMAs of s-1 run.
+                const bool f_first = (s == n - 1);
+                bool failed = false, n_valid = false;
+                float nsc[TC];
+                unsigned nmask = 0u;
+                int nyoff = 0;
+#pragma unroll
+                for (int c = 0; c < TC; ++c) nsc[c] = 0.f;
 #pragma unroll 1
-                    for (int h = dh0; h < dh1; h += 2) {
-                        float y0[TC], y1[TC];
-                        take(y0, y1);
-                        const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? dw2a : dw2b, h & 31);
-                        const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? dw2a : dw2b, (h + 1) & 31);
-                        unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
-                        const bool live = (misc[3] == 0u) && !wt.dead;     // never publish a result that was not computed
-                        const bool two = (h + 1 < nh);
+                for (int step = 0; step < 2; ++step) {
+                if ((step == 0) != f_first) {
+                    if (s >= 1 && d_valid) {
+                        const unsigned long long tagw = (unsigned long long)tag << 32;
+#pragma unroll 1
+                        for (int h = dh0; h < dh1; h += 2) {
+                            float y0[TC], y1[TC];
+                            take(y0, y1);
+                            const float ws0 = __shfl_sync(0xffffffffu, (h < 32) ? dw2a : dw2b, h & 31);
+                            const float ws1 = __shfl_sync(0xffffffffu, (h + 1 < 32) ? dw2a : dw2b, (h + 1) & 31);
+                            unsigned long long* yrow = P.ypl + (size_t)(hb_lo + h) * kBlock + row;
+                            const bool live = (misc[3] == 0u) && !wt.dead;     // never publish a result that was not computed
+                            const bool two = (h + 1 < nh);
+#pragma unroll
+                            for (int c = 0; c < TC; ++c) {
+                                const int yo = __shfl_sync(0xffffffffu, dyoff, c);
+                                if (((dmask >> c) & 1u) && live) {
+                                    st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(y0[c] * (ws0 * sc[c])));
+                                    if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(y1[c] * (ws1 * sc[c])));
+                                }
+                            }
+                        }
+                    }
+                } else {
+                    // ---------------- unit s: gather the cluster's partial sums, SiLU*up, requantise -> the intermediate tile its
+                    // down groups will use one turn later
+                    if (s < n && d1 > d0) {
+                        const int slot = pslot;
+                        // token columns of this expert and where their down results go
+                        const unsigned mask = (unsigned)s_mask[2 * e];
+                        int yoff_lane = 0;
+                        if (lane < TC && ((mask >> lane) & 1u)) {
+                            const unsigned pr = s_pair[s_poff[e] + __popc(mask & ((1u << lane) - 1u))];
+                            yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
+                        }
+                        const long long cf0 = clock64();
+                        if (C > 1) {
+                            bool okw = !wt.dead;
+                            for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, pphase); ++it)
+                                if ((it & 255u) == 0 && wt.expired(31)) okw = false;
+                            if (!okw) misc[3] = 1u;
+                        }
+                        w_xf += clock64() - cf0;
+                        float a[TC];
+                        {
+                            float sg[TC], su[TC];
+#pragma unroll
+                            for (int c = 0; c < TC; ++c) { sg[c] = 0.f; su[c] = 0.f; }
+                            const uint32_t mine = smem_u32(s_part + slot * 2 * TC * kBlock) + (uint32_t)row * 4u;
+                            if (C == 1) {
+                                // a cluster of one: every thread reads back what it parked itself (no barrier, no cluster addressing)
+                                const float* pp = s_part + slot * 2 * TC * kBlock + row;
+#pragma unroll
+                                for (int c = 0; c < TC; ++c) { sg[c] = 0.f + pp[c * kBlock]; su[c] = 0.f + pp[(TC + c) * kBlock]; }
+                            }
+#pragma unroll 1
+                            for (int r = 0; r < C && C > 1; ++r) {             // rank order: every CTA of the cluster gets the same sums
+                                const uint32_t src = map_to_rank(mine, (uint32_t)r);
+                                float vg[TC], vu[TC];
+#pragma unroll
+                                for (int c = 0; c < TC; ++c) {                 // (columns of tokens not routed to this expert are dropped below)
+                                    vg[c] = ld_cluster_f32(src + (uint32_t)(c * kBlock * 4));
+                                    vu[c] = ld_cluster_f32(src + (uint32_t)((TC + c) * kBlock * 4));
+                                }
+#pragma unroll
+                                for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
+                            }
+                            if (SPLIT && (fl & kImport)) {
+                                // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
+                                // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
+                                const unsigned long long* xi = P.xsl + ((size_t)((cl - 1) * C) * 2 * TC) * kBlock + row;
+                                bool okx = !wt.dead;
+#pragma unroll 1
+                                for (int r = 0; r < C && okx; ++r) {
+                                    unsigned long long v[2 * TC];
+                                    unsigned pending = (1u << (2 * TC)) - 1u;
+                                    for (uint32_t it = 1; pending; ++it) {
+#pragma unroll
+                                        for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
+#pragma unroll
+                                        for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
+                                        if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                    }
+                                    if (!okx) break;
+#pragma unroll
+                                    for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
+                                }
+                                if (!okx) misc[3] = 1u;
+                            }
+                            // SiLU(gate)*up (Section 3.3).  The intermediate tile is outside the bit-exact set: fast exp and divide.
+#pragma unroll
+                            for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
+                        }
+                        __syncwarp();
+                        if (C > 1 && lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
+                        // 128-wide amax per token column: warp maximum (as an integer: |a| orders like its bits), then across the four warps
 #pragma unroll
                         for (int c = 0; c < TC; ++c) {
-                            const int yo = __shfl_sync(0xffffffffu, dyoff, c);
-                            if (((dmask >> c) & 1u) && live) {
-                                st_relaxed_u64(yrow + (size_t)yo, tagw | (unsigned long long)__float_as_uint(y0[c] * (ws0 * sc[c])));
-                                if (two) st_relaxed_u64(yrow + (size_t)yo + kBlock, tagw | (unsigned long long)__float_as_uint(y1[c] * (ws1 * sc[c])));
+                            const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
+                            if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
+                        }
+                        if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; failed = true; break; }
+                        const int hslot = dq & 1;
+                        ++dq;
+                        uint8_t* hq = s_hq + hslot * N * kBlock;
+#pragma unroll
+                        for (int c = 0; c < TC; ++c) {
+                            const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
+                            nsc[c] = fmaxf(amax, 1e-10f) * (1.0f / 448.0f);     // (the intermediate tile's scale is outside the bit-exact set)
+                        }
+#pragma unroll
+                        for (int c = 0; c < TC; ++c) {
+                            if ((mask >> c) & 1u) {
+                                const float2 v = make_float2(a[c] * __fdividef(1.0f, nsc[c]), 0.f);
+                                // K-major, 128-byte swizzled B tile: row = token column, 16-byte chunk (row >> 4) sits at chunk ^ (column & 7)
+                                hq[c * kBlock + ((((row >> 4) ^ (c & 7)) << 4) | (row & 15))] = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
                             }
                         }
+                        fence_proxy_async_smem();                              // generic shared-memory writes -> the tensor core's reads (not the tagged global stores in flight)
+                        epi_bar(kEpiThreads);
+                        if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
+                        w_fc += clock64() - cf0;
+                        nmask = mask; nyoff = yoff_lane; n_valid = true;
                     }
                 }
-                // ---------------- unit s: gather the cluster's partial sums, SiLU*up, requantise -> the intermediate tile its
-                // down groups will use one turn later
-                d_valid = false;
-                if (s < n && d1 > d0) {
-                    const int slot = pslot;
-                    // token columns of this expert and where their down results go
-                    const unsigned mask = (unsigned)s_mask[2 * e];
-                    int yoff_lane = 0;
-                    if (lane < TC && ((mask >> lane) & 1u)) {
-                        const unsigned pr = s_pair[s_poff[e] + __popc(mask & ((1u << lane) - 1u))];
-                        yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
-                    }
-                    const long long cf0 = clock64();
-                    if (C > 1) {
-                        bool okw = !wt.dead;
-                        for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, pphase); ++it)
-                            if ((it & 255u) == 0 && wt.expired(31)) okw = false;
-                        if (!okw) misc[3] = 1u;
-                    }
-                    w_xf += clock64() - cf0;
-                    float a[TC];
-                    {
-                        float sg[TC], su[TC];
-#pragma unroll
-                        for (int c = 0; c < TC; ++c) { sg[c] = 0.f; su[c] = 0.f; }
-                        const uint32_t mine = smem_u32(s_part + slot * 2 * TC * kBlock) + (uint32_t)row * 4u;
-                        if (C == 1) {
-                            // a cluster of one: every thread reads back what it parked itself (no barrier, no cluster addressing)
-                            const float* pp = s_part + slot * 2 * TC * kBlock + row;
-#pragma unroll
-                            for (int c = 0; c < TC; ++c) { sg[c] = 0.f + pp[c * kBlock]; su[c] = 0.f + pp[(TC + c) * kBlock]; }
-                        }
-#pragma unroll 1
-                        for (int r = 0; r < C && C > 1; ++r) {             // rank order: every CTA of the cluster gets the same sums
-                            const uint32_t src = map_to_rank(mine, (uint32_t)r);
-                            float vg[TC], vu[TC];
-#pragma unroll
-                            for (int c = 0; c < TC; ++c) {                 // (columns of tokens not routed to this expert are dropped below)
-                                vg[c] = ld_cluster_f32(src + (uint32_t)(c * kBlock * 4));
-                                vu[c] = ld_cluster_f32(src + (uint32_t)((TC + c) * kBlock * 4));
-                            }
-#pragma unroll
-                            for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
-                        }
-                        const long long ci0 = clock64();
-                        if (SPLIT && (fl & kImport)) {
-                            // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
-                            // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
-                            const unsigned long long* xi = P.xsl + ((size_t)((cl - 1) * C) * 2 * TC) * kBlock + row;
-                            bool okx = !wt.dead;
-#pragma unroll 1
-                            for (int r = 0; r < C && okx; ++r) {
-                                unsigned long long v[2 * TC];
-                                unsigned pending = (1u << (2 * TC)) - 1u;
-                                for (uint32_t it = 1; pending; ++it) {
-#pragma unroll
-                                    for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
-#pragma unroll
-                                    for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
-                                    if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
-                                }
-                                if (!okx) break;
-#pragma unroll
-                                for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
-                            }
-                            if (!okx) misc[3] = 1u;
-                        }
-                        w_imp += clock64() - ci0;
-                        // SiLU(gate)*up (Section 3.3).  The intermediate tile is outside the bit-exact set: fast exp and divide.
-#pragma unroll
-                        for (int c = 0; c < TC; ++c) a[c] = ((mask >> c) & 1u) ? __fdividef(sg[c], 1.0f + __expf(-sg[c])) * su[c] : 0.f;
-                    }
-                    __syncwarp();
-                    if (C > 1 && lane < C) mbar_arrive_cluster(map_to_rank(bar_xfree + 8 * slot, (uint32_t)lane));   // my reads of every peer's slot are done
-                    // 128-wide amax per token column: warp maximum (as an integer: |a| orders like its bits), then across the four warps
-#pragma unroll
-                    for (int c = 0; c < TC; ++c) {
-                        const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
-                        if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
-                    }
-                    const long long cb0 = clock64();
-                    w_f1 += cb0 - cf0;
-                    if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; break; }
-                    w_f2 += clock64() - cb0;
-                    const int hslot = dq & 1;
-                    ++dq;
-                    uint8_t* hq = s_hq + hslot * N * kBlock;
-#pragma unroll
-                    for (int c = 0; c < TC; ++c) {
-                        const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
-                        sc[c] = fmaxf(amax, 1e-10f) * (1.0f / 448.0f);      // (the intermediate tile's scale is outside the bit-exact set)
-                    }
-#pragma unroll
-                    for (int c = 0; c < TC; ++c) {
-                        if ((mask >> c) & 1u) {
-                            const float2 v = make_float2(a[c] * __fdividef(1.0f, sc[c]), 0.f);
-                            // K-major, 128-byte swizzled B tile: row = token column, 16-byte chunk (row >> 4) sits at chunk ^ (column & 7)
-                            hq[c * kBlock + ((((row >> 4) ^ (c & 7)) << 4) | (row & 15))] = (uint8_t)(__nv_cvt_float2_to_fp8x2(v, __NV_SATFINITE, __NV_E4M3) & 0xFF);
-                        }
-                    }
-                    w_f3 += clock64() - cf0;
-                    fence_proxy_async_smem();                              // generic shared-memory writes -> the tensor core's reads (not the tagged global stores in flight)
-                    epi_bar(kEpiThreads);
-                    if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
-                    w_fc += clock64() - cf0; ++n_f;
-                    dmask = mask; dyoff = yoff_lane; dw2a = w2a; dw2b = w2b; d_valid = true;
-                    dh0 = 2 * d0; dh1 = (2 * d1 < nh) ? 2 * d1 : nh;
                 }
+                if (failed) break;
+                // unit s moves into its down phase
+#pragma unroll
+                for (int c = 0; c < TC; ++c) sc[c] = nsc[c];
+                dmask = nmask; dyoff = nyoff; dw2a = w2a; dw2b = w2b; d_valid = n_valid;
+                dh0 = 2 * d0; dh1 = (2 * d1 < nh) ? 2 * d1 : nh;
             }
         }
         if (etid == 0) { MOE_STAMP(11); if (P.stamps) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[21] = w_tf; o[22] = w_xf; o[23] = w_fc; } }
-        if (lane == 0 && P.stamps) { unsigned long long* o = P.stamps + (size_t)blockIdx.x * kStampsPerCta; o[24 + q] = w_f1; o[28 + q] = w_f2; }
     }
 
     // ------------------------------------------------------------------ final weighted reduction (Section 3.2: only this
