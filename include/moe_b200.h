@@ -218,9 +218,11 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              tiles at the expected number of distinct experts.  MOE_ERR_OCCUPANCY if the device cannot
  *                              hold such clusters.  With MOE_KNOB_STAGES = 0 the fused variant takes as many stages as
  *                              leave half of the SM's shared memory to the next launch's CTA.
- *   MOE_KNOB_SPLIT_UNITS       (plan-wide) fused-unit variant with more units than clusters: 1 (default) = the list of all
- *                              accumulation groups is cut into equal ranges, one per cluster, so a unit's gate/up groups may
- *                              be shared by two clusters (the first exports its partial sums to the second); 0 = units are
+ *   MOE_KNOB_SPLIT_UNITS       (plan-wide) fused-unit variant: 1 (default) = where a step has more units than clusters, the
+ *                              list of all accumulation groups is cut into equal ranges, one per cluster; a range may begin
+ *                              and end anywhere inside a unit (clusters that share a unit exchange partial sums); 2 = the
+ *                              same also where the step has fewer units than clusters (ranges shorter than a unit; measured
+ *                              slower than whole units on every benchmark shape, kept for experiments); 0 = units are always
  *                              dealt to clusters whole, round-robin
  *   MOE_KNOB_HOST_DIRECT       (plan-wide) moe_forward_host with PINNED host buffers of at most 64 KiB: bit 0 (default on) = the
  *                              kernel writes the result straight into out_host, bit 1 = it reads hidden_host in place; the

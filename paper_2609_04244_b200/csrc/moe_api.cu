@@ -148,7 +148,7 @@ struct moe_plan {
         // fused variants: tagged router logits, and one down-projection partial per (token, slot, intermediate block)
         L.ll = o;       o += with_fused ? align_up((size_t)Tc * E * 8, 256) : 0;
         L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 8, 256) : 0;
-        L.xsl = o;      o += with_fused ? align_up((size_t)G * 2 * 8 * 128 * 8, 256) : 0;     // partial sums exported between clusters
+        L.xsl = o;      o += with_fused ? align_up((size_t)G * 2 * 2 * 8 * 128 * 8, 256) : 0; // partial sums exported between clusters: [CTA][2 pieces][2 x 8 columns][128 rows]
         L.total = o;
         return L;
     }
@@ -398,7 +398,7 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         // units are shared between clusters only where the step can have more units than clusters at all: T tokens select
         // at most min(E, T * top_k) experts (the instantiations without that code are smaller and faster)
         const int max_units = (T * p->K < p->E ? T * p->K : p->E) * (p->I / 128);
-        P.fsplit = (p->split_units && KB % C == 0 && max_units > P.fnCl) ? 1 : 0;
+        P.fsplit = (p->split_units && KB % C == 0 && (max_units > P.fnCl || p->split_units == 2)) ? p->split_units : 0;
         P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
         for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
@@ -489,7 +489,8 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->cluster_knob[t] = value;
             return MOE_OK;
         case MOE_KNOB_SPLIT_UNITS:
-            plan->split_units = value != 0;
+            if (value < 0 || value > 2) return fail(MOE_ERR_ARG, "split_units must be 0, 1 or 2");
+            plan->split_units = value;
             return MOE_OK;
         case MOE_KNOB_HOST_DIRECT:
             if (value < 0 || value > 3) return fail(MOE_ERR_ARG, "host-direct must be 0..3");

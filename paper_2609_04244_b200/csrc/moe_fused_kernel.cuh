@@ -413,46 +413,59 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     const int kb_lo = P.fkb[rank], kb_hi = P.fkb[rank + 1], nk = kb_hi - kb_lo;
     const int hb_lo = P.fhb[rank], hb_hi = P.fhb[rank + 1], nh = hb_hi - hb_lo;
     const int ngd = (nh + 1) >> 1;                               // down groups per unit
-    // Which units this cluster works on.  Fewer units than clusters (or a split the shape does not allow): whole units,
-    // dealt round-robin.  Otherwise the list of all groups -- per unit nk gate/up groups, then ngd down groups -- is cut
-    // into equal contiguous ranges, one per cluster (Section 3.2 gives each expert a group of CTAs; here a range may
-    // end anywhere inside a unit).  A cluster then has, in the order it works on them: the HEAD piece of the unit its
-    // range ends in (gate/up groups [0, g1) and, if the cut lies beyond them, down groups [0, d1); its partial sums are
-    // exported as tagged words for the next cluster right after its gate/up groups, first thing, so they have long
-    // arrived when they are needed), its whole units, and last the TAIL piece of the unit its range starts in (gate/up
-    // groups [g0, nk) -- none if the cut lies beyond them --, the previous cluster's partial sums imported, then the
-    // unit's down groups [d0, ngd)).  When a unit's down groups are shared, both clusters hold its complete sums (one
-    // computed them, one imported them) and both make the intermediate tile, with the same arithmetic in the same order.
-    const bool split = SPLIT && (P.fsplit != 0) && (nU > nCl);
-    int n, first_whole = 0, nw = 0, head_u = -1, head_g1 = 0, head_d1 = 0, tail_u = -1, tail_g0 = 0, tail_d0 = 0;
+    // Which units this cluster works on.  Either whole units, dealt round-robin, or -- where the host allows it and the
+    // step has more units than clusters (or the host asks for it regardless: few crowded experts leave most clusters
+    // without a unit) -- the list of all groups, per unit nk gate/up groups followed by ngd down groups, is cut into
+    // equal contiguous ranges, one per cluster (Section 3.2 gives each expert a group of CTAs; here a range may begin and
+    // end anywhere inside a unit, and be shorter than a unit).  A cluster's range covers the units ua..ue, the first
+    // from position xa and the last up to position xe of their Wg groups.  In the order the cluster works on them:
+    //   HEAD piece  unit ue, groups [0, xe)   if the range ends inside a unit other than its first: exports, never imports
+    //   whole units
+    //   TAIL piece  unit ua, groups [xa, ..)  if the range starts inside a unit (or lies inside a single one)
+    // A piece with gate/up groups whose cluster does not hold all of the unit's down groups EXPORTS its partial sums as
+    // tagged words right after those groups; a piece with down groups that lacks some of the unit's gate/up groups
+    // IMPORTS the partial sums of every other cluster that has some, and adds all of them in cluster order (so every
+    // cluster that makes the unit's intermediate tile makes the same one).  Exports happen before anything the cluster
+    // imports (head piece first, tail piece last; inside a piece the export precedes the import), and a cluster imports
+    // only from clusters below it: nobody waits in a circle, and nobody's export waits for an import.
+    const int Wg = nk + ngd, total_g = nU * Wg;
+    const bool split = SPLIT && (P.fsplit != 0) && (nU > nCl || P.fsplit == 2);
+    auto cut = [&](int c) -> int { return (c >= nCl) ? total_g : (int)div_grid((unsigned)c * (unsigned)total_g, P.grid_magic); };
+    int n, first_whole = 0, nw = 0, hs = 0, ua = 0, xa = 0, ue = 0, xe = 0;
+    bool has_tail = false;
     if (split) {
-        const int Wg = nk + ngd, total = nU * Wg;
-        auto cut = [&](int c) -> int { return (int)div_grid((unsigned)c * (unsigned)total, P.grid_magic); };
-        const int lo = cut(cl), hi = (cl + 1 == nCl) ? total : cut(cl + 1);
-        const int ua = lo / Wg, xa = lo - ua * Wg, ub = hi / Wg, xb = hi - ub * Wg;
-        if (xa > 0) { tail_u = ua; tail_g0 = xa < nk ? xa : nk; tail_d0 = xa > nk ? xa - nk : 0; }
-        if (xb > 0) { head_u = ub; head_g1 = xb < nk ? xb : nk; head_d1 = xb > nk ? xb - nk : 0; }
-        first_whole = ua + (xa > 0 ? 1 : 0);
-        nw = ub - first_whole;
-        if (nw < 0) nw = 0;
-        n = nw + (head_u >= 0 ? 1 : 0) + (tail_u >= 0 ? 1 : 0);
+        const int lo = cut(cl), hi = cut(cl + 1);
+        n = 0;
+        if (hi > lo) {
+            ua = lo / Wg; xa = lo - ua * Wg;
+            ue = (hi - 1) / Wg; xe = hi - ue * Wg;                       // 0 < xe <= Wg
+            hs = (ue > ua && xe < Wg) ? 1 : 0;
+            has_tail = (xa > 0) || (ua == ue && xe < Wg);
+            first_whole = ua + (xa > 0 ? 1 : 0);
+            nw = ((xe < Wg) ? ue - 1 : ue) - first_whole + 1;
+            if (nw < 0) nw = 0;
+            n = hs + nw + (has_tail ? 1 : 0);
+        }
     } else {
         n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units cl, cl + nCl, ... (grid_magic divides by the cluster count)
     }
-    // item s of this cluster, in working order: expert, intermediate block, gate/up groups [g0, g1) of this CTA's K
-    // blocks, down groups [d0, d1) of this CTA's row blocks (none: the item ends with its partial sums), and what
-    // happens to its partial sums: kExport (head piece: stored for the next cluster), kImport (tail piece: the previous
-    // cluster's are added)
+    // item s of this cluster, in working order: unit u = (expert e, intermediate block ib), gate/up groups [g0, g1) of
+    // this CTA's K blocks, down groups [d0, d1) of this CTA's row blocks (none: the item ends with its partial sums),
+    // and whether its partial sums are exported and/or other clusters' imported
     constexpr int kExport = 1, kImport = 2;
-    auto item_of = [&](int s, int& e, int& ib, int& g0, int& g1, int& d0, int& d1) -> int {
-        int u, fl = 0;
+    auto item_of = [&](int s, int& u, int& e, int& ib, int& g0, int& g1, int& d0, int& d1) -> int {
+        int fl = 0;
         g0 = 0; g1 = nk; d0 = 0; d1 = ngd;
         if (!SPLIT || !split) u = cl + s * nCl;
         else {
-            const int hs = (head_u >= 0) ? 1 : 0;
-            if (s < hs) { u = head_u; g1 = head_g1; d1 = head_d1; fl = kExport; }
+            int x0 = 0, x1 = Wg;
+            if (s < hs) { u = ue; x1 = xe; }
             else if (s - hs < nw) u = first_whole + s - hs;
-            else { u = tail_u; g0 = tail_g0; d0 = tail_d0; fl = kImport; }
+            else { u = ua; x0 = xa; x1 = (ua == ue) ? xe : Wg; }
+            g0 = x0 < nk ? x0 : nk; g1 = x1 < nk ? x1 : nk;
+            d0 = x0 > nk ? x0 - nk : 0; d1 = x1 > nk ? x1 - nk : 0;
+            if (g1 > g0 && !(d0 == 0 && d1 == ngd)) fl |= kExport;           // somebody else has down groups of this unit
+            if (d1 > d0 && !(g0 == 0 && g1 == nk)) fl |= kImport;            // somebody else has gate/up groups of it
         }
         const int a = div_small(u, IB);
         ib = u - a * IB;
@@ -461,8 +474,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     };
     int Ntot = 0;                                                // weight tiles of this CTA
     for (int s = 0; s < n; ++s) {
-        int e, ib, g0, g1, d0, d1;
-        item_of(s, e, ib, g0, g1, d0, d1);
+        int u, e, ib, g0, g1, d0, d1;
+        item_of(s, u, e, ib, g0, g1, d0, d1);
         Ntot += 2 * (g1 - g0) + ((2 * d1 < nh ? 2 * d1 : nh) - 2 * d0);     // (a unit's last down group may be a single tile)
     }
 
@@ -504,15 +517,15 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             MOE_STAMP(6);
             for (int s = 0; s <= n && !wt.dead; ++s) {
                 if (s < n) {
-                    int e, ib, g0, g1, d0, d1;
-                    item_of(s, e, ib, g0, g1, d0, d1);
+                    int u, e, ib, g0, g1, d0, d1;
+                    item_of(s, u, e, ib, g0, g1, d0, d1);
                     const int yg = e * 2 * I + ib * kBlock;
                     for (int k = kb_lo + g0; k < kb_lo + g1; ++k)
                         if (!put(&tmW13, k * kBlock, yg, k * kBlock, yg + I, 2, k)) break;
                 }
                 if (s >= 1 && !wt.dead) {
-                    int e, ib, g0, g1, d0, d1;
-                    item_of(s - 1, e, ib, g0, g1, d0, d1);
+                    int u, e, ib, g0, g1, d0, d1;
+                    item_of(s - 1, u, e, ib, g0, g1, d0, d1);
                     for (int h = hb_lo + 2 * d0; h < hb_hi && h < hb_lo + 2 * d1; h += 2)
                         if (!put(&tmW2, ib * kBlock, e * H + h * kBlock, ib * kBlock, e * H + (h + 1) * kBlock, (h + 1 < hb_hi) ? 2 : 1, -1)) break;
                 }
@@ -581,14 +594,14 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             int dq = 0;                                            // items with down groups so far: slot and phase of the intermediate tile
             for (int s = 0; s <= n && !wt.dead; ++s) {
                 if (s < n) {
-                    int e, ib, g0, g1, d0, d1;
-                    item_of(s, e, ib, g0, g1, d0, d1);
+                    int u, e, ib, g0, g1, d0, d1;
+                    item_of(s, u, e, ib, g0, g1, d0, d1);
                     for (int k = g0; k < g1; ++k)
                         if (!group(2, 0u)) break;
                 }
                 if (s >= 1 && !wt.dead) {
-                    int e, ib, g0, g1, d0, d1;
-                    item_of(s - 1, e, ib, g0, g1, d0, d1);
+                    int u, e, ib, g0, g1, d0, d1;
+                    item_of(s - 1, u, e, ib, g0, g1, d0, d1);
                     if (d1 <= d0) continue;                                  // (a head piece that ends with its partial sums)
                     const int slot = dq & 1;
                     // the intermediate tile of the item is in shared memory (written by the accumulator warps)
@@ -634,8 +647,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         float nwg0 = 0.f, nwu0 = 0.f, nwg1 = 0.f, nwu1 = 0.f, nw2a = 0.f, nw2b = 0.f;
         auto fetch_scales = [&](int s) {
             if (s >= n) return;
-            int e, ib, g0, g1, d0, d1;
-            item_of(s, e, ib, g0, g1, d0, d1);
+            int u, e, ib, g0, g1, d0, d1;
+            item_of(s, u, e, ib, g0, g1, d0, d1);
             const float* g13 = P.W13s + ((size_t)e * 2 * IB + ib) * KBu + kb_lo;
             const float* u13 = P.W13s + ((size_t)e * 2 * IB + IB + ib) * KBu + kb_lo;
             const float* w2 = P.W2s + ((size_t)e * HB + hb_lo) * IB + ib;
@@ -656,8 +669,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             int pslot = 0;
             uint32_t pphase = 0u;
             for (int s = 0; s <= n; ++s) {
-                int e = 0, ib = 0, g0 = 0, g1 = 0, d0 = 0, d1 = 0, fl = 0;
-                if (s < n) fl = item_of(s, e, ib, g0, g1, d0, d1);
+                int u = 0, e = 0, ib = 0, g0 = 0, g1 = 0, d0 = 0, d1 = 0, fl = 0;
+                if (s < n) fl = item_of(s, u, e, ib, g0, g1, d0, d1);
                 // ---------------- gate/up groups of item s: accumulate, then park the partial sums for the cluster
                 if (s < n) {
                     const float wg0 = nwg0, wu0 = nwu0;
@@ -683,9 +696,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         }
                     }
                     if (SPLIT && (fl & kExport)) {
-                        // head piece: this CTA's partial sums go to the next cluster as tagged words (it adds them to its own
-                        // at the very end of its range: they are there long before)
-                        unsigned long long* xo = P.xsl + ((size_t)(cl * C + rank) * 2 * TC) * kBlock + row;
+                        // this CTA's partial sums go to the clusters that hold down groups of the unit, as tagged words (they add
+                        // them at the very end of their ranges: they are there long before).  A cluster exports at most two
+                        // pieces: the one of its first unit (slot 0) and the one of its last (slot 1).
+                        unsigned long long* xo = P.xsl + ((size_t)((cl * 2 + (u == ua ? 0 : 1)) * C + rank) * 2 * TC) * kBlock + row;
                         const unsigned long long tagx = (unsigned long long)tag << 32;
                         const bool live = (misc[3] == 0u) && !wt.dead;
 #pragma unroll
@@ -799,24 +813,37 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                                 for (int c = 0; c < TC; ++c) { sg[c] += vg[c]; su[c] += vu[c]; }
                             }
                             if (SPLIT && (fl & kImport)) {
-                                // tail piece: the previous cluster worked on the first gate/up groups of this unit; its CTAs' partial sums are
-                                // tagged words (polled, bounded; they were stored at the very start of that cluster's range)
-                                const unsigned long long* xi = P.xsl + ((size_t)((cl - 1) * C) * 2 * TC) * kBlock + row;
+                                // Other clusters worked on gate/up groups of this unit: the ones whose ranges meet the unit's gate/up
+                                // positions [u Wg, u Wg + nk).  Their CTAs' partial sums are tagged words (polled, bounded; stored
+                                // right after those groups, which every cluster works on before anything it imports for).
+                                auto cluster_of = [&](int pos) -> int {
+                                    int p = (int)(((unsigned)pos * (unsigned)nCl) / (unsigned)total_g);
+                                    while (p + 1 < nCl && cut(p + 1) <= pos) ++p;
+                                    while (p > 0 && cut(p) > pos) --p;
+                                    return p;
+                                };
+                                const int p_lo = cluster_of(u * Wg), p_hi = cluster_of(u * Wg + nk - 1);
                                 bool okx = !wt.dead;
 #pragma unroll 1
-                                for (int r = 0; r < C && okx; ++r) {
-                                    unsigned long long v[2 * TC];
-                                    unsigned pending = (1u << (2 * TC)) - 1u;
-                                    for (uint32_t it = 1; pending; ++it) {
+                                for (int p = p_lo; p <= p_hi && okx; ++p) {
+                                    if (p == cl || cut(p + 1) == cut(p)) continue;            // (a cluster with an empty range exports nothing)
+                                    const int pslot_x = (cut(p) / Wg == u) ? 0 : 1;          // the unit is that cluster's first one, or its last
+                                    const unsigned long long* xi = P.xsl + ((size_t)((p * 2 + pslot_x) * C) * 2 * TC) * kBlock + row;
+#pragma unroll 1
+                                    for (int r = 0; r < C && okx; ++r) {
+                                        unsigned long long v[2 * TC];
+                                        unsigned pending = (1u << (2 * TC)) - 1u;
+                                        for (uint32_t it = 1; pending; ++it) {
 #pragma unroll
-                                        for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
+                                            for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
 #pragma unroll
-                                        for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
-                                        if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                            for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
+                                            if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                        }
+                                        if (!okx) break;
+#pragma unroll
+                                        for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
                                     }
-                                    if (!okx) break;
-#pragma unroll
-                                    for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
                                 }
                                 if (!okx) misc[3] = 1u;
                             }
