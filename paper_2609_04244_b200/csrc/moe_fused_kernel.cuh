@@ -162,7 +162,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     const uint32_t bar_tfull = smem_u32(bars + 2 * kMaxStages), bar_tempty = smem_u32(bars + 2 * kMaxStages + kBufs);
     const uint32_t bar_x = smem_u32(bars + 2 * kMaxStages + 2 * kBufs);
     const uint32_t bar_hq = bar_x, bar_xfull = bar_x + 16, bar_xfree = bar_x + 32, bar_drain = bar_x + 48, bar_hk = bar_x + 80;   // 2 + 2 + 2 + 4 + 1
-    uint32_t* misc = (uint32_t*)(smem + L.misc_off);   // [0] tmem base, [1] U, [3] accumulator give-up, [6] quantised input published (1) or given up (2)
+    uint32_t* misc = (uint32_t*)(smem + L.misc_off);   // [0] tmem base, [1] U, [3] accumulator give-up, [5] ticket for reduction tasks, [6] quantised input published (1) or given up (2)
     int* s_ids = (int*)(smem + L.ids_off);
     float* s_w = (float*)(smem + L.w_off);
     unsigned long long* s_mask = (unsigned long long*)(smem + L.mask_off);
@@ -187,7 +187,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         }
         for (int b = 0; b < 4; ++b) mbar_init(bar_drain + 8 * b, 1);
         mbar_init(bar_hk, 1);
-        misc[3] = 0u; misc[6] = 0u; misc[7] = 0u;
+        misc[3] = 0u; misc[5] = 0xFFFFFFFFu; misc[6] = 0u; misc[7] = 0u;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(misc), kFusedTmemCols); tmem_relinquish(); }
@@ -533,6 +533,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             if (P.stamps) P.stamps[(size_t)blockIdx.x * kStampsPerCta + 16] = (unsigned long long)w_empty;
             misc[7] = cntpar;      // which phase of every stage's `full` barrier was armed last (the teardown waits for them if the launch gave up)
         }
+        // Every copy of this CTA is requested (or it has no unit at all): take a ticket for a share of the final
+        // reduction now, so that it is there when the CTA gets to it.  Tickets go out in the order in which CTAs run out
+        // of work: the reduction is done by those that finish early, and the last CTA to finish finds none left.
+        if (SPLIT && lane == 0 && alive && !wt.dead) misc[5] = atomicAdd(P.ctrl + kDoneCnt + (tag & 1u), 1u);
         __syncwarp();
     }
     // ------------------------------------------------------------------ role: MMA issuers
@@ -911,17 +915,26 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         while (sp > 1 && sp * tpc > 8) sp >>= 1;
         const int slots = 8 / sp, slot = warp / sp, part = warp - slot * sp;
         constexpr int kRG = (SPLIT || TC >= 4) ? 3 : 1;                   // groups of eight tagged words a thread polls side by side
-        // tasks go to the CTAs from the LAST one down: the first CTAs hold the router rows and the units, and with them
-        // the next launch's critical path -- they should be the first to leave (the next launch's CTAs are placed in
-        // index order as SMs free up)
+        // Which tasks.  Steps that cannot have more units than clusters: tasks go to the CTAs from the LAST one down -- the
+        // first CTAs hold the router rows and the units, and with them the next launch's critical path; they should be the
+        // first to leave (the next launch's CTAs are placed in index order as SMs free up).  Steps that can: by ticket,
+        // `slots` consecutive tasks each; the first was taken by the producer when it ran out of work, the next ones are
+        // taken here.  A CTA that finishes late finds the tasks gone: what the grid waits for after the last store is
+        // one poll by CTAs that have been polling all along, not the whole reduction of the CTA that stored last.
         const int rc = G - 1 - cta;
         const int mine = (rc < n_tasks) ? (n_tasks - rc + G - 1) / G : 0;
         float* s_sum = s_part;                                             // [8 warps][32 rows] (the partial buffers are idle now)
         bool ok = !wt.dead;
+        constexpr bool dyn = SPLIT;
+        unsigned ticket = dyn ? misc[5] : 0u;
 #pragma unroll 1
-        for (int i0 = 0; i0 < mine; i0 += slots) {
-            const bool valid = (i0 + slot < mine);
-            const int task = rc + (valid ? i0 + slot : i0) * G;
+        for (int i0 = 0; dyn ? ((unsigned long long)ticket * (unsigned)slots < (unsigned)n_tasks) : (i0 < mine); i0 += slots) {
+            bool valid;
+            int task;
+            unsigned seen = 0u;                   // tickets handed out so far, read now, looked at after this ticket's tasks:
+            if (dyn && tid == 0) asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(P.ctrl + kDoneCnt + (tag & 1u)) : "memory");   // if none are left by then, no round trip is spent on asking
+            if (dyn) { task = (int)ticket * slots + slot; valid = task < n_tasks; if (!valid) task = (int)ticket * slots; }
+            else { valid = (i0 + slot < mine); task = rc + (valid ? i0 + slot : i0) * G; }
             const int t = div_small(task, QB), rb = task - t * QB;
             const unsigned long long* base = P.ypl + (size_t)t * NP * H + (size_t)rb * 32 + lane;
             float acc = 0.f;
@@ -971,7 +984,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 for (int q2 = 1; q2 < sp; ++q2) r += s_sum[(warp + q2) * 32 + lane];
                 P.out[(size_t)t * H + rb * 32 + lane] = __float2bfloat16_rn(r);
             }
+            if (dyn && tid == 0) misc[5] = ((unsigned long long)seen * (unsigned)slots >= (unsigned)n_tasks) ? 0xFFFFFFFFu : atomicAdd(P.ctrl + kDoneCnt + (tag & 1u), 1u);
             named_bar_sync(2, kMain);
+            if (dyn) ticket = misc[5];
         }
         if (tid == 0) MOE_STAMP(13);
     }
