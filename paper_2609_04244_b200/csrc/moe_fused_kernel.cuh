@@ -42,6 +42,13 @@ constexpr int kFusedTmemBufs = 4;                              // accumulator bu
 constexpr int kFusedIssuers = 3;                               // warps 1..3
 constexpr int kFusedTmemCols = 128;
 constexpr int kFusedThreads = 288;                             // 9 warps
+// Wait-time accounting of the roles (cycle counts written next to the time stamps): compiled in only with
+// -DMOE_FUSED_ACCOUNTING; reading the clock around every wait is not free on the short steps.
+#ifdef MOE_FUSED_ACCOUNTING
+#define MOE_CLK() clock64()
+#else
+#define MOE_CLK() 0ll
+#endif
 constexpr int kFusedMaxRows = 4;          // router rows per CTA: ceil(kMaxExperts / 128)
 
 // ---------------------------------------------------------------------------------------------
@@ -498,10 +505,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             // one group: 1 or 2 weight tiles (rows y0 / y1 of `m`, column x) and, for gate/up groups, the activation tile of K block xq_kb
             auto put = [&](const CUtensorMap* m, int x0, int y0, int x1, int y1, int ntiles, int xq_kb) -> bool {
                 const int st0 = st, st1 = (st + 1 == S) ? 0 : st + 1;
-                const long long c0 = clock64();
+                const long long c0 = MOE_CLK();
                 if (!((second >> st0) & 1u) && !wt.mbar(bar_empty + 8 * st0, ((cntpar >> st0) & 1u) ^ 1u, 21)) return false;
                 if (ntiles == 2 && !((second >> st1) & 1u) && !wt.mbar(bar_empty + 8 * st1, ((cntpar >> st1) & 1u) ^ 1u, 21)) return false;
-                w_empty += clock64() - c0;
+                w_empty += MOE_CLK() - c0;
                 const uint32_t full = bar_full + 8 * st0, dst0 = smem_u32(smem) + (uint32_t)st0 * kFusedStage;
                 mbar_expect_tx(full, (uint32_t)(ntiles * kATileBytes + (xq_kb >= 0 ? N * kBlock : 0)));
                 tma_load_2d_hint(dst0, m, x0, y0, full, stream_once);
@@ -568,12 +575,12 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 const uint32_t fp = (fpar >> st0) & 1u;
                 fpar ^= 1u << st0;
                 if (!mine) return true;
-                const long long c0 = clock64();
+                const long long c0 = MOE_CLK();
                 if (!wt.mbar(bar_tempty + 8 * iss, tpar, 24)) return false;
                 tpar ^= 1u;
-                const long long c1 = clock64();
+                const long long c1 = MOE_CLK();
                 if (!wt.mbar(bar_full + 8 * st0, fp, 26)) return false;
-                const long long c2 = clock64();
+                const long long c2 = MOE_CLK();
                 w_te += c1 - c0; w_fu += c2 - c1;
                 if (first && iss == 0) { MOE_STAMP(7); first = false; }
                 const uint32_t a0 = ring + (uint32_t)st0 * (uint32_t)kFusedStage;
@@ -592,7 +599,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                 }
                 if (release) umma_commit(bar_empty + 8 * st0);
                 umma_commit(bar_tfull + 8 * iss);
-                w_is += clock64() - c2;
+                w_is += MOE_CLK() - c2;
                 return true;
             };
             int dq = 0;                                            // items with down groups so far: slot and phase of the intermediate tile
@@ -609,7 +616,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                     if (d1 <= d0) continue;                                  // (a head piece that ends with its partial sums)
                     const int slot = dq & 1;
                     // the intermediate tile of the item is in shared memory (written by the accumulator warps)
-                    { const long long c0 = clock64(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)((dq >> 1) & 1), 27)) break; w_hq += clock64() - c0; }
+                    { const long long c0 = MOE_CLK(); if (!wt.mbar(bar_hq + 8 * slot, (uint32_t)((dq >> 1) & 1), 27)) break; w_hq += MOE_CLK() - c0; }
                     ++dq;
                     for (int h = 2 * d0; h < nh && h < 2 * d1; h += 2)
                         if (!group((h + 1 < nh) ? 2 : 1, smem_u32(s_hq) + (uint32_t)(slot * N * kBlock))) break;
@@ -633,9 +640,9 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         int buf = 0;
         uint32_t bpar = 0u;                                    // parity of the next phase of bar_tfull[buf]
         auto take = [&](float* d0, float* d1) {
-            const long long c0 = clock64();
+            const long long c0 = MOE_CLK();
             if (!wt.mbar(bar_tfull + 8 * buf, bpar, 29)) misc[3] = 1u;
-            w_tf += clock64() - c0;
+            w_tf += MOE_CLK() - c0;
             tc_fence_after();
             const uint32_t tcol = t_lane + (uint32_t)(buf * kBufCols);
             tmem_ld<TC>(tcol, d0);
@@ -784,14 +791,14 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                             const unsigned pr = s_pair[s_poff[e] + __popc(mask & ((1u << lane) - 1u))];
                             yoff_lane = (((int)(pr & 0xFFu) * K + (int)(pr >> 8)) * IB + ib) * H;
                         }
-                        const long long cf0 = clock64();
+                        const long long cf0 = MOE_CLK();
                         if (C > 1) {
                             bool okw = !wt.dead;
                             for (uint32_t it = 1; okw && !mbar_try_wait_cluster(bar_xfull + 8 * slot, pphase); ++it)
                                 if ((it & 255u) == 0 && wt.expired(31)) okw = false;
                             if (!okw) misc[3] = 1u;
                         }
-                        w_xf += clock64() - cf0;
+                        w_xf += MOE_CLK() - cf0;
                         float a[TC];
                         {
                             float sg[TC], su[TC];
@@ -883,7 +890,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         fence_proxy_async_smem();                              // generic shared-memory writes -> the tensor core's reads (not the tagged global stores in flight)
                         epi_bar(kEpiThreads);
                         if (etid == 0) { if (!(P.debug_skip & 1)) mbar_arrive(bar_hq + 8 * hslot); if (dq == 1) MOE_STAMP(10); }
-                        w_fc += clock64() - cf0;
+                        w_fc += MOE_CLK() - cf0;
                         nmask = mask; nyoff = yoff_lane; n_valid = true;
                     }
                 }
