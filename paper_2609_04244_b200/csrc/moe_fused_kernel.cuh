@@ -197,7 +197,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         misc[3] = 0u; misc[5] = 0xFFFFFFFFu; misc[6] = 0u; misc[7] = 0u;
         fence_barrier_init();
     }
-    if (warp == 1) { tmem_alloc(smem_u32(misc), kFusedTmemCols); tmem_relinquish(); }
+    if (warp == kMainWarps) { tmem_alloc(smem_u32(misc), kFusedTmemCols); tmem_relinquish(); }
 #pragma unroll 1
     for (int e = tid; e < 2 * E; e += kFusedThreads) s_mask[e] = 0ull;
     // This CTA's router rows: ask L2 for them now.  (Weights are not written by the previous launch, and a prefetch
@@ -913,8 +913,34 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // when it has eight or more), warp part q of them taking the partials q, q + sp, ...; their sums are combined in
     // fixed order.  sp depends only on the shape, the token count and the grid.
     tc_fence_before();
-    __syncthreads();
+    const int gave_up = __syncthreads_or((wt.dead || misc[3] != 0u) ? 1 : 0);
     tc_fence_after();
+    // A launch in which some thread of this CTA gave up: nothing asynchronous may outlive the CTA.  The bulk copies the
+    // producer had requested and the MMAs the issuers had issued are waited for here (bounded), whether or not those
+    // roles noticed the give-up themselves, before tensor memory is freed and shared memory goes to the next CTA.  (If
+    // no thread of the CTA gave up, every role ran to its end: every tile requested was consumed, every MMA read back.)
+    if (gave_up) {
+        if (tid == 0) {
+            const uint32_t cntpar = misc[7];
+            for (int s = 0; s < S; ++s)
+                for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
+        }
+        if (lane == 0 && warp >= 1 && warp < kEpiWarp0) {
+            const uint32_t bar = bar_drain + 8 * (uint32_t)(warp - 1);
+            umma_commit(bar);
+            for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar, 0); ++i) {}
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    // Tensor memory and the peers' view of this CTA's shared memory are not needed by the reduction: free the one and
+    // arrive on the cluster barrier now (no CTA of a cluster may leave while a peer may still read its shared memory or
+    // arrive on its barriers -- all of that happens in the roles above); the wait is at the very end, when every peer
+    // has long arrived.  (Both used to sit behind the reduction: about a microsecond between the last output row and
+    // the exit.)
+    if (warp == kMainWarps) tmem_dealloc(tmem_base, kFusedTmemCols);
+    cluster_arrive();
     if (alive && warp < kMainWarps) {
         const int QB = H / 32, n_tasks = T * QB, NP = K * IB;
         const int tpc = (n_tasks + G - 1) / G;                             // tasks of the busiest CTA
@@ -999,29 +1025,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
 
     // ------------------------------------------------------------------ teardown
-    const int gave_up = __syncthreads_or((wt.dead || misc[3] != 0u) ? 1 : 0);
-    // A launch in which some thread of this CTA gave up: nothing asynchronous may outlive the CTA.  The bulk copies the
-    // producer had requested and the MMAs the issuers had issued are waited for here (bounded), whether or not those
-    // roles noticed the give-up themselves, before tensor memory is freed and shared memory goes to the next CTA.  (If
-    // no thread of the CTA gave up, every role ran to its end: every tile requested was consumed, every MMA read back.)
-    if (gave_up) {
-        if (tid == 0) {
-            const uint32_t cntpar = misc[7];
-            for (int s = 0; s < S; ++s)
-                for (int i = 0; i < (1 << 18) && !mbar_try_wait(bar_full + 8 * s, ((cntpar >> s) & 1u) ^ 1u); ++i) {}
-        }
-        if (lane == 0 && warp >= 1 && warp < kEpiWarp0) {
-            const uint32_t bar = bar_drain + 8 * (uint32_t)(warp - 1);
-            umma_commit(bar);
-            for (int i = 0; i < (1 << 20) && !mbar_try_wait(bar, 0); ++i) {}
-        }
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-    }
-    if (warp == 1) tmem_dealloc(tmem_base, kFusedTmemCols);
-    // no CTA of the cluster leaves while a peer may still read its shared memory or arrive on its barriers
-    cluster_arrive();
+    // (every thread of the cluster arrived on the cluster barrier right after its roles: nobody waits here for long)
     cluster_wait();
     if (tid == 0) {
         if (P.stamps) { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); P.stamps[(size_t)blockIdx.x * kStampsPerCta + 14] = smid; }
