@@ -1649,13 +1649,11 @@ moe_decode_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_consta
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
     if (tid == 0) {
         MOE_STAMP_ALWAYS(15);
-        __threadfence();
-        const unsigned old = atomicAdd(P.ctrl + kExitCnt, 1u);
-        if (old == (unsigned)G - 1u) {          // last CTA out: open the next epoch
-            P.ctrl[kExitCnt] = 0u;
-            __threadfence();
-            st_release(P.ctrl + kEpoch, tag);
-        }
+        // Open the next epoch.  CTA 0 alone does it, without counting exits: it got here only after the grid-wide routing
+        // wait, that is after every CTA had read this launch's tag; the next launch reads the epoch only once this grid
+        // has completed.  (A fence and a returning atomic per CTA used to sit here: two L2 round trips at every exit.)
+        // Unconditionally: a launch that gave up must not leave its tag to the next one.
+        if (cta == 0) st_release(P.ctrl + kEpoch, tag);
     }
 }
 
