@@ -206,9 +206,11 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     for (int e = cta; e < E; e += G)
         for (int l = tid; l < H / 64; l += kFusedThreads) prefetch_l2(reinterpret_cast<const char*>(P.Wr + (size_t)e * H) + l * 128);
     if (P.bias && tid * 32 < E) prefetch_l2(P.bias + tid * 32);
-    // every CTA of the cluster has initialised its barriers before anyone arrives on them remotely
+    // Every CTA of the cluster must have initialised its barriers before anyone arrives on them remotely.  Real
+    // clusters wait for that here (measured: starting the CTAs of a cluster in step is worth more than the wait costs);
+    // a cluster of one only has to pair the arrival with a wait somewhere before the barrier's second use.
     cluster_arrive();
-    cluster_wait();
+    if (C > 1) cluster_wait();
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     Waiter wt;
@@ -628,6 +630,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
     // ------------------------------------------------------------------ role: accumulator / epilogue warps
     else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
+        if (C == 1) cluster_wait();                            // (pairs with the set-up's arrival)
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -940,6 +943,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // has long arrived.  (Both used to sit behind the reduction: about a microsecond between the last output row and
     // the exit.)
     if (warp == kMainWarps) tmem_dealloc(tmem_base, kFusedTmemCols);
+    if (C == 1 && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();   // (pairs with the set-up's arrival; the accumulator warps have waited)
     cluster_arrive();
     if (alive && warp < kMainWarps) {
         const int QB = H / 32, n_tasks = T * QB, NP = K * IB;
