@@ -53,10 +53,16 @@ CELLS = [("c1_tiny", 1, "natural"), ("c2_qwen3_30b_a3b", 2, "natural"), ("c2_qwe
          ("c5_deepseek_v3", 1, "natural"), ("c5_deepseek_v3", 8, "natural")]
 
 
-def kernel_name(info, T):
+def kernel_name(info, T, shape=None):
     """Name of the kernel instantiation a plan launches for T tokens."""
     if info.get("fused"):
-        return f"moe_fused_kernel<{1 if T <= 1 else 2 if T <= 2 else 4 if T <= 4 else 8}>"
+        tc = 1 if T <= 1 else 2 if T <= 2 else 4 if T <= 4 else 8
+        if shape is None:
+            return f"moe_fused_kernel<{tc}>"
+        # the instantiation with the unit-sharing code runs where a step can have more units than clusters
+        clusters = info["grid"] // max(1, info["cluster"])
+        split = min(shape.E, T * shape.top_k) * (shape.I // 128) > clusters and (shape.H // 128) % max(1, info["cluster"]) == 0
+        return f"moe_fused_kernel<{tc}, {'true' if split else 'false'}>"
     return f"moe_decode_kernel<N={info['n_hw']}>"
 
 
@@ -431,7 +437,7 @@ def main():
                           "algorithmic_bytes_per_step": r["bytes_per_step"], "achieved_gbs": gbs, "frac": gbs / peak_c,
                           "traffic": NCU_TRAFFIC_BYTES.get((name, Tc)) if regime == "natural" else None,
                           "unique_experts_mean": float(np.mean(r["uniq"])), "layer_copies": r["L"],
-                          "variant": kernel_name(r["info"], Tc), "cluster": r["info"]["cluster"], "stages": r["info"]["stages"],
+                          "variant": kernel_name(r["info"], Tc, shp), "cluster": r["info"]["cluster"], "stages": r["info"]["stages"],
                           "clocks": {k: r["clocks"].get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")}})
 
     ms, e2e_ms_max = max_over_ranks([ms, e2e["ms"] if e2e else 0.0], dev)
@@ -454,11 +460,11 @@ def main():
                        f"({L * bytes_per_step / 2**20:.0f} MiB streamed between reuses, L2 is 126 MiB)",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "grid": info["grid"], "stages": info["stages"], "n_hw": info["n_hw"],
-                       "variant": kernel_name(info, T), "cluster": info["cluster"],
+                       "variant": kernel_name(info, T, shape), "cluster": info["cluster"],
                        "launch": "direct launches" if args.no_graph else "CUDA graph replay, one kernel node per step"},
             "achieved_gbs": achieved, "algorithmic_bytes_per_step": bytes_per_step,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}", "kernel": kernel_name(info, T), "kernel_us": kernel_us,
+                         "peak_kind": f"of {peak_kind}", "kernel": kernel_name(info, T, shape), "kernel_us": kernel_us,
                          "traffic": NCU_TRAFFIC_BYTES.get((shape.name, T))},
             "gpu_launches": K * launches_per_step,
             "clocks": clocks,
