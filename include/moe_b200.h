@@ -210,14 +210,14 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              columns in use), instead of ranges of equal length.  0 = equal length, 1..8 = strength
  *                              of the per-column term in quarters of the fitted value, -1 = the library's choice
  *                              (default: 4 from 24 tokens on, from 16 where I <= 256, else 0)
- *   MOE_KNOB_FUSED             (plan-wide) fused-unit variant for 1..8 tokens: 1 = wherever it can run, 0 = never,
- *                              -1 = the library's choice (default).  Changes the scratch layout: query
+ *   MOE_KNOB_FUSED             (per token count 1..8) kernel variant: 1 = the fused-unit variant if it can run, 0 = the
+ *                              general variant, -1 = the library's choice (default).  Changes the scratch layout: query
  *                              moe_workspace_bytes() again.
  *   MOE_KNOB_CLUSTER           fused-unit variant: CTAs that share one unit (thread-block cluster size) 1, 2, 4 or 8;
  *                              0 = the library's choice (default): the size for which the busiest CTA streams the fewest
  *                              tiles at the expected number of distinct experts.  MOE_ERR_OCCUPANCY if the device cannot
  *                              hold such clusters.  With MOE_KNOB_STAGES = 0 the fused variant takes as many stages as
- *                              leave half of the SM's shared memory to the next launch's CTA.
+ *                              fit one CTA per SM.
  *   MOE_KNOB_SPLIT_UNITS       (plan-wide) fused-unit variant: 1 (default) = where a step has more units than clusters, the
  *                              list of all accumulation groups is cut into equal ranges, one per cluster; a range may begin
  *                              and end anywhere inside a unit (clusters that share a unit exchange partial sums); 2 = the

@@ -84,7 +84,7 @@ struct moe_plan {
     int use_pdl = 1;                // programmatic dependent launch
     int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
     // fused-unit variants (1..8 tokens, moe_fused_kernel.cuh)
-    int fused_mode = -1;            // 1: wherever they apply, 0: never, -1: the library's choice
+    int fused_knob[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // per token count 1..8: 1 = the fused variant, 0 = the general one, -1 = the library's choice
     int cluster_knob[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // CTAs per unit for T = 1..8; 0 = the library's choice
     int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
     int smem_per_sm = 0;
@@ -190,8 +190,8 @@ struct moe_plan {
     // down projection is at most two K blocks (there the general variant's per-unit work weighs most) and for a single
     // token.
     bool fused(int T) const {
-        if (fused_mode == 0 || !fused_possible(T)) return false;
-        if (fused_mode == 1) return true;
+        if (!fused_possible(T) || fused_knob[T] == 0) return false;
+        if (fused_knob[T] == 1) return true;
         const double tiles = 3.0 * expected_experts(T) * (I / 128) * (H / 128) / sms;
         return tiles <= 120.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
     }
@@ -481,7 +481,7 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             return MOE_OK;
         case MOE_KNOB_FUSED:
             if (value < -1 || value > 1) return fail(MOE_ERR_ARG, "fused must be -1 (library's choice), 0 or 1");
-            plan->fused_mode = value;
+            for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->fused_knob[t] = value;
             return MOE_OK;
         case MOE_KNOB_CLUSTER:
             if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return fail(MOE_ERR_ARG, "cluster size must be 0 (library's choice), 1, 2, 4 or 8");
@@ -520,7 +520,7 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_COMPACT_MIN: *value = plan->compact_min; return MOE_OK;
         case MOE_KNOB_PDL: *value = plan->use_pdl; return MOE_OK;
         case MOE_KNOB_SPLIT_WEIGHT: *value = plan->split_weight[t]; return MOE_OK;
-        case MOE_KNOB_FUSED: *value = plan->fused_mode; return MOE_OK;
+        case MOE_KNOB_FUSED: *value = t <= 8 ? plan->fused_knob[t] : 0; return MOE_OK;
         case MOE_KNOB_CLUSTER: *value = t <= 8 ? plan->cluster_knob[t] : 0; return MOE_OK;
         case MOE_KNOB_STAMPS: *value = plan->take_stamps; return MOE_OK;
         case MOE_KNOB_DEBUG_SKIP: *value = plan->debug_skip; return MOE_OK;

@@ -3,8 +3,8 @@ numerical check are rejected, the rest are ranked by CUDA-graph timing over toke
 
 The kernel's schedule knobs are those of `moe_plan_set_knob` (include/moe_b200.h): pipeline stages, the whole-unit vs
 split-K threshold, the token count up to which every CTA routes all tokens, equal-weight ranges, the compaction
-threshold.  For one layer
-shape this module times every candidate on seeded synthetic layers (the inputs of `workloads`), validates each
+threshold and, for 1..8 tokens, the kernel variant (general or fused-unit) with the fused variant's cluster size.  For
+one layer shape this module times every candidate on seeded synthetic layers (the inputs of `workloads`), validates each
 candidate's output against the default schedule's output of the same step, and writes a table that
 `MoEPlan(..., schedule=table)` / `MoEPlan.apply_schedule(table)` / `bench.py --schedule FILE` apply:
 
@@ -37,6 +37,8 @@ PER_TOKEN_GRID = {
     "split_weight": [-1, 0, 4],
 }
 PLAN_GRID = {"compact_min": [9, 5]}
+# 1..8 tokens: the kernel variant and, for the fused-unit variant, the cluster size (0 = the library's own choice)
+FUSED_CLUSTERS = [0, 1, 2, 4]
 
 
 def _layers(shape, T, regime, n_layers, device):
@@ -86,6 +88,21 @@ def relevant_knobs(T, per_launch):
     if min(T, per_launch) < 9:                       # equal-weight ranges exist only where tokens are compacted
         grid["split_weight"] = [-1]
     return grid
+
+
+def candidates(T, per_launch, fused_possible):
+    """Every schedule tried for T tokens, as knob dictionaries.  Up to 8 tokens the kernel variant is part of the
+    schedule: the general variant with its knobs, and the fused-unit variant with every cluster size (its other knobs
+    do not apply to it)."""
+    grid = relevant_knobs(T, per_launch)
+    names = list(grid)
+    general = [dict(zip(names, combo)) for combo in itertools.product(*(grid[n] for n in names))]
+    if min(T, per_launch) > 8 or not fused_possible:
+        return general
+    out = [dict(k, fused=0, cluster=0) for k in general]
+    base = {n: plan_default(n, T) for n in names}
+    out += [dict(base, fused=1, cluster=c) for c in FUSED_CLUSTERS]
+    return out
 
 
 def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=3, device="cuda", log=None):
@@ -140,13 +157,18 @@ def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=
             refs.append(plan.forward(d["hidden"], d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"]).clone())
         plan.sync_status()
         default_us = sum(_time_graph(plan, layers, steps, replays) for _, layers in cases) / len(cases)
-        grid = relevant_knobs(T, plan.tokens_per_launch())
-        names = list(grid)
+        plan.set_knob(T, "fused", 1)
+        fused_possible = bool(plan.info(T)["fused"])            # (the shape may not admit the fused variant at all)
+        plan.set_knob(T, "fused", -1)
+        cands = candidates(T, plan.tokens_per_launch(), fused_possible)
+        names = list(cands[0])
         results = []
-        for combo in itertools.product(*(grid[n] for n in names)):
-            knobs = dict(zip(names, combo))
-            for n, v in knobs.items():
-                plan.set_knob(T, n, v)
+        for knobs in cands:
+            try:
+                for n, v in knobs.items():
+                    plan.set_knob(T, n, v)
+            except Exception:                                    # (a cluster size the device or the shape does not admit)
+                continue
             ok, us = True, 0.0
             for (regime, layers), ref in zip(cases, refs):
                 d = layers[0]
@@ -173,7 +195,8 @@ def tune(shape, tokens, regimes=("natural",), n_layers=None, steps=200, replays=
 
 
 def plan_default(knob, T=1):
-    return {"split_slack_kib": 200 if T <= 8 else 100, "stages": 0, "route_all_tokens": 8, "split_weight": -1}[knob]
+    return {"split_slack_kib": 200 if T <= 8 else 100, "stages": 0, "route_all_tokens": 8, "split_weight": -1,
+            "fused": -1, "cluster": 0}[knob]
 
 
 def main(argv=None):

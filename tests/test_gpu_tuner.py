@@ -29,7 +29,22 @@ def test_knobs_round_trip_and_reject_bad_values():
     assert plan.get_knob(16, "split_weight") == 8 and plan.get_knob(12, "split_weight") == -1
     with pytest.raises(Exception):
         plan.set_knob(16, "split_weight", 9)
+    assert plan.get_knob(4, "fused") == -1 and plan.get_knob(4, "cluster") == 0
+    plan.set_knob(4, "fused", 0)                          # the kernel variant is a per-token-count knob
+    assert plan.get_knob(4, "fused") == 0 and plan.get_knob(3, "fused") == -1 and not plan.info(4)["fused"]
+    plan.set_knob(4, "fused", 1)
+    plan.set_knob(4, "cluster", 2)
+    assert plan.info(4)["fused"] and plan.info(4)["cluster"] == 2
+    with pytest.raises(Exception):
+        plan.set_knob(4, "cluster", 3)
     plan.close()
+
+
+def test_candidates_cover_both_kernel_variants_up_to_eight_tokens():
+    small = tuner.candidates(4, 64, True)
+    assert any(c["fused"] == 1 and c["cluster"] == 2 for c in small) and any(c["fused"] == 0 for c in small)
+    assert all("fused" not in c for c in tuner.candidates(16, 64, True))
+    assert all("fused" not in c for c in tuner.candidates(4, 64, False))
 
 
 def test_search_emits_a_table_that_keeps_parity(tmp_path):
