@@ -106,3 +106,26 @@ def test_host_activation_entry_point_matches_device_entry_point():
     plan.sync_status()
     assert torch.equal(h_out, ref.cpu())
     plan.close()
+
+
+@pytest.mark.parametrize("name,T,pinned", [("c2_qwen3_30b_a3b", 1, True), ("c2_qwen3_30b_a3b", 1, False), ("c2_qwen3_30b_a3b", 3, True),
+                                           ("c1_tiny", 1, True), ("small_sig", 1, True), ("small_sig", 8, True)])
+def test_host_entry_point_small_token_counts(name, T, pinned):
+    """Few tokens from host memory: the result is written by the kernel straight into a pinned output buffer; pageable
+    buffers take the staged path.  Same bits as the device entry point either way, also when the host buffers change
+    between calls."""
+    from paper_2609_04244_b200 import MoEPlan
+    shape = SMALL_SIG if name == "small_sig" else wl.SHAPES[name]
+    plan = MoEPlan(shape.H, shape.E, shape.I, shape.top_k, shape.scoring, shape.renorm, T_max=T)
+    for layer in range(3):
+        d = wl.make_layer(shape, T, layer=layer, device="cuda")
+        args = (d["Wr"], d["bias"], d["W13q"], d["W13s"], d["W2q"], d["W2s"])
+        ref = plan.forward(d["hidden"], *args).clone()
+        h_in = d["hidden"].cpu()
+        h_out = torch.zeros((T, shape.H), dtype=torch.bfloat16)
+        if pinned:
+            h_in, h_out = h_in.pin_memory(), h_out.pin_memory()
+        plan.forward_host(h_in, *args, h_out)
+        plan.sync_status()
+        assert torch.equal(h_out, ref.cpu()), (name, T, layer)
+    plan.close()
