@@ -61,7 +61,7 @@ def kernel_name(info, T, shape=None):
         if shape is None:
             return f"moe_fused_kernel<{tc}>"
         # the instantiation with the unit-sharing code runs where a step can have more units than clusters
-        clusters = info["grid"] // max(1, info["cluster"])
+        clusters = info["grid"] if info.get("pairs_at_runtime") else info["grid"] // max(1, info["cluster"])
         split = min(shape.E, T * shape.top_k) * (shape.I // 128) > clusters and (shape.H // 128) % max(1, info["cluster"]) == 0
         return f"moe_fused_kernel<{tc}, {1 if split else 0}>"
     return f"moe_decode_kernel<N={info['n_hw']}>"

@@ -171,10 +171,12 @@ int moe_tokens_per_launch(moe_plan_t plan);
 /* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);
 
-/* Introspection: which kernel variant T tokens get.  *fused = 1 for the fused-unit variant (1..8 tokens: a work unit
- * is one expert's 128-wide intermediate block through gate/up AND its down-projection column block, shared by the
- * *cluster CTAs of a thread-block cluster; Section 3.2's hand-over of the intermediate tile stays on chip), 0 for the
- * general variant (*cluster = 1).  Either out may be NULL. */
+/* Introspection: which kernel variant T tokens get.  *fused = 1 or 2 for the fused-unit variant (1..8 tokens: a work
+ * unit is one expert's 128-wide intermediate block through gate/up AND its down-projection column block, shared by
+ * the *cluster CTAs of a thread-block cluster; Section 3.2's hand-over of the intermediate tile stays on chip), 0 for
+ * the general variant (*cluster = 1).  2: the launch is made in pairs (*cluster = 2) and the kernel decides after
+ * routing whether the CTAs of a pair share units (the step has at most as many units as pairs) or work alone.
+ * Either out may be NULL. */
 int moe_plan_variant(moe_plan_t plan, int T, int* fused, int* cluster);
 
 /* Diagnostics: synchronise `stream` and copy the phase time stamps of the last launch on this workspace to

@@ -188,15 +188,17 @@ def moe_tokens_per_launch(plan) -> int:
 def moe_plan_info(plan, T: int) -> dict:
     g, s, n, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     _check(load_library().moe_plan_info(plan, T, ctypes.byref(g), ctypes.byref(s), ctypes.byref(n), ctypes.byref(b)))
-    f, c = moe_plan_variant(plan, T)
-    return {"grid": g.value, "stages": s.value, "n_hw": n.value, "smem_bytes": b.value, "fused": f, "cluster": c}
+    f, c, dyn = moe_plan_variant(plan, T)
+    return {"grid": g.value, "stages": s.value, "n_hw": n.value, "smem_bytes": b.value, "fused": f, "cluster": c,
+            "pairs_at_runtime": dyn}
 
 
 def moe_plan_variant(plan, T: int):
-    """(fused, cluster): whether T tokens get the fused-unit kernel variant, and the CTAs that share one unit."""
+    """(fused, cluster, pairs_at_runtime): whether T tokens get the fused-unit kernel variant, the CTAs per cluster of the
+    launch, and whether the kernel decides after routing if the CTAs of a pair share units or work alone."""
     f, c = ctypes.c_int(), ctypes.c_int()
     _check(load_library().moe_plan_variant(plan, T, ctypes.byref(f), ctypes.byref(c)))
-    return bool(f.value), c.value
+    return bool(f.value), c.value, f.value == 2
 
 
 class MoEPlan:

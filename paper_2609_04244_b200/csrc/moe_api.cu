@@ -88,6 +88,7 @@ struct moe_plan {
     int cluster_knob[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // CTAs per unit for T = 1..8; 0 = the library's choice
     int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
     int smem_per_sm = 0;
+    int pairs_at_runtime = 1;       // fused variants: launches in pairs decide after routing whether the pairs share units (see fused_dyn)
     int split_units = 1;            // fused variants: equal ranges of the group list per cluster (units may be split between two clusters)
     int host_direct = 1;            // moe_forward_host: bit 0 = write a small result straight into pinned host memory, bit 1 = read a small input in place
     int take_stamps = 0;            // kernels record their phase time stamps (diagnostics)
@@ -170,14 +171,26 @@ struct moe_plan {
     // pairs -- still get a cluster each, so that the step is one round in which every unit's 3 * H/128 tiles are
     // shared by as many CTAs as possible; one CTA per unit once there are more units than SMs.  (Measured on the nine
     // benchmark shapes at 1-8 tokens: this is the fastest size in 47 of 54 cases and within 4 % in the others.)
-    int fused_cluster(int T) const {
+    // Cluster size by the expected number of units: the largest of 4, 2 for which every unit gets a cluster of its own.
+    int fused_cluster_static(int T) const {
         const int KB = H / 128;
-        const int knob = cluster_knob[T];
-        if (knob > 0) return (knob <= 8 && max_clusters[knob] > 0 && knob <= KB) ? knob : 0;
         const long long units = (long long)expected_experts(T) * (I / 128);
         for (int C = 4; C > 1; C /= 2)
             if (max_clusters[C] > 0 && C <= KB && units <= max_clusters[C]) return C;
         return max_clusters[1] > 0 ? 1 : 0;
+    }
+    // Where that says 1 or 2 the launch is made in pairs that cover the whole grid, and the kernel decides after routing,
+    // from the number of units the step really has, whether the CTAs of a pair share units or work alone.
+    bool fused_dyn(int T) const {
+        if (cluster_knob[T] != 0 || !pairs_at_runtime) return false;
+        const int C = fused_cluster_static(T), KB = H / 128;
+        return (C == 1 || C == 2) && KB % 2 == 0 && max_clusters[2] * 2 == sms && max_clusters[1] == sms;
+    }
+    int fused_cluster(int T) const {
+        const int KB = H / 128;
+        const int knob = cluster_knob[T];
+        if (knob > 0) return (knob <= 8 && max_clusters[knob] > 0 && knob <= KB) ? knob : 0;
+        return fused_dyn(T) ? 2 : fused_cluster_static(T);
     }
     int fused_grid(int T) const { const int C = fused_cluster(T); return C ? C * max_clusters[C] : 0; }
     bool fused_possible(int T) const {
@@ -350,7 +363,7 @@ moe::Params make_params(const Plan* p, int T, int stages, const WsLayout& L, uin
     P.ypl = reinterpret_cast<unsigned long long*>(w + L.yp);
     P.xsl = reinterpret_cast<unsigned long long*>(w + L.xsl);
     P.fsplit = 0;
-    P.fC = 1; P.fnCl = p->sms;
+    P.fC = 1; P.fnCl = p->sms; P.fdyn = 0; P.grid_magic1 = 0;
     for (int r = 0; r < 9; ++r) { P.fkb[r] = 0; P.fhb[r] = 0; }
     P.stamps = p->take_stamps ? reinterpret_cast<unsigned long long*>(w + L.stamps) : nullptr;
     P.stamps_buf = reinterpret_cast<unsigned long long*>(w + L.stamps);
@@ -395,10 +408,13 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
         const int KB = p->H / 128;
         P.fC = C; P.fnCl = grid / C;
+        P.fdyn = p->fused_dyn(T) ? (p->fused_cluster_static(T) == 2 ? 1 : 2) : 0;
+        P.grid_magic1 = (1ull << 40) / (unsigned long long)grid + 1ull;
         // units are shared between clusters only where the step can have more units than clusters at all: T tokens select
         // at most min(E, T * top_k) experts (the instantiations without that code are smaller and faster)
         const int max_units = (T * p->K < p->E ? T * p->K : p->E) * (p->I / 128);
-        P.fsplit = (p->split_units && KB % C == 0 && (max_units > P.fnCl || p->split_units == 2)) ? p->split_units : 0;
+        // (pairs that may work alone: then the clusters are the CTAs)
+        P.fsplit = (p->split_units && KB % C == 0 && (max_units > (P.fdyn ? grid : P.fnCl) || p->split_units == 2)) ? p->split_units : 0;
         P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
         for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;
@@ -821,7 +837,7 @@ int moe_plan_variant(moe_plan_t plan, int T, int* fused, int* cluster) {
     if (!plan || T < 1) return fail(MOE_ERR_ARG, "bad arguments");
     const int Tc = plan->cap(T);
     const bool f = plan->fused(Tc);
-    if (fused) *fused = f ? 1 : 0;
+    if (fused) *fused = f ? (plan->fused_dyn(Tc) ? 2 : 1) : 0;
     if (cluster) *cluster = f ? plan->fused_cluster(Tc) : 1;
     return MOE_OK;
 }

@@ -156,8 +156,11 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     constexpr int kBufs = kFusedTmemBufs, kBufCols = 2 * N;          // an accumulator buffer = two 16-column halves
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
-    const int C = P.fC, nCl = P.fnCl, rank = (int)cluster_ctarank();
-    const int cl = (int)cluster_id_x();
+    // LC = the cluster size of the launch.  C, nCl, rank, cl = how the CTAs work: as the launch says or -- decided after
+    // routing, see there -- every CTA on its own although launched in pairs.
+    const int LC = P.fC;
+    int C = LC, nCl = P.fnCl, rank = (int)cluster_ctarank(), cl = (int)cluster_id_x();
+    unsigned long long gmagic = P.grid_magic;                     // division by the number of (working) clusters
     const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock;
     const int S = P.stages;
@@ -189,8 +192,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         for (int b = 0; b < kBufs; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_hq + 8 * b, 1);
-            mbar_init(bar_xfull + 8 * b, 4 * C);             // one arrival per accumulator warp of every CTA of the cluster
-            mbar_init(bar_xfree + 8 * b, 4 * C);
+            mbar_init(bar_xfull + 8 * b, 4 * LC);             // one arrival per accumulator warp of every CTA of the cluster
+            mbar_init(bar_xfree + 8 * b, 4 * LC);
         }
         for (int b = 0; b < 4; ++b) mbar_init(bar_drain + 8 * b, 1);
         mbar_init(bar_hk, 1);
@@ -210,7 +213,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // clusters wait for that here (measured: starting the CTAs of a cluster in step is worth more than the wait costs);
     // a cluster of one only has to pair the arrival with a wait somewhere before the barrier's second use.
     cluster_arrive();
-    if (C > 1) cluster_wait();
+    const bool late_wait = (LC == 1) || (P.fdyn == 2);          // (pairs that are expected to work alone do not meet here either)
+    if (!late_wait) cluster_wait();
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     Waiter wt;
@@ -419,8 +423,17 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     if (P.stamps_fine) { if (tid == 0) MOE_STAMP(5); __syncwarp(); }
     const int nU = U * IB;                                       // units of this step
     // this CTA's share of every unit: K blocks [kb_lo, kb_hi) of the gate/up rows, row blocks [hb_lo, hb_hi) of W2
-    const int kb_lo = P.fkb[rank], kb_hi = P.fkb[rank + 1], nk = kb_hi - kb_lo;
-    const int hb_lo = P.fhb[rank], hb_hi = P.fhb[rank + 1], nh = hb_hi - hb_lo;
+    // Pairs or every CTA on its own?  A launch made with clusters of two where the host could not know (`fdyn`) decides
+    // now that the step's units are counted: as many units as pairs or fewer -- every pair shares one (half of the K
+    // blocks and half of the W2 row blocks each, sums exchanged over distributed shared memory); more -- every CTA
+    // works alone on whole units or ranges, as if launched with clusters of one (the pairing then only places the two
+    // CTAs next to each other).  The expected number of distinct experts says which it will usually be; routing that
+    // crowds a few experts (8 tokens on the same 8 experts: 48 units instead of 312) gets the other arrangement
+    // instead of leaving two thirds of the SMs without a unit.
+    const bool solo = (P.fdyn != 0) && (nU > nCl);
+    if (solo) { C = 1; nCl = G; rank = 0; cl = cta; gmagic = P.grid_magic1; }
+    const int kb_lo = solo ? 0 : P.fkb[rank], kb_hi = solo ? KBu : P.fkb[rank + 1], nk = kb_hi - kb_lo;
+    const int hb_lo = solo ? 0 : P.fhb[rank], hb_hi = solo ? KBu : P.fhb[rank + 1], nh = hb_hi - hb_lo;
     const int ngd = (nh + 1) >> 1;                               // down groups per unit
     // Which units this cluster works on.  Either whole units, dealt round-robin, or -- where the host allows it and the
     // step has more units than clusters (or the host asks for it regardless: few crowded experts leave most clusters
@@ -439,7 +452,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // only from clusters below it: nobody waits in a circle, and nobody's export waits for an import.
     const int Wg = nk + ngd, total_g = nU * Wg;
     const bool split = SPLIT && (P.fsplit != 0) && (nU > nCl || P.fsplit == 2);
-    auto cut = [&](int c) -> int { return (c >= nCl) ? total_g : (int)div_grid((unsigned)c * (unsigned)total_g, P.grid_magic); };
+    auto cut = [&](int c) -> int { return (c >= nCl) ? total_g : (int)div_grid((unsigned)c * (unsigned)total_g, gmagic); };
     int n, first_whole = 0, nw = 0, hs = 0, ua = 0, xa = 0, ue = 0, xe = 0;
     bool has_tail = false;
     if (split) {
@@ -456,7 +469,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             n = hs + nw + (has_tail ? 1 : 0);
         }
     } else {
-        n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), P.grid_magic) : 0;   // units cl, cl + nCl, ... (grid_magic divides by the cluster count)
+        n = (cl < nU) ? (int)div_grid((unsigned)(nU - cl + nCl - 1), gmagic) : 0;   // units cl, cl + nCl, ... (grid_magic divides by the cluster count)
     }
     // item s of this cluster, in working order: unit u = (expert e, intermediate block ib), gate/up groups [g0, g1) of
     // this CTA's K blocks, down groups [d0, d1) of this CTA's row blocks (none: the item ends with its partial sums),
@@ -630,7 +643,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
     // ------------------------------------------------------------------ role: accumulator / epilogue warps
     else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
-        if (C == 1) cluster_wait();                            // (pairs with the set-up's arrival)
+        if (late_wait) cluster_wait();                         // (pairs with the set-up's arrival)
         const int q = warp & 3, row = q * 32 + lane;           // TMEM lane == weight row inside the tile
         const int etid = tid - kEpiWarp0 * 32;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -943,7 +956,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // has long arrived.  (Both used to sit behind the reduction: about a microsecond between the last output row and
     // the exit.)
     if (warp == kMainWarps) tmem_dealloc(tmem_base, kFusedTmemCols);
-    if (C == 1 && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();   // (pairs with the set-up's arrival; the accumulator warps have waited)
+    if (late_wait && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();   // (pairs with the set-up's arrival; the accumulator warps have waited)
     cluster_arrive();
     if (alive && warp < kMainWarps) {
         const int QB = H / 32, n_tasks = T * QB, NP = K * IB;
