@@ -14,22 +14,27 @@
 //     Partial gate/up sums are exchanged through distributed shared memory (each CTA keeps its partial in its own
 //     shared memory, peers read it with ld.shared::cluster after a remote mbarrier arrival) and every CTA of the
 //     cluster computes the same SiLU(gate)*up, amax and FP8 codes (Section 3.3, up-projection epilogue) -- so the
-//     intermediate tile needs no broadcast.  Units go to clusters round-robin; inside a cluster the stream is
-//     software-pipelined by one unit (up(0) up(1) down(0) up(2) down(1) ...), so the exchange of unit i hides under
-//     the gate/up tiles of unit i+1.
+//     intermediate tile needs no broadcast.  Launches in pairs decide after routing, from the number of units the
+//     step really has, whether the CTAs of a pair share units or work alone.
+//   * Units go to clusters whole, round-robin, or -- where a step has more units than clusters -- the list of all
+//     accumulation groups is cut into equal ranges that may begin and end inside a unit; clusters that share a unit
+//     exchange partial sums as tagged words.  Inside a cluster the stream is software-pipelined by one unit
+//     (up(0) up(1) down(0) up(2) down(1) ...), so the exchange of unit i hides under the gate/up tiles of unit i+1.
 //   * Router (Section 3.3): CTA c computes the logits of experts c, c+G, ... for all tokens with plain FMAs (the
 //     rows were prefetched into L2 before the wait on the previous launch) and publishes each as one 64-bit word
 //     {launch tag, logit}; every CTA polls those words directly -- one store trip plus one load trip, no counter,
-//     no fence -- and selects for all tokens itself.
+//     no fence -- and selects for all tokens itself.  The down partials reach the final reduction the same way.
 //   * Input quantisation (Section 4.1) is spread over the grid into the workspace and consumed by bulk-tensor copies,
 //     behind an arrival counter that is off the critical path (the first activation tile is needed a first-tile
 //     latency after the first weight request).
-//   * Shared memory stays below half an SM and tensor memory at 256 columns, so the CTAs of the NEXT launch
-//     (programmatic dependent launch) are resident, initialised and have their router rows in L2 while this launch
-//     still streams (Section 3.3 carries its lookahead across expert boundaries; this carries it across launches).
+//   * One CTA per SM with a stage ring as deep as shared memory allows (two CTAs per SM with half the ring were
+//     measured: the launch-to-launch interval does not shrink, the stream gets slower); the launch is made with the
+//     programmatic-stream-serialization attribute, so the next launch's set-up and the L2 prefetch of its router rows
+//     run ahead of its dependency wait.
 //
-// Warp roles as in moe_kernel.cuh: warp 0 weight-tile producer, warp 2 activation-tile producer, warps 1 and 3
-// tcgen05 MMA issuers (alternate accumulation groups), warps 4..7 accumulator/epilogue (thread = weight row).
+// Warps: 0 producer (weight and activation tiles by bulk-tensor copy), 1..3 tcgen05 MMA issuers (take accumulation
+// groups in turn, each with its own tensor-memory buffer), 4..7 accumulator/epilogue (thread = weight row), 8
+// housekeeping during the routing phase (publishing and awaiting the quantised input, tensor-memory allocation).
 #pragma once
 
 #include "moe_kernel.cuh"
@@ -563,7 +568,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     }
     // ------------------------------------------------------------------ role: MMA issuers
     // Measured in this kernel: one group (two waits, a fence, eight tcgen05.mma, two commits) occupies its issuing thread
-    // for about 1100 cycles, far longer than the tensor pipe needs for it.  So up to four threads (warps 1, 2, 3, 8)
+    // for about 1100 cycles, far longer than the tensor pipe needs for it.  So three threads (warps 1, 2, 3)
     // take the groups in turn, each with the accumulator buffer of its own number; all of them walk the whole sequence
     // to keep the stage positions and barrier phases.  Commits are kept few -- one `empty` and one `full` per group,
     // no `empty` for stages that are never refilled.  With NI issuers and NI buffers nobody runs more than NI groups
