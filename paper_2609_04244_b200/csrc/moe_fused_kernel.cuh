@@ -166,7 +166,8 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     const int LC = P.fC;
     int C = LC, nCl = P.fnCl, rank = (int)cluster_ctarank(), cl = (int)cluster_id_x();
     unsigned long long gmagic = P.grid_magic;                     // division by the number of (working) clusters
-    const int T = P.T, H = P.H, E = P.E, I = P.I, K = P.K;
+    const int T = (TC == 1) ? 1 : P.T;                          // (one token column means one token: its loops fold)
+    const int H = P.H, E = P.E, I = P.I, K = P.K;
     const int KBu = H / kBlock, IB = I / kBlock, HB = H / kBlock;
     const int S = P.stages;
     const FusedSmem L = fused_smem_layout(TC, T, K, E, H, S);
