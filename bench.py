@@ -57,7 +57,7 @@ CELLS = [("c1_tiny", 1, "natural"), ("c2_qwen3_30b_a3b", 2, "natural"), ("c2_qwe
 def kernel_name(info, T, shape=None):
     """Name of the kernel instantiation a plan launches for T tokens."""
     if info.get("fused"):
-        tc = 1 if T <= 1 else 2 if T <= 2 else 4 if T <= 4 else 8
+        tc = 1 if T <= 1 else 2 if T <= 2 else 4 if T <= 4 else 8 if T <= 8 else 16
         if shape is None:
             return f"moe_fused_kernel<{tc}>"
         # the instantiation with the unit-sharing code runs where a step can have more units than clusters

@@ -171,7 +171,7 @@ int moe_tokens_per_launch(moe_plan_t plan);
 /* Introspection: persistent grid size, pipeline stages and hardware N used for T tokens; any out may be NULL. */
 int moe_plan_info(moe_plan_t plan, int T, int* grid, int* stages, int* n_hw, int* smem_bytes);
 
-/* Introspection: which kernel variant T tokens get.  *fused = 1 or 2 for the fused-unit variant (1..8 tokens: a work
+/* Introspection: which kernel variant T tokens get.  *fused = 1 or 2 for the fused-unit variant (1..16 tokens: a work
  * unit is one expert's 128-wide intermediate block through gate/up AND its down-projection column block, shared by
  * the *cluster CTAs of a thread-block cluster; Section 3.2's hand-over of the intermediate tile stays on chip), 0 for
  * the general variant (*cluster = 1).  2: the launch is made in pairs (*cluster = 2) and the kernel decides after
@@ -212,7 +212,7 @@ int moe_debug_stamps(moe_plan_t plan, void* workspace, moe_stream_t stream, uint
  *                              columns in use), instead of ranges of equal length.  0 = equal length, 1..8 = strength
  *                              of the per-column term in quarters of the fitted value, -1 = the library's choice
  *                              (default: 4 from 24 tokens on, from 16 where I <= 256, else 0)
- *   MOE_KNOB_FUSED             (per token count 1..8) kernel variant: 1 = the fused-unit variant if it can run, 0 = the
+ *   MOE_KNOB_FUSED             (per token count 1..16) kernel variant: 1 = the fused-unit variant if it can run, 0 = the
  *                              general variant, -1 = the library's choice (default).  Changes the scratch layout: query
  *                              moe_workspace_bytes() again.
  *   MOE_KNOB_CLUSTER           fused-unit variant: CTAs that share one unit (thread-block cluster size) 1, 2, 4 or 8;

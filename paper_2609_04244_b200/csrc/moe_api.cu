@@ -56,6 +56,8 @@ bool encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+constexpr int kFusedMaxT = 16;      // the fused-unit variants take up to 16 tokens (one MMA N)
+
 struct WsLayout {
     size_t ctrl, e_cnt, dn_flag, pu_flag, pd_flag, flags_end;   // zero-initialised region = [0, flags_end)
     size_t stamps, logits, lpart, ids, wts, xs, xq, hq, hs, part_up, part_dn, y, stage_in, stage_out, ll, yp, xsl, total;
@@ -83,9 +85,9 @@ struct moe_plan {
     int compact_min = 9;            // fewest tokens for which the tokens are compacted per expert
     int use_pdl = 1;                // programmatic dependent launch
     int auto_stages = 1;            // stage-ring depth by default_stages() where the knob is 0 (MOE_B200_AUTO_STAGES=0: always all that fit)
-    // fused-unit variants (1..8 tokens, moe_fused_kernel.cuh)
-    int fused_knob[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // per token count 1..8: 1 = the fused variant, 0 = the general one, -1 = the library's choice
-    int cluster_knob[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // CTAs per unit for T = 1..8; 0 = the library's choice
+    // fused-unit variants (1..16 tokens, moe_fused_kernel.cuh)
+    int fused_knob[kFusedMaxT + 1];  // per token count 1..16: 1 = the fused variant, 0 = the general one, -1 = the library's choice
+    int cluster_knob[kFusedMaxT + 1];   // CTAs per unit for T = 1..16; 0 = the library's choice
     int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // clusters of that size that are co-resident at one CTA per SM (0: cannot be launched)
     int smem_per_sm = 0;
     int pairs_at_runtime = 1;       // fused variants: launches in pairs decide after routing whether the pairs share units (see fused_dyn)
@@ -95,6 +97,7 @@ struct moe_plan {
     int debug_skip = 0;             // test hook: readiness signals the kernel leaves out (see MOE_KNOB_DEBUG_SKIP)
     moe_plan() {
         for (int t = 0; t <= moe::kMaxTokens; ++t) { split_slack_kib[t] = t <= 8 ? 200 : 100; route_all_tokens[t] = 8; stages_cap[t] = 0; split_weight[t] = -1; }
+        for (int t = 0; t <= kFusedMaxT; ++t) { fused_knob[t] = -1; cluster_knob[t] = 0; }
     }
     std::mutex mu;
     std::vector<std::pair<MapKey, CUtensorMap>> maps;   // small cache of encoded descriptors
@@ -149,13 +152,13 @@ struct moe_plan {
         // fused variants: tagged router logits, and one down-projection partial per (token, slot, intermediate block)
         L.ll = o;       o += with_fused ? align_up((size_t)Tc * E * 8, 256) : 0;
         L.yp = o;       o += with_fused ? align_up((size_t)Tc * K * (I / 128) * H * 8, 256) : 0;
-        L.xsl = o;      o += with_fused ? align_up((size_t)G * 2 * 2 * 8 * 128 * 8, 256) : 0; // partial sums exported between clusters: [CTA][2 pieces][2 x 8 columns][128 rows]
+        L.xsl = o;      o += with_fused ? align_up((size_t)G * 2 * 2 * 16 * 128 * 8, 256) : 0; // partial sums exported between clusters: [CTA][2 pieces][2 x 16 columns][128 rows]
         L.total = o;
         return L;
     }
 
     // ---- fused-unit variants -------------------------------------------------------------------------------------
-    static int fused_tc(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
+    static int fused_tc(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : T <= 8 ? 8 : 16; }
     // shared memory that still lets two CTAs share an SM (the next launch's CTAs become resident under this one)
     int fused_smem_budget() const { const int half = smem_per_sm / 2 - 1024; return half < smem_optin ? half : smem_optin; }
     int fused_stages(int T) const {
@@ -194,7 +197,9 @@ struct moe_plan {
     }
     int fused_grid(int T) const { const int C = fused_cluster(T); return C ? C * max_clusters[C] : 0; }
     bool fused_possible(int T) const {
-        return T >= 1 && T <= 8 && T < compact_min && H <= 8192 && fused_cluster(T) > 0 && fused_stages(T) >= 2;
+        // (up to 8 tokens the compaction threshold of the general variant also says where the fused one may run: a
+        // caller who lowers it asks for compaction there)
+        return T >= 1 && T <= kFusedMaxT && (T > 8 || T < compact_min) && H <= 8192 && fused_cluster(T) > 0 && fused_stages(T) >= 2;
     }
     // The library's choice, by the length of the weight stream: tiles per CTA at the expected number of distinct experts.
     // The fused variant has the shorter latency chain (routing, hand-over, reduction) but its accumulator warps work
@@ -206,6 +211,10 @@ struct moe_plan {
         if (!fused_possible(T) || fused_knob[T] == 0) return false;
         if (fused_knob[T] == 1) return true;
         const double tiles = 3.0 * expected_experts(T) * (I / 128) * (H / 128) / sms;
+        // 9..16 tokens: the 16-column instantiation computes every column for every unit while the general variant
+        // compacts (an expert sees one or two of the tokens): it pays only where the whole step is a few tiles per CTA
+        // (measured: config 1 +15..18 %; the Qwen-sized layers -15..-25 %, the TP8 shards -4..+2 %)
+        if (T > 8) return tiles <= 30.0;
         return tiles <= 120.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
     }
 
@@ -422,7 +431,8 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
             case 1: return P.fsplit ? launch_fused<1, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<1, false>(p, grid, C, m13, m2, mx, P, smem, stream);
             case 2: return P.fsplit ? launch_fused<2, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<2, false>(p, grid, C, m13, m2, mx, P, smem, stream);
             case 4: return P.fsplit ? launch_fused<4, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<4, false>(p, grid, C, m13, m2, mx, P, smem, stream);
-            default: return P.fsplit ? launch_fused<8, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<8, false>(p, grid, C, m13, m2, mx, P, smem, stream);
+            case 8: return P.fsplit ? launch_fused<8, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<8, false>(p, grid, C, m13, m2, mx, P, smem, stream);
+            default: return P.fsplit ? launch_fused<16, true>(p, grid, C, m13, m2, mx, P, smem, stream) : launch_fused<16, false>(p, grid, C, m13, m2, mx, P, smem, stream);
         }
     }
     const int N = p->n_hw(T);
@@ -497,12 +507,12 @@ int moe_plan_set_knob(moe_plan_t plan, int T, int knob, int value) {
             return MOE_OK;
         case MOE_KNOB_FUSED:
             if (value < -1 || value > 1) return fail(MOE_ERR_ARG, "fused must be -1 (library's choice), 0 or 1");
-            for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->fused_knob[t] = value;
+            for (int t = (lo < 1 ? 1 : lo); t <= (hi > kFusedMaxT ? kFusedMaxT : hi); ++t) plan->fused_knob[t] = value;
             return MOE_OK;
         case MOE_KNOB_CLUSTER:
             if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return fail(MOE_ERR_ARG, "cluster size must be 0 (library's choice), 1, 2, 4 or 8");
             if (value > 0 && plan->max_clusters[value] <= 0) return fail(MOE_ERR_OCCUPANCY, "clusters of %d CTAs cannot be launched on this device", value);
-            for (int t = (lo < 1 ? 1 : lo); t <= (hi > 8 ? 8 : hi); ++t) plan->cluster_knob[t] = value;
+            for (int t = (lo < 1 ? 1 : lo); t <= (hi > kFusedMaxT ? kFusedMaxT : hi); ++t) plan->cluster_knob[t] = value;
             return MOE_OK;
         case MOE_KNOB_SPLIT_UNITS:
             if (value < 0 || value > 2) return fail(MOE_ERR_ARG, "split_units must be 0, 1 or 2");
@@ -536,8 +546,8 @@ int moe_plan_get_knob(moe_plan_t plan, int T, int knob, int* value) {
         case MOE_KNOB_COMPACT_MIN: *value = plan->compact_min; return MOE_OK;
         case MOE_KNOB_PDL: *value = plan->use_pdl; return MOE_OK;
         case MOE_KNOB_SPLIT_WEIGHT: *value = plan->split_weight[t]; return MOE_OK;
-        case MOE_KNOB_FUSED: *value = t <= 8 ? plan->fused_knob[t] : 0; return MOE_OK;
-        case MOE_KNOB_CLUSTER: *value = t <= 8 ? plan->cluster_knob[t] : 0; return MOE_OK;
+        case MOE_KNOB_FUSED: *value = t <= kFusedMaxT ? plan->fused_knob[t] : 0; return MOE_OK;
+        case MOE_KNOB_CLUSTER: *value = t <= kFusedMaxT ? plan->cluster_knob[t] : 0; return MOE_OK;
         case MOE_KNOB_STAMPS: *value = plan->take_stamps; return MOE_OK;
         case MOE_KNOB_DEBUG_SKIP: *value = plan->debug_skip; return MOE_OK;
         case MOE_KNOB_SPLIT_UNITS: *value = plan->split_units; return MOE_OK;
@@ -594,8 +604,9 @@ int moe_plan_ex(int H, int E, int I, int top_k, int scoring, int renorm, float r
     for (int C = 1; C <= 8; C *= 2) {
         const int n1 = fused_clusters<1>(C, p->smem_optin, p->sms), n2 = fused_clusters<2>(C, p->smem_optin, p->sms);
         const int n4 = fused_clusters<4>(C, p->smem_optin, p->sms), n8 = fused_clusters<8>(C, p->smem_optin, p->sms);
-        const int a = n1 < n2 ? n1 : n2, b = n4 < n8 ? n4 : n8;
-        p->max_clusters[C] = a < b ? a : b;
+        const int n16 = fused_clusters<16>(C, p->smem_optin, p->sms);
+        const int a = n1 < n2 ? n1 : n2, b = n4 < n8 ? n4 : n8, c = a < b ? a : b;
+        p->max_clusters[C] = c < n16 ? c : n16;
     }
     if (const char* v = getenv("MOE_B200_FUSED")) moe_plan_set_knob(p, 0, MOE_KNOB_FUSED, atoi(v));
     if (const char* v = getenv("MOE_B200_CLUSTER")) moe_plan_set_knob(p, 0, MOE_KNOB_CLUSTER, atoi(v));
@@ -641,7 +652,7 @@ int moe_workspace_init(moe_plan_t plan, void* workspace, size_t workspace_bytes,
         return fail(MOE_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(cudaGetLastError()));
     // Fused variants: their exchange words carry the launch tag, and the tag restarts with the control words -- so no
     // word of those regions may keep an old tag (or, in fresh memory, something that looks like one).
-    for (int T = 1; T <= 8; ++T) {
+    for (int T = 1; T <= kFusedMaxT; ++T) {
         if (!plan->fused(T)) continue;
         const WsLayout F = plan->layout(T, true);
         if (F.total > workspace_bytes) continue;             // a workspace sized for fewer tokens: that layout is never used on it

@@ -1,4 +1,4 @@
-// Fused-unit variant of the routed-MoE decode kernel for 1..8 tokens (sm_100a).
+// Fused-unit variant of the routed-MoE decode kernel for 1..16 tokens (sm_100a).
 //
 // Same operator as moe_kernel.cuh (Section 3 of the paper: top-k/quantise, up projection, down projection, reduce, in
 // one launch), laid out for the few-token case where the step is a chain of latencies rather than a stream:
@@ -41,7 +41,7 @@
 
 namespace moe {
 
-constexpr int kFusedN = 16;                                   // MMA N of the fused variants (tokens 0..7 are columns 0..7)
+constexpr int kFusedN = 16;                                   // MMA N of the fused variants (token t is column t)
 constexpr int kFusedStage = kATileBytes + kFusedN * kBlock;    // weight tile + activation tile
 constexpr int kFusedTmemBufs = 4;                              // accumulator buffers of 2 x 16 columns, one per MMA issuer
 constexpr int kFusedIssuers = 3;                               // warps 1..3
@@ -54,6 +54,7 @@ constexpr int kFusedThreads = 288;                             // 9 warps
 #else
 #define MOE_CLK() 0ll
 #endif
+constexpr int kFusedMaxTok = 16;           // token columns of the widest instantiation (= MMA N)
 constexpr int kFusedMaxRows = 4;          // router rows per CTA: ceil(kMaxExperts / 128)
 
 // ---------------------------------------------------------------------------------------------
@@ -132,7 +133,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
     L.uidx_off = o; o += E * 4;
     o = (o + 15) & ~15;
     L.xs_off = o;   o += ((T + 3) & ~3) * (H / kBlock) * 4;    // input activation scales [H/128][T rounded up to 4]
-    L.red_off = o;  o += 8 * kFusedMaxRows * 8 * 4;            // router partial dot products [warp][row][token]; later the amax scratch
+    L.red_off = o;  o += 8 * kFusedMaxRows * kFusedMaxTok * 4;  // router partial dot products [warp][row][token]; later the amax scratch
     L.poff_off = o; o += E * 4;
     L.pair_off = o; o += ((T * K * 2 + 15) & ~15);
     L.total = o;
@@ -140,7 +141,7 @@ __host__ __device__ inline FusedSmem fused_smem_layout(int TC, int T, int K, int
 }
 
 // ---------------------------------------------------------------------------------------------
-// the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8 >= T).  SPLIT = the step may have more units
+// the kernel.  TC = token columns the accumulator warps read (1, 2, 4, 8, 16 >= T).  SPLIT = the step may have more units
 // than clusters, so the code that shares a unit between two clusters is compiled in (the host knows the largest unit
 // count a token count can give; the instantiations without it are smaller and measurably faster on the short steps).
 // Warps: 0 producer (weight and activation tiles), 1..3 MMA issuers, 4..7 accumulator warps; warp 8 keeps house
@@ -264,7 +265,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             for (int t = 0; t < TC; ++t) {
 #pragma unroll
                 for (int o = 16; o; o >>= 1) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], o);
-                if (lane == 0) s_red[(warp * kFusedMaxRows + nrows) * 8 + t] = acc[t];
+                if (lane == 0) s_red[(warp * kFusedMaxRows + nrows) * kFusedMaxTok + t] = acc[t];
             }
         }
         named_bar_sync(2, kMain);
@@ -273,7 +274,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
             if (t < T) {
                 float v = 0.f;
 #pragma unroll
-                for (int w = 0; w < kMainWarps; ++w) v += s_red[(w * kFusedMaxRows + r) * 8 + t];
+                for (int w = 0; w < kMainWarps; ++w) v += s_red[(w * kFusedMaxRows + r) * kFusedMaxTok + t];
                 st_relaxed_u64(P.ll + (size_t)t * E + cta + r * G, ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v));
             }
         }
@@ -373,18 +374,28 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
         // Token t is selected by warp 7 - t: the accumulator warps come first (they have a first-tile latency to spare),
         // the producer and the issuers last.  Only the ids and the token masks are needed to start the weight stream;
         // the routing weights are computed after the barrier.
-        int my_id = 0;
-        float my_v = 0.f, my_total = 1.f;
-        const int my_t = kMainWarps - 1 - warp;
-        if (alive && my_t < T) {
-            if (E <= 128) my_id = route_pick<4>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
-            else if (E <= 256) my_id = route_pick<8>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
-            else my_id = route_pick<16>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
-            my_v = route_vals(P, lane, my_id, s_val + my_t * E, my_total);     // (the score table lies in the stage ring: read before the stream may start)
+        // (more than eight tokens: a second round; a warp then keeps two selections until the weights are computed)
+        constexpr int kRounds = (TC + kMainWarps - 1) / kMainWarps;
+        int my_id[kRounds];
+        float my_v[kRounds], my_total[kRounds];
+#pragma unroll
+        for (int r = 0; r < kRounds; ++r) {
+            my_id[r] = 0; my_v[r] = 0.f; my_total[r] = 1.f;
+            const int my_t = r * kMainWarps + kMainWarps - 1 - warp;
+            if (alive && my_t < T) {
+                if (E <= 128) my_id[r] = route_pick<4>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+                else if (E <= 256) my_id[r] = route_pick<8>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+                else my_id[r] = route_pick<16>(P, my_t, lane, s_key + my_t * E, s_ids, s_mask);
+                my_v[r] = route_vals(P, lane, my_id[r], s_val + my_t * E, my_total[r]);     // (the score table lies in the stage ring: read before the stream may start)
+            }
         }
         named_bar_sync(2, kMain);            // the selected experts and token masks of every token are in shared memory
         if (P.stamps_fine) { if (tid == 0) MOE_STAMP(4); __syncwarp(); }
-        if (alive && my_t < T) route_weights(P, my_t, lane, my_id, my_v, my_total, s_ids, s_w, cta == 0);
+#pragma unroll
+        for (int r = 0; r < kRounds; ++r) {
+            const int my_t = r * kMainWarps + kMainWarps - 1 - warp;
+            if (alive && my_t < T) route_weights(P, my_t, lane, my_id[r], my_v[r], my_total[r], s_ids, s_w, cta == 0);
+        }
     } else {
         alive = false;                       // (the housekeeping warp takes no further part)
     }
@@ -864,18 +875,29 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                                     const unsigned long long* xi = P.xsl + ((size_t)((p * 2 + pslot_x) * C) * 2 * TC) * kBlock + row;
 #pragma unroll 1
                                     for (int r = 0; r < C && okx; ++r) {
-                                        unsigned long long v[2 * TC];
-                                        unsigned pending = (1u << (2 * TC)) - 1u;
-                                        for (uint32_t it = 1; pending; ++it) {
+                                        // all 2 TC words of a source at once up to eight columns; the gate columns, then the up
+                                        // columns beyond (32 words in flight would cost 64 registers)
+                                        constexpr int kPass = (TC > 8) ? 2 : 1, kW = 2 * TC / kPass;
+#pragma unroll 1
+                                        for (int pass = 0; pass < kPass && okx; ++pass) {
+                                            unsigned long long v[kW];
+                                            unsigned pending = (1u << kW) - 1u;
+                                            for (uint32_t it = 1; pending; ++it) {
 #pragma unroll
-                                            for (int c = 0; c < 2 * TC; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + c) * kBlock);
+                                                for (int c = 0; c < kW; ++c) if (pending & (1u << c)) v[c] = ld_relaxed_u64(xi + ((size_t)r * 2 * TC + pass * kW + c) * kBlock);
 #pragma unroll
-                                            for (int c = 0; c < 2 * TC; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
-                                            if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                                for (int c = 0; c < kW; ++c) if ((pending & (1u << c)) && (unsigned)(v[c] >> 32) == tag) pending &= ~(1u << c);
+                                                if (pending && (it & 63u) == 0 && wt.expired(34)) { okx = false; break; }
+                                            }
+                                            if (!okx) break;
+                                            if (kPass == 1) {
+#pragma unroll
+                                                for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[(kW > TC ? TC : 0) + c]); }
+                                            } else {
+#pragma unroll
+                                                for (int c = 0; c < TC; ++c) { if (pass == 0) sg[c] += __uint_as_float((unsigned)v[c]); else su[c] += __uint_as_float((unsigned)v[c]); }
+                                            }
                                         }
-                                        if (!okx) break;
-#pragma unroll
-                                        for (int c = 0; c < TC; ++c) { sg[c] += __uint_as_float((unsigned)v[c]); su[c] += __uint_as_float((unsigned)v[TC + c]); }
                                     }
                                 }
                                 if (!okx) misc[3] = 1u;
@@ -890,7 +912,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
 #pragma unroll
                         for (int c = 0; c < TC; ++c) {
                             const uint32_t m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(a[c])));
-                            if (lane == 0) s_red[q * 8 + c] = __uint_as_float(m);
+                            if (lane == 0) s_red[q * kFusedMaxTok + c] = __uint_as_float(m);
                         }
                         if (!epi_all(misc[3] == 0u && !wt.dead, kEpiThreads)) { wt.dead = true; failed = true; break; }
                         const int hslot = dq & 1;
@@ -898,7 +920,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
                         uint8_t* hq = s_hq + hslot * N * kBlock;
 #pragma unroll
                         for (int c = 0; c < TC; ++c) {
-                            const float amax = fmaxf(fmaxf(s_red[c], s_red[8 + c]), fmaxf(s_red[16 + c], s_red[24 + c]));
+                            const float amax = fmaxf(fmaxf(s_red[c], s_red[kFusedMaxTok + c]), fmaxf(s_red[2 * kFusedMaxTok + c], s_red[3 * kFusedMaxTok + c]));
                             nsc[c] = fmaxf(amax, 1e-10f) * (1.0f / 448.0f);     // (the intermediate tile's scale is outside the bit-exact set)
                         }
 #pragma unroll

@@ -3,7 +3,7 @@ numerical check are rejected, the rest are ranked by CUDA-graph timing over toke
 
 The kernel's schedule knobs are those of `moe_plan_set_knob` (include/moe_b200.h): pipeline stages, the whole-unit vs
 split-K threshold, the token count up to which every CTA routes all tokens, equal-weight ranges, the compaction
-threshold and, for 1..8 tokens, the kernel variant (general or fused-unit) with the fused variant's cluster size.  For
+threshold and, for 1..16 tokens, the kernel variant (general or fused-unit) with the fused variant's cluster size.  For
 one layer shape this module times every candidate on seeded synthetic layers (the inputs of `workloads`), validates each
 candidate's output against the default schedule's output of the same step, and writes a table that
 `MoEPlan(..., schedule=table)` / `MoEPlan.apply_schedule(table)` / `bench.py --schedule FILE` apply:
@@ -37,7 +37,7 @@ PER_TOKEN_GRID = {
     "split_weight": [-1, 0, 4],
 }
 PLAN_GRID = {"compact_min": [9, 5]}
-# 1..8 tokens: the kernel variant and, for the fused-unit variant, the cluster size (0 = the library's own choice)
+# 1..16 tokens: the kernel variant and, for the fused-unit variant, the cluster size (0 = the library's own choice)
 FUSED_CLUSTERS = [0, 1, 2, 4]
 
 
@@ -97,7 +97,7 @@ def candidates(T, per_launch, fused_possible):
     grid = relevant_knobs(T, per_launch)
     names = list(grid)
     general = [dict(zip(names, combo)) for combo in itertools.product(*(grid[n] for n in names))]
-    if min(T, per_launch) > 8 or not fused_possible:
+    if min(T, per_launch) > 16 or not fused_possible:
         return general
     out = [dict(k, fused=0, cluster=0) for k in general]
     base = {n: plan_default(n, T) for n in names}

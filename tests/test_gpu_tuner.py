@@ -43,7 +43,7 @@ def test_knobs_round_trip_and_reject_bad_values():
 def test_candidates_cover_both_kernel_variants_up_to_eight_tokens():
     small = tuner.candidates(4, 64, True)
     assert any(c["fused"] == 1 and c["cluster"] == 2 for c in small) and any(c["fused"] == 0 for c in small)
-    assert all("fused" not in c for c in tuner.candidates(16, 64, True))
+    assert all("fused" not in c for c in tuner.candidates(17, 64, True))
     assert all("fused" not in c for c in tuner.candidates(4, 64, False))
 
 
