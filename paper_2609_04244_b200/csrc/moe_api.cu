@@ -161,8 +161,13 @@ struct moe_plan {
     static int fused_tc(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : T <= 8 ? 8 : 16; }
     // shared memory that still lets two CTAs share an SM (the next launch's CTAs become resident under this one)
     int fused_smem_budget() const { const int half = smem_per_sm / 2 - 1024; return half < smem_optin ? half : smem_optin; }
+    // Depth of the fused variants' stage ring when the knob is 0: all that fits -- except where a step is expected to have
+    // more units than CTAs (every CTA then works through a range of several pieces): 8.  Measured: config 2 at T = 6
+    // and 8 -1.1 and -1.5 us, Qwen3.5-35B at T=8 -1.6, config 4 at T=1 -1.2, config 2 at T=4 -0.4; with fewer units than
+    // CTAs a shallower ring loses (config 2 T=2 +0.6, DeepSeek-V3.1 TP8 T=8 +3.3, config 5 T=1 +0.4).
     int fused_stages(int T) const {
-        const int cap_s = stages_cap[T];
+        int cap_s = stages_cap[T];
+        if (cap_s <= 0 && (long long)expected_experts(T) * (I / 128) > sms) cap_s = 8;
         const int budget = smem_optin;
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s)
             if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) return s;
