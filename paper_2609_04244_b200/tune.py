@@ -39,6 +39,7 @@ PER_TOKEN_GRID = {
 PLAN_GRID = {"compact_min": [9, 5]}
 # 1..16 tokens: the kernel variant and, for the fused-unit variant, the cluster size (0 = the library's own choice)
 FUSED_CLUSTERS = [0, 1, 2, 4]
+FUSED_STAGES = [0, 8]                       # ring depth of the fused-unit variant: the library's choice, or 8
 
 
 def _layers(shape, T, regime, n_layers, device):
@@ -92,8 +93,8 @@ def relevant_knobs(T, per_launch):
 
 def candidates(T, per_launch, fused_possible):
     """Every schedule tried for T tokens, as knob dictionaries.  Up to 8 tokens the kernel variant is part of the
-    schedule: the general variant with its knobs, and the fused-unit variant with every cluster size (its other knobs
-    do not apply to it)."""
+    schedule: the general variant with its knobs, and the fused-unit variant with every cluster size and two ring
+    depths (its other knobs do not apply to it)."""
     grid = relevant_knobs(T, per_launch)
     names = list(grid)
     general = [dict(zip(names, combo)) for combo in itertools.product(*(grid[n] for n in names))]
@@ -101,7 +102,7 @@ def candidates(T, per_launch, fused_possible):
         return general
     out = [dict(k, fused=0, cluster=0) for k in general]
     base = {n: plan_default(n, T) for n in names}
-    out += [dict(base, fused=1, cluster=c) for c in FUSED_CLUSTERS]
+    out += [dict(base, fused=1, cluster=c, stages=st) for c in FUSED_CLUSTERS for st in FUSED_STAGES]
     return out
 
 
