@@ -170,7 +170,11 @@ struct moe_plan {
         if (cap_s <= 0 && (long long)expected_experts(T) * (I / 128) > sms) cap_s = 8;
         const int budget = smem_optin;
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s)
-            if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) return s;
+            if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) {
+                // (the library's own choice is an even depth: groups are pairs of tiles, and with an odd ring every other lap
+                // has a pair that wraps around its end -- config 2 at one token: 17.3 us with 10 stages, 17.7 with 11, 17.8 with 9)
+                return (stages_cap[T] <= 0 && (s & 1) && s > 2) ? s - 1 : s;
+            }
         return 0;
     }
     // Expected distinct experts of a step of T tokens under uniform routing (text after Eq. 5), rounded up.
