@@ -33,17 +33,17 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the step's kernel from the ncu
 # captures summarised under profiles/; keyed by (config, tokens).  None where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("c1_tiny", 1): 3.508e6,                         # profiles/moe_fused_kernel_c1_tiny_t1.md
-    ("c2_qwen3_30b_a3b", 1): 39.221e6 + 0.129e6,     # profiles/moe_fused_kernel_c2_qwen3_t1.md
-    ("c2_qwen3_30b_a3b", 2): 76.986e6 + 2.427e6,     # profiles/moe_fused_kernel_c2_qwen3_t2.md
-    ("c2_qwen3_30b_a3b", 4): 149.65e6 + 4.93e6,      # profiles/moe_fused_kernel_c2_qwen3_t4.md
-    ("c2_qwen3_30b_a3b", 8): 250.71e6 + 7.67e6,      # profiles/moe_fused_kernel_c2_qwen3_t8.md
-    ("c2_qwen3_30b_a3b", 16): 379.42e6 + 6.42e6,     # profiles/moe_decode_kernel_c2_qwen3_t16.md
+    ("c1_tiny", 1): 3.507e6,                         # profiles/moe_fused_kernel_c1_tiny_t1.md
+    ("c2_qwen3_30b_a3b", 1): 39.221e6 + 0.097e6,     # profiles/moe_fused_kernel_c2_qwen3_t1.md
+    ("c2_qwen3_30b_a3b", 2): 76.986e6 + 2.952e6,     # profiles/moe_fused_kernel_c2_qwen3_t2.md
+    ("c2_qwen3_30b_a3b", 4): 149.72e6 + 4.71e6,      # profiles/moe_fused_kernel_c2_qwen3_t4.md
+    ("c2_qwen3_30b_a3b", 8): 251.81e6 + 6.10e6,      # profiles/moe_fused_kernel_c2_qwen3_t8.md
+    ("c2_qwen3_30b_a3b", 16): 379.39e6 + 4.64e6,     # profiles/moe_decode_kernel_c2_qwen3_t16.md
     ("c2_qwen3_30b_a3b", 64): 601.9e6 + 5.6e6,       # profiles/moe_decode_kernel_c2_qwen3_t64.md
-    ("c4_mixtral_8x7b", 1): 366.14e6 + 5.74e6,       # profiles/moe_fused_kernel_c4_mixtral_t1.md
+    ("c4_mixtral_8x7b", 1): 365.72e6 + 5.35e6,       # profiles/moe_fused_kernel_c4_mixtral_t1.md
     ("c4_mixtral_8x7b", 64): 1416.3e6 + 6.8e6,       # profiles/moe_decode_kernel_c4_mixtral_t64.md
     ("c5_deepseek_v3[E=16]", 1): 356.76e6 + 4.67e6,  # profiles/moe_decode_kernel_c5like_e16_t1.md
-    ("c5_deepseek_v3[E=32]", 1): 353.61e6 + 5.66e6,  # profiles/moe_fused_kernel_c5like_e32_t1.md
+    ("c5_deepseek_v3[E=32]", 1): 353.59e6 + 5.62e6,  # profiles/moe_fused_kernel_c5like_e32_t1.md
     ("c5_deepseek_v3[E=64]", 8): 1680.1e6 + 4.8e6,   # profiles/moe_decode_kernel_c5like_e64_t8.md
 }
 
