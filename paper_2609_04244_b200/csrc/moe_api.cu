@@ -213,7 +213,7 @@ struct moe_plan {
     // The library's choice, by the length of the weight stream: tiles per CTA at the expected number of distinct experts.
     // The fused variant has the shorter latency chain (routing, hand-over, reduction) but its accumulator warps work
     // per group; the general variant streams longer runs at a higher rate.
-    // Measured crossover on the nine benchmark shapes (1-8 tokens): about 120 tiles per CTA; about 160 where a unit's
+    // Measured crossover on the nine benchmark shapes (1-8 tokens): about 125 tiles per CTA; about 160 where a unit's
     // down projection is at most two K blocks (there the general variant's per-unit work weighs most) and for a single
     // token.
     bool fused(int T) const {
@@ -224,7 +224,7 @@ struct moe_plan {
         // compacts (an expert sees one or two of the tokens): it pays only where the whole step is a few tiles per CTA
         // (measured: config 1 +15..18 %; the Qwen-sized layers -15..-25 %, the TP8 shards -4..+2 %)
         if (T > 8) return tiles <= 30.0;
-        return tiles <= 120.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
+        return tiles <= 125.0 || ((I / 128 <= 2 || T == 1) && tiles <= 160.0);
     }
 
     // Default depth of the stage ring when the knob is 0.  Measured (config 2 and the paper's shapes,
