@@ -167,7 +167,8 @@ struct moe_plan {
     // CTAs a shallower ring loses (config 2 T=2 +0.6, DeepSeek-V3.1 TP8 T=8 +3.3, config 5 T=1 +0.4).
     int fused_stages(int T) const {
         int cap_s = stages_cap[T];
-        if (cap_s <= 0 && (long long)expected_experts(T) * (I / 128) > sms) cap_s = 8;
+        const long long eu = (long long)expected_experts(T) * (I / 128);
+        if (cap_s <= 0 && (eu > sms || (fused_dyn(T) && long_units() && eu > sms / 2 && eu * 5 <= (long long)sms * 4))) cap_s = 8;
         const int budget = smem_optin;
         for (int s = (cap_s > 0 && cap_s < moe::kMaxStages) ? cap_s : moe::kMaxStages; s >= 2; --s)
             if (moe::fused_smem_layout(fused_tc(T), T, K, E, H, s).total + 1024 <= budget) {
@@ -198,6 +199,8 @@ struct moe_plan {
         const int C = fused_cluster_static(T), KB = H / 128;
         return (C == 1 || C == 2) && KB % 2 == 0 && max_clusters[2] * 2 == sms && max_clusters[1] == sms;
     }
+    // a unit of 60 accumulation groups and more (H/128 gate/up groups and half as many down groups)
+    bool long_units() const { return (H / 128) * 3 / 2 >= 60; }
     int fused_cluster(int T) const {
         const int KB = H / 128;
         const int knob = cluster_knob[T];
@@ -426,13 +429,13 @@ int run_step(Plan* p, int T, bool fused, const WsLayout& L, bool cache_maps, con
         moe::Params P = make_params(p, T, stages, L, w, hidden, Wr, bias, W13s, W2s, out);
         const int KB = p->H / 128;
         P.fC = C; P.fnCl = grid / C;
-        P.fdyn = p->fused_dyn(T) ? (p->fused_cluster_static(T) == 2 ? 1 : 2) : 0;
+        P.fdyn = p->fused_dyn(T) ? (p->fused_cluster_static(T) == 2 ? 1 : 2) + (p->long_units() ? 4 : 0) : 0;
         P.grid_magic1 = (1ull << 40) / (unsigned long long)grid + 1ull;
         // units are shared between clusters only where the step can have more units than clusters at all: T tokens select
         // at most min(E, T * top_k) experts (the instantiations without that code are smaller and faster)
         const int max_units = (T * p->K < p->E ? T * p->K : p->E) * (p->I / 128);
         // (pairs that may work alone: then the clusters are the CTAs)
-        P.fsplit = (p->split_units && KB % C == 0 && (max_units > (P.fdyn ? grid : P.fnCl) || p->split_units == 2)) ? p->split_units : 0;
+        P.fsplit = (p->split_units && KB % C == 0 && (max_units > ((P.fdyn && !(P.fdyn & 4)) ? grid : P.fnCl) || p->split_units == 2)) ? p->split_units : 0;
         P.grid_magic = (1ull << 40) / (unsigned long long)P.fnCl + 1ull;     // the fused kernel divides by the cluster count
         for (int r = 0; r <= C; ++r) { P.fkb[r] = r * KB / C; P.fhb[C - r] = KB - r * KB / C; }   // W2 row blocks in reverse rank order: the two shares add up evenly
         const int smem = moe::fused_smem_layout(TC, T, p->K, p->E, p->H, stages).total + 1024;

@@ -220,7 +220,7 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // clusters wait for that here (measured: starting the CTAs of a cluster in step is worth more than the wait costs);
     // a cluster of one only has to pair the arrival with a wait somewhere before the barrier's second use.
     cluster_arrive();
-    const bool late_wait = (LC == 1) || (P.fdyn == 2);          // (pairs that are expected to work alone do not meet here either)
+    const bool late_wait = (LC == 1) || ((P.fdyn & 3) == 2);          // (pairs that are expected to work alone do not meet here either)
     if (!late_wait) cluster_wait();
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -447,7 +447,10 @@ moe_fused_kernel(const __grid_constant__ CUtensorMap tmW13, const __grid_constan
     // CTAs next to each other).  The expected number of distinct experts says which it will usually be; routing that
     // crowds a few experts (8 tokens on the same 8 experts: 48 units instead of 312) gets the other arrangement
     // instead of leaving two thirds of the SMs without a unit.
-    const bool solo = (P.fdyn != 0) && (nU > nCl);
+    // (Long units -- 60 groups and more, the layers with 5120 and more hidden columns -- stay in pairs up to 80 % as many
+    // units as CTAs and cut the group list into one range per pair instead: alone, every fifth CTA or more would be
+    // without a unit while the others each stream megabytes.  Measured on the two TP8 shards at 6 and 8 tokens: 4-8 %.)
+    const bool solo = (P.fdyn != 0) && (nU > nCl) && !((P.fdyn & 4) != 0 && nU * 5 <= G * 4);
     if (solo) { C = 1; nCl = G; rank = 0; cl = cta; gmagic = P.grid_magic1; }
     const int kb_lo = solo ? 0 : P.fkb[rank], kb_hi = solo ? KBu : P.fkb[rank + 1], nk = kb_hi - kb_lo;
     const int hb_lo = solo ? 0 : P.fhb[rank], hb_hi = solo ? KBu : P.fhb[rank + 1], nh = hb_hi - hb_lo;

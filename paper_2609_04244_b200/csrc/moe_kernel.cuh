@@ -91,7 +91,7 @@ struct Params {
     unsigned long long* xsl;        // [clusters][C][2 TC][128] fused variants: partial gate/up sums a cluster exports to the next one, {launch tag, fp32 bits}
     int fsplit;                     // fused variants: cut the group list into equal ranges per cluster (units may be split between two clusters)
     int fC, fnCl;                   // fused variants: CTAs per cluster, clusters in the grid
-    int fdyn;                       // fused variants launched in pairs: nonzero = the CTAs work alone when the step has more units than pairs (1: sharing is the expected case, 2: working alone is)
+    int fdyn;                       // fused variants launched in pairs: nonzero = the CTAs work alone when the step has more units than pairs (1: sharing is the expected case, 2: working alone is; +4: long units stay in pairs up to 80 % as many units as CTAs)
     unsigned long long grid_magic1; // ... and then divide by the grid size: floor(2^40 / grid) + 1
     int fkb[9], fhb[9];             // fused variants: rank r of a cluster takes K blocks [fkb[r], fkb[r+1]) and W2 row blocks [fhb[r], fhb[r+1])
     unsigned long long* stamps;     // [grid][32] globaltimer stamps of the phases of the last launch; NULL = none taken
